@@ -1,0 +1,48 @@
+"""The workload generator reproduces the stored length lists and the SplitMix64 test vector."""
+import os
+
+from paper_2608_07524_b200 import inputs
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def read_ints(name, base=10):
+    with open(os.path.join(GOLD, name)) as f:
+        return [int(line, base) for line in f if line.strip() and not line.startswith("#")]
+
+
+def test_splitmix64_vector():
+    g = inputs.SplitMix64(0)
+    assert [g.next_u64() for _ in range(3)] == read_ints("splitmix64_seed0.txt", 16)
+
+
+def test_length_lists():
+    assert inputs.text_lengths() == read_ints("lengths_text.txt")
+    assert inputs.video_lengths() == read_ints("lengths_video.txt")
+    assert inputs.extreme_lengths() == read_ints("lengths_extreme.txt")
+    assert sum(inputs.text_lengths()) == 79299
+    assert sum(inputs.video_lengths()) == 124992
+    assert sum(inputs.extreme_lengths()) == 206646
+
+
+def test_stream_shape():
+    s = inputs.stream_batches()
+    assert len(s) == 256 and all(len(b) == 24 for b in s)
+    allowed = {256, 1024, 2048, 3328, 1200, 4800, 9600, 15600, 3600, 14400, 28800, 46800}
+    assert set(x for b in s for x in b) <= allowed
+    assert sum(map(sum, s)) == 34231792
+
+
+def test_values_are_reproducible_bf16():
+    import torch
+    a = inputs.make_qkvg(50, 2, 64, 4)
+    b = inputs.make_qkvg(50, 2, 64, 4)
+    assert all(x.dtype == torch.bfloat16 and torch.equal(x, y) for x, y in zip(a, b))
+    assert not torch.equal(a[0], a[1])
+
+
+def test_flop_convention():
+    w = inputs.config(3)
+    assert abs(w.fwd_flops() / 1e12 - 22.785) < 0.01 and abs(w.fwd_bwd_flops() / 1e12 - 79.748) < 0.03
+    w = inputs.config(2)
+    assert abs(w.fwd_bwd_flops() / 1e12 - 4.086) < 0.01

@@ -1,0 +1,168 @@
+"""Pins for the brute-force planner oracle: hand-worked answers, a second enumeration over ALL set
+partitions (a lower bound that coincides whenever grouping by length is optimal), and invariants."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden", "plan_config1.txt")
+CFG1 = [17, 64, 100, 255]
+
+
+def golden_rows():
+    with open(GOLD) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            bud, lam, K, sizes, rec, cost = line.split()
+            yield int(bud), int(lam), K, sizes, rec, cost
+
+
+def sizes_of(mb_id):
+    K = max(mb_id) + 1
+    return [mb_id.count(b) for b in range(K)]
+
+
+@pytest.mark.parametrize("row", list(golden_rows()))
+def test_hand_worked_config1(row):
+    bud, lam, K, sizes, rec, cost = row
+    kw = dict(n_heads=2, head_dim=64, n_layers=lam)
+    if K == "-":
+        with pytest.raises(oracle.Infeasible):
+            oracle.plan_bruteforce(CFG1, bud, **kw)
+        return
+    mb, r, c = oracle.plan_bruteforce(CFG1, bud, **kw)
+    assert sizes_of(mb) == [int(x) for x in sizes.split(",")]
+    assert r == [int(x) for x in rec.split(",")]
+    assert c == int(cost)
+    # micro-batch 0 holds the longest sequence (index 3)
+    assert mb[3] == 0
+
+
+def set_partitions(items):
+    if not items:
+        yield []
+        return
+    first, rest = items[0], items[1:]
+    for part in set_partitions(rest):
+        for i in range(len(part)):
+            yield part[:i] + [[first] + part[i]] + part[i + 1:]
+        yield [[first]] + part
+
+
+def block_cost(block, budget, H, d, e, lam, MC, TC):
+    """Eq. 4-6 as read in the design notes, written independently of the C oracle, in Python ints."""
+    tok = sum(block)
+    W = sum(x * x for x in block)
+    unit = tok * H * d * e
+    for r in range(lam + 1):
+        if (lam - r) * 4 * unit + lam * unit + MC <= budget:
+            return TC + 2 * r * W
+    return None
+
+
+def best_over_set_partitions(lengths, budget, **p):
+    best = None
+    for part in set_partitions(list(lengths)):
+        costs = [block_cost(b, budget, **p) for b in part]
+        if any(c is None for c in costs):
+            continue
+        tot = sum(costs)
+        best = tot if best is None or tot < best else best
+    return best
+
+
+def test_contiguous_optimum_against_all_set_partitions():
+    rng = np.random.default_rng(0)
+    gaps = 0
+    for trial in range(120):
+        n = int(rng.integers(1, 8))
+        lengths = [int(x) for x in rng.integers(1, 400, size=n)]
+        lam = int(rng.choice([1, 2, 4]))
+        TC = int(rng.choice([0, 1, 50, 10 ** 5]))
+        H, d, e = 2, 8, 2
+        unit = H * d * e
+        budget = int(rng.integers(lam * unit * max(lengths), 5 * lam * unit * sum(lengths) + 2))
+        p = dict(H=H, d=d, e=e, lam=lam, MC=0, TC=TC)
+        bound = best_over_set_partitions(lengths, budget, **p)
+        try:
+            mb, rec, cost = oracle.plan_bruteforce(lengths, budget, n_heads=H, head_dim=d, elt_bytes=e,
+                                                   n_layers=lam, fixed_cost=TC)
+        except oracle.Infeasible:
+            assert bound is None
+            continue
+        assert bound is not None and cost >= bound
+        gaps += cost > bound
+        # the returned plan is a partition, every block fits at its recompute count and the
+        # reported cost is the sum of block costs recomputed here from the formulas
+        K = len(rec)
+        assert sorted(set(mb)) == list(range(K))
+        tot = 0
+        for b in range(K):
+            block = [lengths[i] for i in range(n) if mb[i] == b]
+            c = block_cost(block, budget, **p)
+            assert c == TC + 2 * rec[b] * sum(x * x for x in block)
+            tot += c
+        assert tot == cost
+        # blocks are contiguous in the length-sorted order
+        order = sorted(range(n), key=lambda i: (-lengths[i], i))
+        ids = [mb[i] for i in order]
+        assert ids == sorted(ids)
+    # grouping by length is usually but not always optimal; the test must have seen both
+    assert gaps < 40
+
+
+def test_invariants():
+    rng = np.random.default_rng(1)
+    lengths = [int(x) for x in rng.integers(1, 3000, size=10)]
+    kw = dict(n_heads=4, head_dim=32, n_layers=3, fixed_cost=12345)
+    unit = 4 * 32 * 2
+    big = (4 * 3 + 3) * unit * sum(lengths)
+    mb, rec, cost = oracle.plan_bruteforce(lengths, big, **kw)
+    assert set(mb) == {0} and rec == [0] and cost == 12345        # everything fits: one block, r = 0
+    prev = None
+    for budget in sorted(int(x) for x in rng.integers(3 * unit * max(lengths), big, size=12)):
+        _, _, c = oracle.plan_bruteforce(lengths, budget, **kw)
+        assert prev is None or c <= prev                           # more memory never costs more
+        prev = c
+    # permuting the input permutes mb_id and leaves the cost unchanged
+    budget = 6 * unit * max(lengths)
+    mb, rec, cost = oracle.plan_bruteforce(lengths, budget, **kw)
+    perm = rng.permutation(len(lengths))
+    mb2, rec2, cost2 = oracle.plan_bruteforce([lengths[i] for i in perm], budget, **kw)
+    assert cost2 == cost and rec2 == rec
+    assert sorted(zip([lengths[i] for i in perm], mb2)) == sorted(zip(lengths, mb))
+    # T_C = 0: the cost is exactly the forced recomputation
+    mb, rec, cost = oracle.plan_bruteforce(lengths, budget, **{**kw, "fixed_cost": 0})
+    assert cost == sum(2 * rec[b] * sum(l * l for l, m in zip(lengths, mb) if m == b) for b in range(len(rec)))
+
+
+def test_full_recompute_time_matches_profiling_estimate():
+    # Section 3.5: with every layer recomputed the model time is Lambda * (2 t_f + t_b) + T_C.
+    # In this reading t_f = 2W, t_b = 5W, so cost + Lambda*7W must equal Lambda*(2*2W + 5W) + T_C.
+    lengths, lam, TC = [100, 50], 3, 10 ** 9     # T_C large enough that one block wins
+    unit = 2 * 8 * 2
+    budget = lam * unit * 150            # only r = Lambda fits
+    mb, rec, cost = oracle.plan_bruteforce(lengths, budget, n_heads=2, head_dim=8, n_layers=lam, fixed_cost=TC)
+    W = 100 * 100 + 50 * 50
+    assert rec == [lam] and cost + lam * 7 * W == lam * (2 * 2 * W + 5 * W) + TC
+
+
+def test_tie_break_prefers_fewer_then_front_loaded_blocks():
+    # T_C = 0 and a budget where nothing needs recompute in blocks of <= 2: many plans cost 0.
+    # Fewest blocks first; among equal counts the first block is as large as possible.
+    lengths = [10, 10, 10, 10, 10]
+    unit = 1 * 8 * 2
+    budget = 5 * unit * 20               # two sequences fit at r = 0, three do not
+    mb, rec, cost = oracle.plan_bruteforce(lengths, budget, n_heads=1, head_dim=8, n_layers=1, fixed_cost=0)
+    assert cost == 0 and rec == [0, 0, 0]
+    assert mb == [0, 0, 1, 1, 2]
+
+
+def test_rejects_bad_arguments():
+    with pytest.raises(ValueError):
+        oracle.plan_bruteforce([0, 5], 1000)
+    with pytest.raises(ValueError):
+        oracle.plan_bruteforce([5] * 25, 10 ** 12)
