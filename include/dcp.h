@@ -1,0 +1,120 @@
+/*
+ * dcp.h - C ABI of the B200 (sm_100a) packed variable-length attention library and of the
+ * single-GPU micro-batch / recomputation planner.
+ *
+ * All entry points return an int status (DCP_OK = 0).  No exception crosses this boundary and no
+ * entry point below allocates device memory: every buffer, the workspace included, belongs to the
+ * caller.  On any error the outputs are left untouched and dcp_last_error() gives a message.
+ *
+ * Tensor layout: q, k, v, o, d_o, dq, dk, dv are bf16, shape [total_tokens, n_heads, head_dim],
+ * contiguous, sequences packed back to back; sequence b owns tokens cu_seqlens[b] ..
+ * cu_seqlens[b+1]-1.  lse is fp32, shape [n_heads, total_tokens].  Device pointers must be
+ * 16-byte aligned.  Supported head_dim: 64 and 128.  n_heads is the same for q, k and v.
+ */
+#ifndef DCP_H_
+#define DCP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    DCP_OK = 0,
+    DCP_ERR_INVALID_ARG = 1, /* null pointer, negative size, misaligned pointer, ...            */
+    DCP_ERR_INFEASIBLE = 2,  /* planner: one sequence exceeds the budget even at full recompute */
+    DCP_ERR_UNSUPPORTED = 3, /* head_dim not 64/128, device is not sm_100                       */
+    DCP_ERR_WORKSPACE = 4,   /* workspace missing or smaller than dcp_varlen_attn_workspace     */
+    DCP_ERR_CUDA = 5,        /* a CUDA runtime/driver call or a launch failed                   */
+    DCP_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired (see dcp_query_status)       */
+    DCP_ERR_OVERFLOW = 7     /* planner: a quantity does not fit in int64                       */
+};
+
+/* ---------------------------------------------------------------------------------------------
+ * Planner.
+ *
+ * Paper: Section 3.2 (problem statement; here at sequence-parallel size p = 1, so only the
+ * throughput target Eq. 1 remains), Section 3.4 Eq. 4-6 (time and memory of a batch with r
+ * recomputed layers) and the inner rule of Algorithm 1 (smallest recompute count that fits the
+ * memory capacity); Section 3.1 (sequences of similar length are grouped).
+ *
+ * Splits one batch of sequences into gradient-accumulation micro-batches and picks, per
+ * micro-batch, how many layers recompute their forward pass, minimising modelled time under an
+ * HBM budget.  Indices are sorted by (length descending, index ascending); a plan is a split of
+ * that order into contiguous blocks.  For a block with tok = sum L and W = sum L^2:
+ *     m = 4*tok*H*d*e,  m_inp = tok*H*d*e,  mem(r) = (Lambda-r)*m + Lambda*m_inp + M_C,
+ *     r* = smallest r in [0, Lambda] with mem(r) <= budget,
+ *     time = Lambda*7*W + r* * 2*W + T_C.
+ * Returned cost = K*T_C + 2*sum_k r*_k W_k (the plan-independent part is dropped).  Ties: fewer
+ * micro-batches, then the lexicographically largest block-size vector.
+ * Host pointers throughout; runs on the host only; integer arithmetic only (int64, checked).
+ */
+typedef struct {
+    int32_t n_heads;     /* H, >= 1 */
+    int32_t head_dim;    /* d, >= 1 */
+    int32_t elt_bytes;   /* e, >= 1 (2 for bf16) */
+    int32_t n_layers;    /* Lambda, >= 1; with 1 the recompute count is a 0/1 flag */
+    int64_t const_bytes; /* M_C >= 0 */
+    int64_t fixed_cost;  /* T_C >= 0, in units of one L^2 product over all heads */
+} dcp_plan_params;
+
+/* params == NULL selects H = 16, d = 128, e = 2, Lambda = 1, M_C = 0, T_C = 2^24.
+ * lengths [n] (each >= 1), n >= 1.  Outputs: mb_id [n] = micro-batch of each INPUT index
+ * (micro-batch 0 holds the longest sequence); *n_mb = K; recompute [n], first K entries valid;
+ * cost (nullable). */
+int dcp_plan(const int32_t* lengths, int32_t n, int64_t hbm_budget_bytes, const dcp_plan_params* params,
+             int32_t* mb_id, int32_t* n_mb, int32_t* recompute, int64_t* cost);
+
+/* ---------------------------------------------------------------------------------------------
+ * Attention.
+ *
+ * Paper: Section 4.1 ("Implementation details": a fused attention library is enabled in every
+ * run) and Section 4.2 ("Effect of model architecture": attention time dominates).  The paper
+ * gives no formula; the operation is softmax(Q K^T * scale + mask) V per sequence and head, with
+ * key j visible to query i iff (not causal) or j <= i, indices relative to the sequence start.
+ * lse_i = ln sum_j exp(scale * q_i.k_j) over visible keys (natural log).
+ *
+ * Both calls only enqueue work on `cuda_stream` (a cudaStream_t; NULL = the default stream);
+ * they neither synchronise nor read cu_seqlens on the host.  softmax_scale = 0 selects
+ * 1/sqrt(head_dim).  Zero-length sequences are legal.  max_seqlen must be >= every length.
+ */
+
+/* Bytes of caller-provided device workspace needed by the forward and the backward call. */
+int dcp_varlen_attn_workspace(int32_t total_tokens, int32_t n_seqs, int32_t n_heads, int32_t head_dim,
+                              size_t* fwd_bytes, size_t* bwd_bytes);
+
+/* q, k, v (device, in) -> o, lse (device, out).  workspace: device, >= fwd_bytes, 256-byte
+ * aligned; its first word is a status word that dcp_query_status reads. */
+int dcp_varlen_attn_fwd(const void* q, const void* k, const void* v, const int32_t* cu_seqlens, int32_t n_seqs,
+                        int32_t total_tokens, int32_t max_seqlen, int32_t n_heads, int32_t head_dim,
+                        int32_t causal, float softmax_scale, void* o, float* lse, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream);
+
+/* Gradients of sum(o * d_o): q, k, v, o, d_o, lse (device, in) -> dq, dk, dv (device, out).
+ * `causal` and `softmax_scale` must equal the forward call's.  workspace >= bwd_bytes; it holds
+ * the fp32 dQ accumulator and the per-row D = sum_c dO*O.  dQ is summed with floating-point
+ * atomics, so its low bits may differ from run to run. */
+int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                        const float* lse, const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens,
+                        int32_t max_seqlen, int32_t n_heads, int32_t head_dim, int32_t causal,
+                        float softmax_scale, void* dq, void* dk, void* dv, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream);
+
+/* Synchronises `cuda_stream`, then reads the status word at the start of `workspace`.
+ * Returns DCP_OK, DCP_ERR_TIMEOUT (a kernel abandoned a bounded wait; results are invalid) or
+ * DCP_ERR_CUDA. */
+int dcp_query_status(const void* workspace, void* cuda_stream);
+
+/* Number of kernel launches this library has enqueued since it was loaded (all threads). */
+int64_t dcp_launch_count(void);
+
+/* Message for the last error on the calling thread ("" if none). The pointer stays valid until
+ * the thread's next failing call. */
+const char* dcp_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DCP_H_ */

@@ -1,0 +1,262 @@
+// C ABI of libdcp: argument checks, tensor-map construction, workspace carving and kernel launches.
+// Definitions of every operation are in include/dcp.h.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <mutex>
+
+#include "../../include/dcp.h"
+#include "attn_kernels.h"
+#include "dcp_internal.h"
+#include "sched.cuh"
+
+namespace dcp {
+
+char* error_buffer() {
+    static thread_local char buf[512] = "";
+    return buf;
+}
+
+namespace {
+
+std::atomic<int64_t> g_launches{0};
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver entry point is looked up at run time so that the library loads (and the planner
+// works) on machines without a CUDA driver.
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+struct DeviceInfo {
+    int device = -1;
+    int sm_count = 0;
+    int cc_major = 0;
+};
+
+// Properties of the current device, cached per device id.
+int device_info(DeviceInfo* out) {
+    static std::mutex mu;
+    static DeviceInfo cache[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return fail(DCP_ERR_CUDA, "cudaGetDevice failed (no CUDA device?)");
+    if (dev < 0 || dev >= 64) return fail(DCP_ERR_CUDA, "device index %d out of range", dev);
+    std::lock_guard<std::mutex> lock(mu);
+    if (cache[dev].device != dev) {
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return fail(DCP_ERR_CUDA, "cudaGetDeviceProperties failed");
+        cache[dev].device = dev;
+        cache[dev].sm_count = prop.multiProcessorCount;
+        cache[dev].cc_major = prop.major;
+    }
+    *out = cache[dev];
+    return DCP_OK;
+}
+
+// [T, H, d] bf16 viewed as a 3-D tensor (d, H, T); a box is 64 columns x 1 head x 128 tokens,
+// written to shared memory as 128 rows of 128 bytes with the 128-byte swizzle.  Rows past T are
+// zero-filled.
+int make_map(CUtensorMap* map, const void* base, int32_t total_tokens, int32_t n_heads, int32_t head_dim) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return fail(DCP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the CUDA driver");
+    const cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)n_heads, (cuuint64_t)total_tokens};
+    const cuuint64_t strides[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)n_heads * head_dim * 2};
+    const cuuint32_t box[3] = {64, 1, (cuuint32_t)kTile};
+    const cuuint32_t elem_strides[3] = {1, 1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+                           elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(DCP_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+    return DCP_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(const char* fn, int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen, int32_t n_heads,
+                int32_t head_dim, float softmax_scale) {
+    if (n_seqs < 0 || total_tokens < 0 || max_seqlen < 0 || n_heads < 1)
+        return fail(DCP_ERR_INVALID_ARG, "%s: negative size or n_heads < 1", fn);
+    if (n_seqs > 65535) return fail(DCP_ERR_UNSUPPORTED, "%s: at most 65535 sequences per call", fn);
+    if (n_heads > 65535) return fail(DCP_ERR_UNSUPPORTED, "%s: at most 65535 heads", fn);
+    if (head_dim != 64 && head_dim != 128)
+        return fail(DCP_ERR_UNSUPPORTED, "%s: head_dim %d is not supported (64 or 128)", fn, head_dim);
+    if (max_seqlen > total_tokens) return fail(DCP_ERR_INVALID_ARG, "%s: max_seqlen exceeds total_tokens", fn);
+    if (!(softmax_scale >= 0.f) || std::isinf(softmax_scale))
+        return fail(DCP_ERR_INVALID_ARG, "%s: softmax_scale must be finite and >= 0 (0 selects 1/sqrt(d))", fn);
+    if ((int64_t)total_tokens * n_heads >= ((int64_t)1 << 31))
+        return fail(DCP_ERR_UNSUPPORTED, "%s: total_tokens * n_heads must be below 2^31", fn);
+    return DCP_OK;
+}
+
+SchedView carve_sched(void* workspace, int32_t n_seqs) {
+    SchedView s;
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    s.hdr = reinterpret_cast<WorkspaceHeader*>(base);
+    s.order = reinterpret_cast<const int32_t*>(base + sizeof(WorkspaceHeader));
+    s.prefix = reinterpret_cast<const uint32_t*>(base + sizeof(WorkspaceHeader) + sizeof(int32_t) * (size_t)n_seqs);
+    s.n_seqs = n_seqs;
+    return s;
+}
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+}  // namespace
+}  // namespace dcp
+
+using namespace dcp;
+
+extern "C" const char* dcp_last_error(void) { return error_buffer(); }
+
+extern "C" int64_t dcp_launch_count(void) { return g_launches.load(); }
+
+extern "C" int dcp_varlen_attn_workspace(int32_t total_tokens, int32_t n_seqs, int32_t n_heads, int32_t head_dim,
+                                         size_t* fwd_bytes, size_t* bwd_bytes) {
+    if (total_tokens < 0 || n_seqs < 0 || n_heads < 1 || head_dim < 1)
+        return fail(DCP_ERR_INVALID_ARG, "dcp_varlen_attn_workspace: bad sizes");
+    const size_t sched = sched_bytes(n_seqs);
+    if (fwd_bytes) *fwd_bytes = sched;
+    if (bwd_bytes)
+        *bwd_bytes = sched + align256(sizeof(float) * (size_t)total_tokens * n_heads) +
+                     align256(sizeof(float) * (size_t)total_tokens * n_heads * head_dim);
+    return DCP_OK;
+}
+
+extern "C" int dcp_varlen_attn_fwd(const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
+                                   int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen, int32_t n_heads,
+                                   int32_t head_dim, int32_t causal, float softmax_scale, void* o, float* lse,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    const char* fn = "dcp_varlen_attn_fwd";
+    if (int rc = check_shape(fn, n_seqs, total_tokens, max_seqlen, n_heads, head_dim, softmax_scale)) return rc;
+    if (!cu_seqlens) return fail(DCP_ERR_INVALID_ARG, "%s: cu_seqlens is null", fn);
+    if (!workspace) return fail(DCP_ERR_WORKSPACE, "%s: workspace is null", fn);
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+        return fail(DCP_ERR_WORKSPACE, "%s: workspace must be 256-byte aligned", fn);
+    if (workspace_bytes < sched_bytes(n_seqs))
+        return fail(DCP_ERR_WORKSPACE, "%s: workspace has %zu bytes, needs %zu", fn, workspace_bytes, sched_bytes(n_seqs));
+    if (total_tokens > 0 && (!q || !k || !v || !o || !lse)) return fail(DCP_ERR_INVALID_ARG, "%s: null tensor pointer", fn);
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o))
+        return fail(DCP_ERR_INVALID_ARG, "%s: tensor pointers must be 16-byte aligned", fn);
+    DeviceInfo dev;
+    if (int rc = device_info(&dev)) return rc;
+    if (dev.cc_major != 10) return fail(DCP_ERR_UNSUPPORTED, "%s: this library runs on sm_100 devices only", fn);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    const SchedView sched = carve_sched(workspace, n_seqs);
+    cudaError_t e = launch_prep(cu_seqlens, n_seqs, kFwdRowsPerItem, n_heads, sched, stream);
+    if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: work-list kernel: %s", fn, cudaGetErrorString(e));
+    g_launches.fetch_add(1);
+    if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
+
+    CUtensorMap tq, tk, tv;
+    if (int rc = make_map(&tq, q, total_tokens, n_heads, head_dim)) return rc;
+    if (int rc = make_map(&tk, k, total_tokens, n_heads, head_dim)) return rc;
+    if (int rc = make_map(&tv, v, total_tokens, n_heads, head_dim)) return rc;
+
+    FwdParams p;
+    p.cu_seqlens = cu_seqlens;
+    p.o = static_cast<__nv_bfloat16*>(o);
+    p.lse = lse;
+    p.sched = sched;
+    p.n_heads = n_heads;
+    p.total_tokens = total_tokens;
+    p.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
+    p.scale_log2 = p.scale * 1.4426950408889634f;
+    e = launch_attn_fwd(tq, tk, tv, p, head_dim, causal != 0, dev.sm_count, stream);
+    if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: attention kernel: %s", fn, cudaGetErrorString(e));
+    g_launches.fetch_add(1);
+    return DCP_OK;
+}
+
+extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                                   const float* lse, const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens,
+                                   int32_t max_seqlen, int32_t n_heads, int32_t head_dim, int32_t causal,
+                                   float softmax_scale, void* dq, void* dk, void* dv, void* workspace,
+                                   size_t workspace_bytes, void* cuda_stream) {
+    const char* fn = "dcp_varlen_attn_bwd";
+    if (int rc = check_shape(fn, n_seqs, total_tokens, max_seqlen, n_heads, head_dim, softmax_scale)) return rc;
+    if (!cu_seqlens) return fail(DCP_ERR_INVALID_ARG, "%s: cu_seqlens is null", fn);
+    if (!workspace) return fail(DCP_ERR_WORKSPACE, "%s: workspace is null", fn);
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+        return fail(DCP_ERR_WORKSPACE, "%s: workspace must be 256-byte aligned", fn);
+    size_t need = 0;
+    dcp_varlen_attn_workspace(total_tokens, n_seqs, n_heads, head_dim, nullptr, &need);
+    if (workspace_bytes < need) return fail(DCP_ERR_WORKSPACE, "%s: workspace has %zu bytes, needs %zu", fn, workspace_bytes, need);
+    if (total_tokens > 0 && (!q || !k || !v || !o || !d_o || !lse || !dq || !dk || !dv))
+        return fail(DCP_ERR_INVALID_ARG, "%s: null tensor pointer", fn);
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(dq) ||
+        !aligned16(dk) || !aligned16(dv))
+        return fail(DCP_ERR_INVALID_ARG, "%s: tensor pointers must be 16-byte aligned", fn);
+    DeviceInfo dev;
+    if (int rc = device_info(&dev)) return rc;
+    if (dev.cc_major != 10) return fail(DCP_ERR_UNSUPPORTED, "%s: this library runs on sm_100 devices only", fn);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    const SchedView sched = carve_sched(workspace, n_seqs);
+    uint8_t* base = static_cast<uint8_t*>(workspace) + sched_bytes(n_seqs);
+    float* dsum = reinterpret_cast<float*>(base);
+    float* dq_acc = reinterpret_cast<float*>(base + align256(sizeof(float) * (size_t)total_tokens * n_heads));
+
+    cudaError_t e = launch_prep(cu_seqlens, n_seqs, kTile, n_heads, sched, stream);
+    if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: work-list kernel: %s", fn, cudaGetErrorString(e));
+    g_launches.fetch_add(1);
+    if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
+
+    CUtensorMap tq, tk, tv, tg;
+    if (int rc = make_map(&tq, q, total_tokens, n_heads, head_dim)) return rc;
+    if (int rc = make_map(&tk, k, total_tokens, n_heads, head_dim)) return rc;
+    if (int rc = make_map(&tv, v, total_tokens, n_heads, head_dim)) return rc;
+    if (int rc = make_map(&tg, d_o, total_tokens, n_heads, head_dim)) return rc;
+
+    e = launch_bwd_pre(static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), dsum, dq_acc,
+                       total_tokens, n_heads, head_dim, stream);
+    if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: pre kernel: %s", fn, cudaGetErrorString(e));
+    g_launches.fetch_add(1);
+
+    BwdParams p;
+    p.cu_seqlens = cu_seqlens;
+    p.lse = lse;
+    p.dsum = dsum;
+    p.dq_acc = dq_acc;
+    p.dk = static_cast<__nv_bfloat16*>(dk);
+    p.dv = static_cast<__nv_bfloat16*>(dv);
+    p.sched = sched;
+    p.n_heads = n_heads;
+    p.total_tokens = total_tokens;
+    p.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
+    p.scale_log2 = p.scale * 1.4426950408889634f;
+    e = launch_attn_bwd(tq, tk, tv, tg, p, head_dim, causal != 0, dev.sm_count, stream);
+    if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: main kernel: %s", fn, cudaGetErrorString(e));
+    g_launches.fetch_add(1);
+
+    e = launch_bwd_post(dq_acc, static_cast<__nv_bfloat16*>(dq), (size_t)total_tokens * n_heads * head_dim, p.scale, stream);
+    if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: post kernel: %s", fn, cudaGetErrorString(e));
+    g_launches.fetch_add(1);
+    return DCP_OK;
+}
+
+extern "C" int dcp_query_status(const void* workspace, void* cuda_stream) {
+    if (!workspace) return fail(DCP_ERR_INVALID_ARG, "dcp_query_status: workspace is null");
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint32_t status = 0;
+    cudaError_t e = cudaMemcpyAsync(&status, workspace, sizeof status, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "dcp_query_status: %s", cudaGetErrorString(e));
+    if (status != 0) return fail(DCP_ERR_TIMEOUT, "a kernel abandoned a bounded wait (device status %u); results are invalid", status);
+    return DCP_OK;
+}

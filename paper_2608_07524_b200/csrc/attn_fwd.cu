@@ -1,0 +1,388 @@
+// Forward packed variable-length attention for sm_100a.
+//
+// One persistent CTA per SM.  A work item is (sequence, head, 256 query rows) = two 128-row Q
+// tiles.  Roles:
+//   warps 0-3   softmax group 0 (Q tile 0): one thread per query row
+//   warps 4-7   softmax group 1 (Q tile 1)
+//   warp  8     MMA issue (one thread): S_t = Q_t K_j^T and O_t += P_t V_j with tcgen05, fp32
+//               accumulators in tensor memory
+//   warp  9     scheduler + TMA producer (one thread): pulls work items from the global counter,
+//               streams Q once and K_j, V_j through a shared-memory ring
+// The two Q tiles alternate on the tensor pipe: while one group runs exp on its S tile, the pipe
+// computes the other tile's products.  P overwrites S in tensor memory as packed bf16 and is the
+// A operand of the second product, so probabilities never touch shared memory.
+//
+// Softmax is the online form: a running row maximum m and sum l; the maximum is only raised when
+// it grew by more than 2^8, which keeps exp2 arguments bounded while making rescales of the O
+// accumulator rare.  Results: O = acc / l (bf16), lse = m*scale + ln l (fp32).
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "attn_kernels.h"
+#include "sched.cuh"
+#include "sm100_ptx.cuh"
+
+namespace dcp {
+
+constexpr int kFwdThreads = 320;
+constexpr int kKvStages = 4;
+constexpr float kRescaleThreshold = 8.0f;   // in log2 units
+
+struct FwdShared {
+    uint64_t q_full[2], q_empty[2];
+    uint64_t kv_full[kKvStages], kv_empty[kKvStages];
+    uint64_t s_full[2], p_full[2], o_full[2], o_free[2];
+    uint64_t work_full[2], work_empty[2];
+    WorkItem work[2];
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+
+template <int D>
+struct FwdCfg {
+    static constexpr int kTileBytes = kTile * D * 2;   // one Q, K or V tile
+    static constexpr int kBoxes = D / 64;               // TMA boxes per tile (64 columns = 128 bytes each)
+    static constexpr int kBoxBytes = kTile * 128;
+    static constexpr int kSmemBytes = (2 + kKvStages) * kTileBytes + 1024;
+    static constexpr uint32_t kS0 = 0, kS1 = 128, kO0 = 256, kO1 = 256 + D;   // tensor-memory columns
+};
+
+// Number of K/V tiles a Q tile starting at row r0 attends to (0 if the tile is past the end).
+template <bool CAUSAL>
+__device__ __forceinline__ int kv_tiles_for(int r0, int len) {
+    if (r0 >= len) return 0;
+    const int all = (len + kTile - 1) / kTile;
+    if (!CAUSAL) return all;
+    const int diag = r0 / kTile + 1;
+    return diag < all ? diag : all;
+}
+
+template <int D>
+__device__ __forceinline__ void load_tile(uint8_t* dst, const CUtensorMap* map, uint64_t* bar, int head, int row) {
+    mbar_expect_tx(bar, FwdCfg<D>::kTileBytes);
+#pragma unroll
+    for (int b = 0; b < FwdCfg<D>::kBoxes; ++b)
+        tma_load_3d(dst + b * FwdCfg<D>::kBoxBytes, map, bar, b * 64, head, row);
+}
+
+// S = Q K^T for one 128x128 tile: both operands K-contiguous in shared memory.
+template <int D>
+__device__ __forceinline__ void issue_qk(uint32_t d_tmem, uint32_t q_addr, uint32_t k_addr) {
+    constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, false);
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+        const uint32_t off = (ks / 4) * FwdCfg<D>::kBoxBytes + (ks % 4) * 32;
+        tc_mma_ss(d_tmem, make_sdesc_sw128(q_addr + off, 16, 1024), make_sdesc_sw128(k_addr + off, 16, 1024), idesc,
+                  ks > 0);
+    }
+}
+
+// O (+)= P V: P from tensor memory (bf16 pairs per column), V with head_dim contiguous.
+template <int D>
+__device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint32_t v_addr, bool accumulate) {
+    constexpr uint32_t idesc = make_idesc_bf16(128, D, false, true);
+#pragma unroll
+    for (int ks = 0; ks < kTile / 16; ++ks)
+        tc_mma_ts(d_tmem, p_tmem + ks * 8, make_sdesc_sw128(v_addr + ks * 2048, FwdCfg<D>::kBoxBytes, 1024), idesc,
+                  accumulate || ks > 0);
+}
+
+template <int D, bool CAUSAL>
+__global__ void __launch_bounds__(kFwdThreads, 1)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                const __grid_constant__ CUtensorMap tmap_v, const FwdParams p) {
+    using Cfg = FwdCfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sQ = smem;
+    uint8_t* sKV = smem + 2 * Cfg::kTileBytes;
+    __shared__ FwdShared sh;
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const WaitGuard guard{&sh.abort_flag, &p.sched.hdr->status};
+
+    if (tid == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&sh.q_full[i], 1);
+            mbar_init(&sh.q_empty[i], 1);
+            mbar_init(&sh.s_full[i], 1);
+            mbar_init(&sh.p_full[i], 4);       // one arrival per softmax warp
+            mbar_init(&sh.o_full[i], 1);
+            mbar_init(&sh.o_free[i], 4);
+            mbar_init(&sh.work_full[i], 1);
+            mbar_init(&sh.work_empty[i], 9);   // 8 softmax warps + the MMA thread
+        }
+        for (int i = 0; i < kKvStages; ++i) {
+            mbar_init(&sh.kv_full[i], 1);
+            mbar_init(&sh.kv_empty[i], 1);
+        }
+        sh.abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(&sh.tmem_base, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh.tmem_base;
+
+    if (warp == 9) {
+        // ---------------------------------------------------------------- scheduler + TMA producer
+        if (lane == 0) {
+            tma_prefetch_desc(&tmap_q);
+            tma_prefetch_desc(&tmap_k);
+            tma_prefetch_desc(&tmap_v);
+            const uint32_t n_items = p.sched.hdr->n_items;
+            uint32_t n_work = 0, kv_count = 0, q_use[2] = {0, 0};
+            while (true) {
+                const uint32_t slot = n_work & 1u;
+                if (n_work >= 2) mbar_wait(&sh.work_empty[slot], ((n_work >> 1) - 1) & 1u, guard);
+                const uint32_t item = atomicAdd(&p.sched.hdr->work_counter, 1u);
+                WorkItem w;
+                if (item < n_items && !sh.abort_flag) {
+                    w = decode_item(p.sched, p.cu_seqlens, item, kFwdRowsPerItem, p.n_heads, CAUSAL);
+                } else {
+                    w.tok0 = 0; w.len = -1; w.head = 0; w.blk = 0;
+                }
+                sh.work[slot] = w;
+                mbar_arrive(&sh.work_full[slot]);
+                ++n_work;
+                if (w.len < 0) break;
+
+                const int r0 = w.blk * kFwdRowsPerItem;
+                const int nkv_t[2] = {kv_tiles_for<CAUSAL>(r0, w.len), kv_tiles_for<CAUSAL>(r0 + kTile, w.len)};
+                const int nkv = nkv_t[0] > nkv_t[1] ? nkv_t[0] : nkv_t[1];
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (nkv_t[t] == 0) continue;
+                    if (q_use[t] >= 1) mbar_wait(&sh.q_empty[t], (q_use[t] - 1) & 1u, guard);
+                    load_tile<D>(sQ + t * Cfg::kTileBytes, &tmap_q, &sh.q_full[t], w.head, w.tok0 + r0 + t * kTile);
+                    ++q_use[t];
+                }
+                for (int j = 0; j < nkv; ++j) {
+#pragma unroll
+                    for (int which = 0; which < 2; ++which) {
+                        const uint32_t stage = kv_count % kKvStages, fill = kv_count / kKvStages;
+                        if (fill >= 1) mbar_wait(&sh.kv_empty[stage], (fill - 1) & 1u, guard);
+                        load_tile<D>(sKV + stage * Cfg::kTileBytes, which == 0 ? &tmap_k : &tmap_v, &sh.kv_full[stage],
+                                     w.head, w.tok0 + j * kTile);
+                        ++kv_count;
+                    }
+                }
+            }
+        }
+    } else if (warp == 8) {
+        // ---------------------------------------------------------------- MMA issue
+        if (lane == 0) {
+            uint32_t n_work = 0, kv_base = 0, use[2] = {0, 0}, n_p[2] = {0, 0};
+            const uint32_t q_addr[2] = {smem_u32(sQ), smem_u32(sQ) + Cfg::kTileBytes};
+            const uint32_t kv_addr = smem_u32(sKV);
+            const uint32_t s_tmem[2] = {tmem + Cfg::kS0, tmem + Cfg::kS1};
+            const uint32_t o_tmem[2] = {tmem + Cfg::kO0, tmem + Cfg::kO1};
+            auto kv_wait = [&](uint32_t idx) {
+                mbar_wait(&sh.kv_full[idx % kKvStages], (idx / kKvStages) & 1u, guard);
+            };
+            auto kv_smem = [&](uint32_t idx) { return kv_addr + (idx % kKvStages) * Cfg::kTileBytes; };
+            while (true) {
+                const uint32_t slot = n_work & 1u;
+                if (!mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard)) break;
+                const WorkItem w = sh.work[slot];
+                mbar_arrive(&sh.work_empty[slot]);
+                ++n_work;
+                if (w.len < 0) break;
+                const int r0 = w.blk * kFwdRowsPerItem;
+                const int nkv_t[2] = {kv_tiles_for<CAUSAL>(r0, w.len), kv_tiles_for<CAUSAL>(r0 + kTile, w.len)};
+                const int nkv = nkv_t[0] > nkv_t[1] ? nkv_t[0] : nkv_t[1];
+
+                // S_t(0) for both tiles
+                kv_wait(kv_base);
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (nkv_t[t] == 0) continue;
+                    mbar_wait(&sh.q_full[t], use[t] & 1u, guard);
+                    tc_fence_after();
+                    issue_qk<D>(s_tmem[t], q_addr[t], kv_smem(kv_base));
+                    tc_commit(&sh.s_full[t]);
+                }
+                tc_commit(&sh.kv_empty[kv_base % kKvStages]);
+
+                for (int j = 0; j < nkv; ++j) {
+                    const uint32_t iv = kv_base + 2 * j + 1, ik = kv_base + 2 * j + 2;
+                    const bool has_next = j + 1 < nkv;
+                    kv_wait(iv);
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        if (t == 1 && has_next) kv_wait(ik);
+                        if (t == 1 && j + 1 < nkv_t[0]) {      // S_0(j+1) goes between the two PV products
+                            tc_fence_after();
+                            issue_qk<D>(s_tmem[0], q_addr[0], kv_smem(ik));
+                            tc_commit(&sh.s_full[0]);
+                        }
+                        if (j < nkv_t[t]) {
+                            mbar_wait(&sh.p_full[t], n_p[t] & 1u, guard);
+                            ++n_p[t];
+                            if (j == 0 && use[t] >= 1) mbar_wait(&sh.o_free[t], (use[t] - 1) & 1u, guard);
+                            tc_fence_after();
+                            issue_pv<D>(o_tmem[t], s_tmem[t], kv_smem(iv), j > 0);
+                            if (j == nkv_t[t] - 1) tc_commit(&sh.o_full[t]);
+                        }
+                    }
+                    tc_commit(&sh.kv_empty[iv % kKvStages]);
+                    if (j + 1 < nkv_t[1]) {
+                        issue_qk<D>(s_tmem[1], q_addr[1], kv_smem(ik));
+                        tc_commit(&sh.s_full[1]);
+                    }
+                    if (has_next) tc_commit(&sh.kv_empty[ik % kKvStages]);
+                }
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (nkv_t[t] == 0) continue;
+                    tc_commit(&sh.q_empty[t]);
+                    ++use[t];
+                }
+                kv_base += 2 * nkv;
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- softmax groups
+        const int t = warp >> 2;                        // Q tile of this group
+        const int row_in_tile = tid & 127;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t s_tmem = tmem + lane_base + (t == 0 ? Cfg::kS0 : Cfg::kS1);
+        const uint32_t o_tmem = tmem + lane_base + (t == 0 ? Cfg::kO0 : Cfg::kO1);
+        uint32_t n_work = 0, n_s = 0, use = 0;
+        while (true) {
+            const uint32_t slot = n_work & 1u;
+            const bool got = mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard);
+            if (!__all_sync(0xffffffffu, got)) break;
+            const WorkItem w = sh.work[slot];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.work_empty[slot]);
+            ++n_work;
+            if (w.len < 0) break;
+            const int r_tile = w.blk * kFwdRowsPerItem + t * kTile;
+            const int nkv = kv_tiles_for<CAUSAL>(r_tile, w.len);
+            if (nkv == 0) continue;
+            const int row = r_tile + row_in_tile;       // row inside the sequence (may be >= len)
+
+            float m = -INFINITY, l = 0.f;
+            for (int j = 0; j < nkv; ++j) {
+                mbar_wait(&sh.s_full[t], n_s & 1u, guard);
+                ++n_s;
+                tc_fence_after();
+                uint32_t s[128];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_ld_x32(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+                tmem_wait_ld();
+
+                const bool boundary = (j == nkv - 1) && (CAUSAL || (w.len & (kTile - 1)) != 0);
+                if (boundary) {
+                    const int last_key = CAUSAL ? (row < w.len - 1 ? row : w.len - 1) : w.len - 1;
+                    const int n_valid = last_key - j * kTile + 1;     // >= 1
+#pragma unroll
+                    for (int c = 0; c < 128; ++c)
+                        if (c >= n_valid) s[c] = 0xff800000u;         // -inf
+                }
+                float mx = __uint_as_float(s[0]);
+#pragma unroll
+                for (int c = 1; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
+
+                const bool need = (mx - m) * p.scale_log2 > kRescaleThreshold;
+                if (__any_sync(0xffffffffu, need)) {
+                    const float m_new = fmaxf(m, mx);
+                    const float factor = fast_exp2((m - m_new) * p.scale_log2);
+                    m = m_new;
+                    l *= factor;
+                    if (j > 0) {
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t acc[32];
+                            tmem_ld_x32(o_tmem + c * 32, acc);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * factor);
+                            tmem_st_x32(o_tmem + c * 32, acc);
+                        }
+                    }
+                }
+                const float neg_m = -m * p.scale_log2;
+                float sum = 0.f;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + 2 * i]), p.scale_log2, neg_m));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + 2 * i + 1]), p.scale_log2, neg_m));
+                        sum += p0 + p1;
+                        pk[i] = pack_bf16x2(p0, p1);
+                    }
+                    tmem_st_x16(s_tmem + c * 16, pk);
+                }
+                l += sum;
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.p_full[t]);
+            }
+
+            // epilogue: O = acc / l, lse = m*scale + ln l
+            mbar_wait(&sh.o_full[t], use & 1u, guard);
+            ++use;
+            tc_fence_after();
+            const float inv_l = 1.0f / l;
+            const bool valid = row < w.len;
+            const size_t tok = (size_t)w.tok0 + (size_t)row;
+            __nv_bfloat16* out = p.o + (tok * p.n_heads + w.head) * D;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t acc[32];
+                tmem_ld_x32(o_tmem + c * 32, acc);
+                tmem_wait_ld();
+                if (valid) {
+#pragma unroll
+                    for (int v4 = 0; v4 < 4; ++v4) {
+                        uint4 val;
+                        val.x = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 0]) * inv_l, __uint_as_float(acc[v4 * 8 + 1]) * inv_l);
+                        val.y = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 2]) * inv_l, __uint_as_float(acc[v4 * 8 + 3]) * inv_l);
+                        val.z = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 4]) * inv_l, __uint_as_float(acc[v4 * 8 + 5]) * inv_l);
+                        val.w = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 6]) * inv_l, __uint_as_float(acc[v4 * 8 + 7]) * inv_l);
+                        *reinterpret_cast<uint4*>(out + c * 32 + v4 * 8) = val;
+                    }
+                }
+            }
+            if (valid) p.lse[(size_t)w.head * p.total_tokens + tok] = m * p.scale + __logf(l);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.o_free[t]);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+template <int D, bool CAUSAL>
+static cudaError_t launch_one(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
+                              int n_ctas, cudaStream_t stream) {
+    auto kern = attn_fwd_kernel<D, CAUSAL>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<D>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    kern<<<n_ctas, kFwdThreads, FwdCfg<D>::kSmemBytes, stream>>>(tq, tk, tv, p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
+                            int head_dim, bool causal, int n_ctas, cudaStream_t stream) {
+    if (head_dim == 128)
+        return causal ? launch_one<128, true>(tq, tk, tv, p, n_ctas, stream) : launch_one<128, false>(tq, tk, tv, p, n_ctas, stream);
+    return causal ? launch_one<64, true>(tq, tk, tv, p, n_ctas, stream) : launch_one<64, false>(tq, tk, tv, p, n_ctas, stream);
+}
+
+}  // namespace dcp

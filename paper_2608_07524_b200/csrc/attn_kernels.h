@@ -1,0 +1,53 @@
+// Host-visible launch interface of the attention kernels (internal to libdcp).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "sched.cuh"
+
+namespace dcp {
+
+struct FwdParams {
+    const int32_t* cu_seqlens;
+    __nv_bfloat16* o;
+    float* lse;
+    SchedView sched;
+    int32_t n_heads;
+    int32_t total_tokens;
+    float scale;        // softmax scale
+    float scale_log2;   // scale * log2(e)
+};
+
+struct BwdParams {
+    const int32_t* cu_seqlens;
+    const float* lse;     // [H, T]
+    const float* dsum;    // [H, T]   D_i = sum_c dO_ic O_ic
+    float* dq_acc;        // [T, H, d] fp32, zeroed before the main kernel
+    __nv_bfloat16* dk;
+    __nv_bfloat16* dv;
+    SchedView sched;
+    int32_t n_heads;
+    int32_t total_tokens;
+    float scale;
+    float scale_log2;
+};
+
+// Builds the work list (longest sequence first) and resets the work counter and status word.
+cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t rows_per_block, int32_t n_heads,
+                        const SchedView& sched, cudaStream_t stream);
+
+cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
+                            int head_dim, bool causal, int n_ctas, cudaStream_t stream);
+
+// D = rowsum(dO * O) and dq_acc = 0.
+cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* dsum, float* dq_acc,
+                           int32_t total_tokens, int32_t n_heads, int32_t head_dim, cudaStream_t stream);
+
+cudaError_t launch_attn_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
+                            const BwdParams& p, int head_dim, bool causal, int n_ctas, cudaStream_t stream);
+
+// dq = bf16(scale * dq_acc)
+cudaError_t launch_bwd_post(const float* dq_acc, __nv_bfloat16* dq, size_t n_elems, float scale, cudaStream_t stream);
+
+}  // namespace dcp

@@ -1,0 +1,101 @@
+// Host-side micro-batch / recomputation planner (dcp_plan).
+//
+// Section 3.4 of the paper models a batch with r recomputed layers as
+//     T = T_f + T_b + r * t_f + T_C                        (Eq. 4-5)
+//     M = (Lambda - r) * m + Lambda * m_inp + M_C          (Eq. 6)
+// and Algorithm 1 picks, per candidate, the smallest r that fits the memory capacity.  On one GPU
+// (sequence-parallel size 1) the remaining freedom is how the batch is cut into gradient-
+// accumulation micro-batches; sequences are first ordered by length (Section 3.1) and a plan is
+// a cut of that order into contiguous blocks.  This file finds the optimum with an O(n^2)
+// dynamic programme over suffixes of the sorted order; the definition, cost units and tie rules
+// are stated in include/dcp.h.
+#include <algorithm>
+#include <cstdint>
+#include <numeric>
+#include <vector>
+
+#include "../../include/dcp.h"
+#include "dcp_internal.h"
+
+namespace {
+
+using u128 = unsigned __int128;
+constexpr u128 kInt64Max = (u128)INT64_MAX;
+
+struct Key {           // objective of a suffix plan: (cost, number of blocks)
+    u128 cost;
+    int32_t blocks;
+    bool operator<(const Key& o) const { return cost != o.cost ? cost < o.cost : blocks < o.blocks; }
+    bool operator==(const Key& o) const { return cost == o.cost && blocks == o.blocks; }
+};
+
+// Smallest r in [0, Lambda] whose memory fits, or -1.  mem(r) falls as r grows, so the answer is
+// ceil((mem(0) - budget) / m) clamped; computed here without division to keep it obviously exact.
+int min_recompute(u128 tok, const dcp_plan_params& p, u128 budget) {
+    const u128 unit = (u128)p.n_heads * (u128)p.head_dim * (u128)p.elt_bytes * tok;   // < 2^31*2^31*2^31*2^36
+    const u128 base = (u128)p.n_layers * unit + (u128)p.const_bytes;
+    if (base > budget) return -1;
+    const u128 room = budget - base;           // bytes left for un-recomputed layers
+    const u128 m = 4 * unit;
+    const u128 keep = m == 0 ? (u128)p.n_layers : std::min<u128>((u128)p.n_layers, room / m);
+    return p.n_layers - (int)keep;
+}
+
+}  // namespace
+
+extern "C" int dcp_plan(const int32_t* lengths, int32_t n, int64_t hbm_budget_bytes, const dcp_plan_params* params,
+                        int32_t* mb_id, int32_t* n_mb, int32_t* recompute, int64_t* cost) {
+    static const dcp_plan_params kDefaults = {16, 128, 2, 1, 0, (int64_t)1 << 24};
+    const dcp_plan_params p = params ? *params : kDefaults;
+    if (!lengths || !mb_id || !n_mb || !recompute) return dcp::fail(DCP_ERR_INVALID_ARG, "dcp_plan: null pointer");
+    if (n < 1) return dcp::fail(DCP_ERR_INVALID_ARG, "dcp_plan: n = %d, need n >= 1", n);
+    if (hbm_budget_bytes < 0) return dcp::fail(DCP_ERR_INVALID_ARG, "dcp_plan: negative budget");
+    if (p.n_heads < 1 || p.head_dim < 1 || p.elt_bytes < 1 || p.n_layers < 1 || p.const_bytes < 0 || p.fixed_cost < 0)
+        return dcp::fail(DCP_ERR_INVALID_ARG, "dcp_plan: bad params (H, d, e, Lambda >= 1; M_C, T_C >= 0)");
+    for (int32_t i = 0; i < n; ++i)
+        if (lengths[i] < 1) return dcp::fail(DCP_ERR_INVALID_ARG, "dcp_plan: lengths[%d] = %d, need >= 1", i, lengths[i]);
+
+    std::vector<int32_t> order(n);
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return lengths[a] > lengths[b]; });
+
+    // prefix sums over the sorted order
+    std::vector<u128> tok(n + 1, 0), sq(n + 1, 0);
+    for (int32_t i = 0; i < n; ++i) {
+        const u128 L = (u128)lengths[order[i]];
+        tok[i + 1] = tok[i] + L;
+        sq[i + 1] = sq[i] + L * L;
+    }
+    const u128 budget = (u128)hbm_budget_bytes;
+    if (min_recompute(tok[1] - tok[0], p, budget) < 0)
+        return dcp::fail(DCP_ERR_INFEASIBLE,
+                         "dcp_plan: the longest sequence (%d tokens) exceeds the budget even with every layer recomputed",
+                         lengths[order[0]]);
+
+    // best[i] = optimum for the sorted suffix i..n-1; cut[i] = end of its first block (largest on ties)
+    std::vector<Key> best(n + 1);
+    std::vector<int32_t> cut(n + 1, n), rec(n + 1, 0);
+    best[n] = {0, 0};
+    for (int32_t i = n - 1; i >= 0; --i) {
+        bool have = false;
+        for (int32_t j = i + 1; j <= n; ++j) {
+            const int r = min_recompute(tok[j] - tok[i], p, budget);
+            if (r < 0) break;                                  // larger blocks only need more memory
+            const Key cand = {best[j].cost + (u128)p.fixed_cost + 2 * (u128)r * (sq[j] - sq[i]), best[j].blocks + 1};
+            if (!have || cand < best[i] || cand == best[i]) {  // '==' keeps the LARGEST j among ties
+                best[i] = cand; cut[i] = j; rec[i] = r; have = true;
+            }
+        }
+        // a single sequence always fits here: the longest one does and memory grows with length
+    }
+    if (best[0].cost > kInt64Max) return dcp::fail(DCP_ERR_OVERFLOW, "dcp_plan: cost does not fit in int64");
+
+    int32_t k = 0;
+    for (int32_t i = 0; i < n; i = cut[i], ++k) {
+        recompute[k] = rec[i];
+        for (int32_t a = i; a < cut[i]; ++a) mb_id[order[a]] = k;
+    }
+    *n_mb = k;
+    if (cost) *cost = (int64_t)best[0].cost;
+    return DCP_OK;
+}

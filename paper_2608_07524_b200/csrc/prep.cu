@@ -1,0 +1,148 @@
+// Work-list construction and the two small memory-bound backward helpers.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "attn_kernels.h"
+#include "sched.cuh"
+
+namespace dcp {
+
+constexpr int kPrepThreads = 1024;
+
+// One CTA.  order[] = sequence ids sorted by (length descending, id ascending) via a rank sort;
+// prefix[i] = number of work items of the first i sequences in that order, where a sequence of
+// length L contributes ceil(L / rows_per_block) * n_heads items.
+__global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __restrict__ cu, int32_t n_seqs,
+                                                            int32_t rows_per_block, int32_t n_heads,
+                                                            WorkspaceHeader* hdr, int32_t* order, uint32_t* prefix) {
+    __shared__ uint32_t chunk_sum[kPrepThreads];
+    const int tid = threadIdx.x;
+    for (int i = tid; i < n_seqs; i += kPrepThreads) {
+        const int32_t len_i = cu[i + 1] - cu[i];
+        int rank = 0;
+        for (int j = 0; j < n_seqs; ++j) {
+            const int32_t len_j = cu[j + 1] - cu[j];
+            rank += (len_j > len_i) || (len_j == len_i && j < i);
+        }
+        order[rank] = i;
+    }
+    __syncthreads();
+    // exclusive scan of item counts over the sorted order: contiguous chunk per thread
+    const int per = (n_seqs + kPrepThreads - 1) / kPrepThreads;
+    const int begin = tid * per, end = min(begin + per, n_seqs);
+    auto items_of = [&](int pos) -> uint32_t {
+        const int s = order[pos];
+        const int32_t len = cu[s + 1] - cu[s];
+        return (uint32_t)((len + rows_per_block - 1) / rows_per_block) * (uint32_t)n_heads;
+    };
+    uint32_t local = 0;
+    for (int i = begin; i < end; ++i) local += items_of(i);
+    chunk_sum[tid] = local;
+    __syncthreads();
+    if (tid == 0) {
+        uint32_t run = 0;
+        for (int i = 0; i < kPrepThreads; ++i) {
+            const uint32_t c = chunk_sum[i];
+            chunk_sum[i] = run;
+            run += c;
+        }
+        prefix[n_seqs] = run;
+        hdr->n_items = run;
+        hdr->work_counter = 0;
+        hdr->status = 0;
+    }
+    __syncthreads();
+    uint32_t run = chunk_sum[tid];
+    for (int i = begin; i < end; ++i) {
+        prefix[i] = run;
+        run += items_of(i);
+    }
+}
+
+cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t rows_per_block, int32_t n_heads,
+                        const SchedView& sched, cudaStream_t stream) {
+    prep_kernel<<<1, kPrepThreads, 0, stream>>>(cu_seqlens, n_seqs, rows_per_block, n_heads, sched.hdr,
+                                                const_cast<int32_t*>(sched.order), const_cast<uint32_t*>(sched.prefix));
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Backward helper 1: D[h][t] = sum_c dO[t][h][c] * O[t][h][c]; dq_acc[t][h][:] = 0.
+// One warp per (token, head) row; HBM-bound: reads 2*d*2 bytes, writes d*4 + 4 bytes per row.
+template <int D>
+__global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __restrict__ o,
+                                                      const __nv_bfloat16* __restrict__ d_o, float* __restrict__ dsum,
+                                                      float* __restrict__ dq_acc, int32_t total_tokens, int32_t n_heads) {
+    const int lane = threadIdx.x & 31;
+    const size_t n_rows = (size_t)total_tokens * n_heads;
+    const size_t warps = (size_t)gridDim.x * (blockDim.x >> 5);
+    for (size_t row = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); row < n_rows; row += warps) {
+        constexpr int kPer = D / 32;           // elements per lane: 2 or 4
+        const __nv_bfloat16* po = o + row * D + lane * kPer;
+        const __nv_bfloat16* pg = d_o + row * D + lane * kPer;
+        float acc = 0.f;
+        if (kPer == 4) {
+            const uint2 a = *reinterpret_cast<const uint2*>(po), b = *reinterpret_cast<const uint2*>(pg);
+            const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.x));
+            const float2 a1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.y));
+            const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.x));
+            const float2 b1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.y));
+            acc = a0.x * b0.x + a0.y * b0.y + a1.x * b1.x + a1.y * b1.y;
+            *reinterpret_cast<float4*>(dq_acc + row * D + lane * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+        } else {
+            const uint32_t a = *reinterpret_cast<const uint32_t*>(po), b = *reinterpret_cast<const uint32_t*>(pg);
+            const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a));
+            const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b));
+            acc = a0.x * b0.x + a0.y * b0.y;
+            *reinterpret_cast<float2*>(dq_acc + row * D + lane * 2) = make_float2(0.f, 0.f);
+        }
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+        if (lane == 0) {
+            const size_t tok = row / n_heads, h = row % n_heads;
+            dsum[h * total_tokens + tok] = acc;
+        }
+    }
+}
+
+cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* dsum, float* dq_acc,
+                           int32_t total_tokens, int32_t n_heads, int32_t head_dim, cudaStream_t stream) {
+    const size_t n_rows = (size_t)total_tokens * n_heads;
+    const int blocks = (int)min((size_t)148 * 8, (n_rows + 7) / 8);
+    if (blocks == 0) return cudaSuccess;
+    if (head_dim == 128)
+        bwd_pre_kernel<128><<<blocks, 256, 0, stream>>>(o, d_o, dsum, dq_acc, total_tokens, n_heads);
+    else
+        bwd_pre_kernel<64><<<blocks, 256, 0, stream>>>(o, d_o, dsum, dq_acc, total_tokens, n_heads);
+    return cudaGetLastError();
+}
+
+// Backward helper 2: dq = bf16(scale * dq_acc).  8 elements per thread.
+__global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict__ dq,
+                                                       size_t n_vec8, float scale) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec8; i += stride) {
+        const float4 a = reinterpret_cast<const float4*>(dq_acc)[2 * i];
+        const float4 b = reinterpret_cast<const float4*>(dq_acc)[2 * i + 1];
+        __nv_bfloat162 r0 = __floats2bfloat162_rn(a.x * scale, a.y * scale);
+        __nv_bfloat162 r1 = __floats2bfloat162_rn(a.z * scale, a.w * scale);
+        __nv_bfloat162 r2 = __floats2bfloat162_rn(b.x * scale, b.y * scale);
+        __nv_bfloat162 r3 = __floats2bfloat162_rn(b.z * scale, b.w * scale);
+        uint4 out;
+        out.x = *reinterpret_cast<uint32_t*>(&r0);
+        out.y = *reinterpret_cast<uint32_t*>(&r1);
+        out.z = *reinterpret_cast<uint32_t*>(&r2);
+        out.w = *reinterpret_cast<uint32_t*>(&r3);
+        reinterpret_cast<uint4*>(dq)[i] = out;
+    }
+}
+
+cudaError_t launch_bwd_post(const float* dq_acc, __nv_bfloat16* dq, size_t n_elems, float scale, cudaStream_t stream) {
+    const size_t n_vec8 = n_elems / 8;          // head_dim is a multiple of 64
+    if (n_vec8 == 0) return cudaSuccess;
+    const int blocks = (int)min((size_t)148 * 16, (n_vec8 + 255) / 256);
+    bwd_post_kernel<<<blocks, 256, 0, stream>>>(dq_acc, dq, n_vec8, scale);
+    return cudaGetLastError();
+}
+
+}  // namespace dcp

@@ -1,0 +1,70 @@
+// Workspace layout and the length-aware work list shared by the forward and backward kernels.
+//
+// The paper's subject is load imbalance caused by widely varying sequence lengths (Section 2.3);
+// on one GPU the same problem shows up as SMs idling while one long sequence finishes.  The work
+// list therefore orders sequences longest first, and persistent CTAs pull items from it through a
+// global atomic counter, so the cheap items of short sequences fill the tail.
+#pragma once
+#include <cstdint>
+
+namespace dcp {
+
+constexpr int kTile = 128;            // rows of a Q tile / keys of a K,V tile
+constexpr int kFwdRowsPerItem = 256;  // a forward work item is two Q tiles of one (sequence, head)
+
+// First bytes of every workspace.  `status` must stay at offset 0 (dcp_query_status reads it).
+struct WorkspaceHeader {
+    uint32_t status;        // 0 = ok, else a kStatus* code left by a kernel
+    uint32_t work_counter;  // next unclaimed work item
+    uint32_t n_items;       // items in the list
+    uint32_t pad[61];
+};
+static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
+
+// After the header: int32 order[n_seqs] (sequence ids, longest first, ties by id) and
+// uint32 prefix[n_seqs + 1] (items before the i-th sequence of `order`).
+struct SchedView {
+    WorkspaceHeader* hdr;
+    const int32_t* order;
+    const uint32_t* prefix;
+    int32_t n_seqs;
+};
+
+__host__ __device__ inline size_t sched_bytes(int32_t n_seqs) {
+    size_t b = sizeof(WorkspaceHeader) + sizeof(int32_t) * (size_t)n_seqs + sizeof(uint32_t) * ((size_t)n_seqs + 1);
+    return (b + 255) & ~(size_t)255;
+}
+
+// A decoded work item.  len < 0 marks the end of the list.
+struct WorkItem {
+    int32_t tok0;   // first token of the sequence in the packed batch
+    int32_t len;    // sequence length
+    int32_t head;
+    int32_t blk;    // row block inside the sequence (256 query rows forward, 128 keys backward)
+};
+
+// Map item index -> (sequence, head, block).  Within a sequence, blocks vary fastest so that CTAs
+// running at the same time share one head's K and V in L2; under a causal mask the heaviest
+// blocks come first (forward: last rows see the most keys; backward: first keys are seen by the
+// most rows).
+__device__ inline WorkItem decode_item(const SchedView& s, const int32_t* cu_seqlens, uint32_t item, int rows_per_blk,
+                                       int n_heads, bool heavy_is_last) {
+    int lo = 0, hi = s.n_seqs;              // largest i with prefix[i] <= item
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (s.prefix[mid] <= item) lo = mid; else hi = mid;
+    }
+    const int seq = s.order[lo];
+    WorkItem w;
+    w.tok0 = cu_seqlens[seq];
+    w.len = cu_seqlens[seq + 1] - w.tok0;
+    const uint32_t local = item - s.prefix[lo];
+    const uint32_t nblk = (uint32_t)(w.len + rows_per_blk - 1) / (uint32_t)rows_per_blk;
+    w.head = (int32_t)(local / nblk);
+    const uint32_t b = local % nblk;
+    w.blk = (int32_t)(heavy_is_last ? nblk - 1 - b : b);
+    (void)n_heads;
+    return w;
+}
+
+}  // namespace dcp
