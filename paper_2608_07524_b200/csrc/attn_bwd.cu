@@ -1,7 +1,474 @@
+// Backward packed variable-length attention for sm_100a (main kernel).
+//
+// One persistent CTA per SM.  A work item is (sequence, head, 128 keys); the CTA keeps that K and V
+// tile in shared memory and walks over every Q tile that sees it.  Everything is computed in the
+// transposed orientation, keys on tensor-memory lanes and queries on columns, so that P^T can feed
+// the dV product straight from tensor memory:
+//
+//     S^T  = K Q^T                      (tcgen05, fp32 in tensor memory)
+//     P^T  = exp2(S^T*scale*log2e - lse*log2e), masked            -> bf16, overwrites S^T
+//     dP^T = V dO^T
+//     dS^T = P^T o (dP^T - D)                                      -> bf16, shared memory
+//     dV  += P^T dO          dK += dS^T Q          dQ_tile = dS K  (dQ aliases dP^T's columns)
+//
+// dQ tiles are added into an fp32 accumulator in global memory with vector atomics because every
+// key block of a sequence contributes to the same query rows; dK and dV stay in tensor memory for
+// the whole item and are written once (dK scaled by the softmax scale).
+//
+// Roles:  warps 0-7 compute (two groups, each owns 64 of the 128 query columns, one key per thread),
+//         warp 8 MMA issue, warp 9 scheduler + TMA producer + per-row statistics staging,
+//         warps 10-13 dQ drain (tensor memory -> global atomics).
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
 #include "attn_kernels.h"
+#include "sched.cuh"
+#include "sm100_ptx.cuh"
+
 namespace dcp {
-cudaError_t launch_attn_bwd(const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, const CUtensorMap&,
-                            const BwdParams&, int, bool, int, cudaStream_t) {
-    return cudaErrorNotSupported;
+
+constexpr int kBwdThreads = 448;
+constexpr float kLog2e = 1.4426950408889634f;
+
+template <int D>
+struct BwdCfg {
+    static constexpr int kTileBytes = kTile * D * 2;     // K, V, Q or dO tile
+    static constexpr int kBoxBytes = kTile * 128;
+    static constexpr int kBoxes = D / 64;
+    static constexpr int kDsBytes = kTile * kTile * 2;   // dS^T tile, bf16
+    // shared-memory map (offsets from a 1024-byte aligned base)
+    static constexpr int kOffK = 0;
+    static constexpr int kOffV = kTileBytes;
+    static constexpr int kOffQ = 2 * kTileBytes;          // 2 stages
+    static constexpr int kOffDo = 4 * kTileBytes;         // 2 stages
+    static constexpr int kOffDs = 6 * kTileBytes;
+    static constexpr int kOffStat = kOffDs + kDsBytes;    // 2 stages x (128 nlse + 128 D) floats
+    static constexpr int kOffCtl = kOffStat + 2 * 256 * 4;
+    static constexpr int kSmemBytes = kOffCtl + 512;
+    // tensor-memory columns
+    static constexpr uint32_t kSt = 0, kDp = 128, kDv = 256, kDk = 384;
+};
+
+struct BwdControl {
+    uint64_t work_full[2], work_empty[2];
+    uint64_t kv_full, kv_empty;
+    uint64_t q_full[2], q_empty[2], do_full[2], do_empty[2];
+    uint64_t s_full, p_full, dp_full, ds_full, ds_free, dq_full, dq_free, dkv_full, dkv_free;
+    WorkItem work[2];
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+static_assert(sizeof(BwdControl) <= 512, "control block must fit its slot");
+
+__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
+
+template <int D>
+__device__ __forceinline__ void bwd_load_tile(uint8_t* dst, const CUtensorMap* map, uint64_t* bar, int head, int row) {
+#pragma unroll
+    for (int b = 0; b < BwdCfg<D>::kBoxes; ++b)
+        tma_load_3d(dst + b * BwdCfg<D>::kBoxBytes, map, bar, b * 64, head, row);
+}
+
+// D[128 x 128] = A B^T with A, B both [128 x D] row-major tiles (contraction over head_dim).
+template <int D>
+__device__ __forceinline__ void issue_abt(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr) {
+    constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, false);
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+        const uint32_t off = (ks / 4) * BwdCfg<D>::kBoxBytes + (ks % 4) * 32;
+        tc_mma_ss(d_tmem, make_sdesc_sw128(a_addr + off, 16, 1024), make_sdesc_sw128(b_addr + off, 16, 1024), idesc, ks > 0);
+    }
+}
+
+template <int D, bool CAUSAL>
+__global__ void __launch_bounds__(kBwdThreads, 1)
+attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_do,
+                const BwdParams p) {
+    using Cfg = BwdCfg<D>;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    BwdControl& sh = *reinterpret_cast<BwdControl*>(smem + Cfg::kOffCtl);
+    float* stats = reinterpret_cast<float*>(smem + Cfg::kOffStat);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const WaitGuard guard{&sh.abort_flag, &p.sched.hdr->status};
+
+    if (tid == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&sh.work_full[i], 1);
+            mbar_init(&sh.work_empty[i], 13);   // 8 compute warps + 4 drain warps + the MMA thread
+            mbar_init(&sh.q_full[i], 2);        // TMA bytes + statistics staged
+            mbar_init(&sh.q_empty[i], 1);
+            mbar_init(&sh.do_full[i], 1);
+            mbar_init(&sh.do_empty[i], 1);
+        }
+        mbar_init(&sh.kv_full, 1);
+        mbar_init(&sh.kv_empty, 1);
+        mbar_init(&sh.s_full, 1);
+        mbar_init(&sh.p_full, 8);
+        mbar_init(&sh.dp_full, 1);
+        mbar_init(&sh.ds_full, 8);
+        mbar_init(&sh.ds_free, 1);
+        mbar_init(&sh.dq_full, 1);
+        mbar_init(&sh.dq_free, 4);
+        mbar_init(&sh.dkv_full, 1);
+        mbar_init(&sh.dkv_free, 8);
+        sh.abort_flag = 0;
+        fence_mbar_init();
+        // the swizzled tile layout needs a 1024-byte aligned base; refuse to run otherwise
+        if ((smem_u32(smem) & 1023u) != 0) {
+            sh.abort_flag = 1;
+            atomicMax(&p.sched.hdr->status, (uint32_t)kStatusBadSmemAlign);
+        }
+    }
+    if (warp == 0) {
+        tmem_alloc(&sh.tmem_base, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh.tmem_base;
+
+    // Q tiles that see key block `blk`: [first_q, n_q)
+    auto q_range = [](const WorkItem& w, int& first_q, int& n_q) {
+        n_q = (w.len + kTile - 1) / kTile;
+        first_q = CAUSAL ? w.blk : 0;
+    };
+
+    if (warp == 9) {
+        // ------------------------------------------------- scheduler, TMA producer, statistics staging
+        if (lane == 0) {
+            tma_prefetch_desc(&tmap_q);
+            tma_prefetch_desc(&tmap_k);
+            tma_prefetch_desc(&tmap_v);
+            tma_prefetch_desc(&tmap_do);
+        }
+        const uint32_t n_items = p.sched.hdr->n_items;
+        uint32_t n_work = 0, g = 0;
+        while (true) {
+            const uint32_t slot = n_work & 1u;
+            WorkItem w;
+            if (lane == 0) {
+                if (n_work >= 2) mbar_wait(&sh.work_empty[slot], ((n_work >> 1) - 1) & 1u, guard);
+                const uint32_t item = atomicAdd(&p.sched.hdr->work_counter, 1u);
+                if (item < n_items && !sh.abort_flag) {
+                    w = decode_item(p.sched, p.cu_seqlens, item, kTile, p.n_heads, false);
+                } else {
+                    w.tok0 = 0; w.len = -1; w.head = 0; w.blk = 0;
+                }
+                sh.work[slot] = w;
+                mbar_arrive(&sh.work_full[slot]);
+            }
+            w.tok0 = __shfl_sync(0xffffffffu, w.tok0, 0);
+            w.len = __shfl_sync(0xffffffffu, w.len, 0);
+            w.head = __shfl_sync(0xffffffffu, w.head, 0);
+            w.blk = __shfl_sync(0xffffffffu, w.blk, 0);
+            if (w.len < 0) break;
+            int first_q, n_q;
+            q_range(w, first_q, n_q);
+            if (lane == 0) {
+                if (n_work >= 1) mbar_wait(&sh.kv_empty, (n_work - 1) & 1u, guard);
+                mbar_expect_tx(&sh.kv_full, 2 * Cfg::kTileBytes);
+                bwd_load_tile<D>(smem + Cfg::kOffK, &tmap_k, &sh.kv_full, w.head, w.tok0 + w.blk * kTile);
+                bwd_load_tile<D>(smem + Cfg::kOffV, &tmap_v, &sh.kv_full, w.head, w.tok0 + w.blk * kTile);
+            }
+            ++n_work;
+            for (int i = first_q; i < n_q; ++i, ++g) {
+                const uint32_t stage = g & 1u;
+                const int row = w.tok0 + i * kTile;
+                if (lane == 0) {
+                    if (g >= 2) {
+                        mbar_wait(&sh.q_empty[stage], ((g >> 1) - 1) & 1u, guard);
+                        mbar_wait(&sh.do_empty[stage], ((g >> 1) - 1) & 1u, guard);
+                    }
+                    mbar_expect_tx(&sh.q_full[stage], Cfg::kTileBytes);
+                    bwd_load_tile<D>(smem + Cfg::kOffQ + stage * Cfg::kTileBytes, &tmap_q, &sh.q_full[stage], w.head, row);
+                    mbar_expect_tx(&sh.do_full[stage], Cfg::kTileBytes);
+                    bwd_load_tile<D>(smem + Cfg::kOffDo + stage * Cfg::kTileBytes, &tmap_do, &sh.do_full[stage], w.head, row);
+                }
+                __syncwarp();
+                // per-row statistics of this Q tile: -lse*log2(e) (or +inf past the sequence end,
+                // which zeroes P there) and D
+                float* st = stats + stage * 256;
+                const size_t base = (size_t)w.head * p.total_tokens + row;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int r = lane + 32 * e;
+                    const bool ok = i * kTile + r < w.len;
+                    st[r] = ok ? -p.lse[base + r] * kLog2e : -INFINITY;
+                    st[128 + r] = ok ? p.dsum[base + r] : 0.f;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.q_full[stage]);
+            }
+        }
+    } else if (warp == 8) {
+        // ------------------------------------------------- MMA issue
+        if (lane == 0) {
+            const uint32_t k_addr = smem_u32(smem + Cfg::kOffK), v_addr = smem_u32(smem + Cfg::kOffV);
+            const uint32_t q_addr0 = smem_u32(smem + Cfg::kOffQ), do_addr0 = smem_u32(smem + Cfg::kOffDo);
+            const uint32_t ds_addr = smem_u32(smem + Cfg::kOffDs);
+            constexpr uint32_t idesc_nd_kb = make_idesc_bf16(128, D, false, true);   // A K-contig / tmem, B N-contig
+            constexpr uint32_t idesc_nd_mm = make_idesc_bf16(128, D, true, true);    // A M-contig, B N-contig
+            uint32_t n_work = 0, g = 0;
+            while (true) {
+                const uint32_t slot = n_work & 1u;
+                if (!mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard)) break;
+                const WorkItem w = sh.work[slot];
+                mbar_arrive(&sh.work_empty[slot]);
+                if (w.len < 0) break;
+                int first_q, n_q;
+                q_range(w, first_q, n_q);
+                const int N = n_q - first_q;
+                mbar_wait(&sh.kv_full, n_work & 1u, guard);
+                // S^T and dP^T of the first tile
+                mbar_wait(&sh.q_full[g & 1u], (g >> 1) & 1u, guard);
+                tc_fence_after();
+                issue_abt<D>(tmem + Cfg::kSt, k_addr, q_addr0 + (g & 1u) * Cfg::kTileBytes);
+                tc_commit(&sh.s_full);
+                mbar_wait(&sh.do_full[g & 1u], (g >> 1) & 1u, guard);
+                if (g >= 1) mbar_wait(&sh.dq_free, (g - 1) & 1u, guard);
+                tc_fence_after();
+                issue_abt<D>(tmem + Cfg::kDp, v_addr, do_addr0 + (g & 1u) * Cfg::kTileBytes);
+                tc_commit(&sh.dp_full);
+                for (int n = 0; n < N; ++n, ++g) {
+                    const uint32_t stage = g & 1u, nstage = stage ^ 1u;
+                    const uint32_t q_addr = q_addr0 + stage * Cfg::kTileBytes, do_addr = do_addr0 + stage * Cfg::kTileBytes;
+                    const bool has_next = n + 1 < N;
+                    // dV += P^T dO
+                    mbar_wait(&sh.p_full, g & 1u, guard);
+                    if (n == 0 && n_work >= 1) mbar_wait(&sh.dkv_free, (n_work - 1) & 1u, guard);
+                    tc_fence_after();
+#pragma unroll
+                    for (int ks = 0; ks < kTile / 16; ++ks)
+                        tc_mma_ts(tmem + Cfg::kDv, tmem + Cfg::kSt + (ks / 4) * 64 + (ks % 4) * 8,
+                                  make_sdesc_sw128(do_addr + ks * 2048, Cfg::kBoxBytes, 1024), idesc_nd_kb, n > 0 || ks > 0);
+                    tc_commit(&sh.do_empty[stage]);
+                    // S^T of the next tile
+                    if (has_next) {
+                        mbar_wait(&sh.q_full[nstage], ((g + 1) >> 1) & 1u, guard);
+                        tc_fence_after();
+                        issue_abt<D>(tmem + Cfg::kSt, k_addr, q_addr0 + nstage * Cfg::kTileBytes);
+                        tc_commit(&sh.s_full);
+                    }
+                    // dQ tile = dS K  (A: dS^T read M-contiguous; B: K with head_dim contiguous)
+                    mbar_wait(&sh.ds_full, g & 1u, guard);
+                    tc_fence_after();
+#pragma unroll
+                    for (int ks = 0; ks < kTile / 16; ++ks)
+                        tc_mma_ss(tmem + Cfg::kDp, make_sdesc_sw128(ds_addr + ks * 2048, 16384, 1024),
+                                  make_sdesc_sw128(k_addr + ks * 2048, Cfg::kBoxBytes, 1024), idesc_nd_mm, ks > 0);
+                    tc_commit(&sh.dq_full);
+                    // dK += dS^T Q
+#pragma unroll
+                    for (int ks = 0; ks < kTile / 16; ++ks) {
+                        const uint32_t offa = (ks / 4) * 16384 + (ks % 4) * 32;
+                        tc_mma_ss(tmem + Cfg::kDk, make_sdesc_sw128(ds_addr + offa, 16, 1024),
+                                  make_sdesc_sw128(q_addr + ks * 2048, Cfg::kBoxBytes, 1024), idesc_nd_kb, n > 0 || ks > 0);
+                    }
+                    tc_commit(&sh.q_empty[stage]);
+                    tc_commit(&sh.ds_free);
+                    // dP^T of the next tile (its columns hold dQ until the drain warps have read it)
+                    if (has_next) {
+                        mbar_wait(&sh.do_full[nstage], ((g + 1) >> 1) & 1u, guard);
+                        mbar_wait(&sh.dq_free, g & 1u, guard);
+                        tc_fence_after();
+                        issue_abt<D>(tmem + Cfg::kDp, v_addr, do_addr0 + nstage * Cfg::kTileBytes);
+                        tc_commit(&sh.dp_full);
+                    }
+                }
+                tc_commit(&sh.dkv_full);
+                tc_commit(&sh.kv_empty);
+                ++n_work;
+            }
+        }
+    } else if (warp < 8) {
+        // ------------------------------------------------- compute: P^T, dS^T, final dK / dV
+        const int half = warp >> 2;                                  // which 64 query columns
+        const int key_in_tile = (warp & 3) * 32 + lane;              // tensor-memory lane = key
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t st_tmem = tmem + lane_base + Cfg::kSt + half * 64;
+        const uint32_t pt_tmem = tmem + lane_base + Cfg::kSt + half * 64;   // bf16 pairs, inside this group's own S^T columns
+        const uint32_t dp_tmem = tmem + lane_base + Cfg::kDp + half * 64;
+        uint8_t* ds_row = smem + Cfg::kOffDs + half * 16384;
+        uint32_t n_work = 0, g = 0;
+        while (true) {
+            const uint32_t slot = n_work & 1u;
+            const bool got = mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard);
+            if (!__all_sync(0xffffffffu, got)) break;
+            const WorkItem w = sh.work[slot];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.work_empty[slot]);
+            if (w.len < 0) break;
+            int first_q, n_q;
+            q_range(w, first_q, n_q);
+            const int key = w.blk * kTile + key_in_tile;
+            const bool key_valid = key < w.len;
+            const bool key_tail = (w.blk + 1) * kTile > w.len;
+
+            for (int i = first_q; i < n_q; ++i, ++g) {
+                const float* st = stats + (g & 1u) * 256 + half * 64;
+                const bool diag = CAUSAL && i == w.blk;
+                float pf[64];
+                mbar_wait(&sh.q_full[g & 1u], (g >> 1) & 1u, guard);    // statistics of this tile are staged
+                mbar_wait(&sh.s_full, g & 1u, guard);
+                tc_fence_after();
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t sr[16];
+                    tmem_ld_x16(st_tmem + c * 16, sr);
+                    float nl[16];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        *reinterpret_cast<float4*>(&nl[e * 4]) = *reinterpret_cast<const float4*>(st + c * 16 + e * 4);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 16; ++e)
+                        pf[c * 16 + e] = fast_exp2(fmaf(__uint_as_float(sr[e]), p.scale_log2, nl[e]));
+                    if (key_tail || diag) {
+                        const int q_first = i * kTile + half * 64 + c * 16;   // query index of element 0
+#pragma unroll
+                        for (int e = 0; e < 16; ++e)
+                            if (!key_valid || (diag && key > q_first + e)) pf[c * 16 + e] = 0.f;
+                    }
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) pk[e] = pack_bf16x2(pf[c * 16 + 2 * e], pf[c * 16 + 2 * e + 1]);
+                    tmem_st_x8(pt_tmem + c * 8, pk);
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.p_full);
+
+                // dS^T = P^T o (dP^T - D)
+                mbar_wait(&sh.dp_full, g & 1u, guard);
+                if (g >= 1) mbar_wait(&sh.ds_free, (g - 1) & 1u, guard);
+                tc_fence_after();
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t dr[16];
+                    tmem_ld_x16(dp_tmem + c * 16, dr);
+                    float dd[16];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        *reinterpret_cast<float4*>(&dd[e * 4]) = *reinterpret_cast<const float4*>(st + 128 + c * 16 + e * 4);
+                    tmem_wait_ld();
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float a = pf[c * 16 + 2 * e] * (__uint_as_float(dr[2 * e]) - dd[2 * e]);
+                        const float b = pf[c * 16 + 2 * e + 1] * (__uint_as_float(dr[2 * e + 1]) - dd[2 * e + 1]);
+                        pk[e] = pack_bf16x2(a, b);
+                    }
+                    *reinterpret_cast<uint4*>(ds_row + sw128_offset(key_in_tile, c * 2)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    *reinterpret_cast<uint4*>(ds_row + sw128_offset(key_in_tile, c * 2 + 1)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                }
+                fence_async_smem();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.ds_full);
+            }
+
+            // item epilogue: dV and dK rows of this key block (each group writes half the columns)
+            mbar_wait(&sh.dkv_full, n_work & 1u, guard);
+            tc_fence_after();
+            const size_t tok = (size_t)w.tok0 + (size_t)key;
+            const size_t out_off = (tok * p.n_heads + w.head) * D + half * (D / 2);
+#pragma unroll
+            for (int which = 0; which < 2; ++which) {
+                const uint32_t src = tmem + lane_base + (which == 0 ? Cfg::kDv : Cfg::kDk) + half * (D / 2);
+                __nv_bfloat16* dst = (which == 0 ? p.dv : p.dk) + out_off;
+                const float mul = which == 0 ? 1.0f : p.scale;
+#pragma unroll
+                for (int c = 0; c < D / 64; ++c) {
+                    uint32_t acc[32];
+                    tmem_ld_x32(src + c * 32, acc);
+                    tmem_wait_ld();
+                    if (key_valid) {
+#pragma unroll
+                        for (int v4 = 0; v4 < 4; ++v4) {
+                            uint4 val;
+                            val.x = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 0]) * mul, __uint_as_float(acc[v4 * 8 + 1]) * mul);
+                            val.y = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 2]) * mul, __uint_as_float(acc[v4 * 8 + 3]) * mul);
+                            val.z = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 4]) * mul, __uint_as_float(acc[v4 * 8 + 5]) * mul);
+                            val.w = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 6]) * mul, __uint_as_float(acc[v4 * 8 + 7]) * mul);
+                            *reinterpret_cast<uint4*>(dst + c * 32 + v4 * 8) = val;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.dkv_free);
+            ++n_work;
+        }
+    } else {
+        // ------------------------------------------------- dQ drain: tensor memory -> fp32 atomics
+        const int q_in_tile = (warp & 3) * 32 + lane;               // warps 10-13 -> lane quarters 2,3,0,1
+        const uint32_t dq_tmem = tmem + ((uint32_t)((warp & 3) * 32) << 16) + Cfg::kDp;
+        uint32_t n_work = 0, g = 0;
+        while (true) {
+            const uint32_t slot = n_work & 1u;
+            const bool got = mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard);
+            if (!__all_sync(0xffffffffu, got)) break;
+            const WorkItem w = sh.work[slot];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.work_empty[slot]);
+            if (w.len < 0) break;
+            ++n_work;
+            int first_q, n_q;
+            q_range(w, first_q, n_q);
+            for (int i = first_q; i < n_q; ++i, ++g) {
+                mbar_wait(&sh.dq_full, g & 1u, guard);
+                tc_fence_after();
+                uint32_t acc[D];
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) tmem_ld_x32(dq_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&acc[c * 32]));
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.dq_free);
+                const int qrow = i * kTile + q_in_tile;
+                if (qrow < w.len) {
+                    float* dst = p.dq_acc + (((size_t)w.tok0 + qrow) * p.n_heads + w.head) * D;
+#pragma unroll
+                    for (int c = 0; c < D / 4; ++c)
+                        red_add_v4(dst + c * 4, __uint_as_float(acc[c * 4]), __uint_as_float(acc[c * 4 + 1]),
+                                   __uint_as_float(acc[c * 4 + 2]), __uint_as_float(acc[c * 4 + 3]));
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+template <int D, bool CAUSAL>
+static cudaError_t launch_one(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
+                              const BwdParams& p, int n_ctas, cudaStream_t stream) {
+    auto kern = attn_bwd_kernel<D, CAUSAL>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<D>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    kern<<<n_ctas, kBwdThreads, BwdCfg<D>::kSmemBytes, stream>>>(tq, tk, tv, tdo, p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_attn_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
+                            const BwdParams& p, int head_dim, bool causal, int n_ctas, cudaStream_t stream) {
+    if (head_dim == 128)
+        return causal ? launch_one<128, true>(tq, tk, tv, tdo, p, n_ctas, stream)
+                      : launch_one<128, false>(tq, tk, tv, tdo, p, n_ctas, stream);
+    return causal ? launch_one<64, true>(tq, tk, tv, tdo, p, n_ctas, stream)
+                  : launch_one<64, false>(tq, tk, tv, tdo, p, n_ctas, stream);
+}
+
 }  // namespace dcp
