@@ -1,0 +1,333 @@
+#!/usr/bin/env python
+"""Benchmark of the packed variable-length attention hot path (plan -> forward -> backward).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload video|text|extreme|stream]
+    python bench.py --impl reference ...        # the fp64 CPU oracle on a bounded sample
+
+One step = one pass of the whole path over one synthetic batch: dcp_plan on the batch's lengths,
+then for every micro-batch the work-list kernel, forward attention, and the three backward kernels
+(plus a second forward when the plan asks for recomputation).  Inputs are resident in HBM before
+the timed region; they are several times larger than L2, so no flush is needed between steps.
+Prints one JSON line (rank 0).  Under torchrun every rank runs the same batch shape on its own GPU
+(weak scaling, no data-path collective); time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "varlen_attn_fwd_bwd_tflops"
+UNIT = "TFLOP/s"
+HBM_BUDGET = 180 * 10 ** 9
+# DRAM traffic of one backward-main launch on the bench workload, from the ncu summary under
+# profiles/ (None until a capture exists for the current kernel).
+BWD_MAIN_DRAM_BYTES_PER_LAUNCH = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"burst": float(p["bf16_tflops"]), "sustained": float(p["bf16_tflops_sustained"]),
+                "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    except Exception:
+        return {"burst": 1590.0, "sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index: int, period: float = 0.05):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_flag = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self._stop_flag.is_set():
+            try:
+                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+                bits = int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_flag.set()
+        self.join(timeout=2)
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def physical_gpu_index(local_index: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+def workload(name: str):
+    from paper_2608_07524_b200 import inputs
+    idx = {"text": 2, "video": 3, "extreme": 4}.get(name)
+    return inputs.config(idx) if idx else None
+
+
+# ------------------------------------------------------------------------------------------ oracle arm
+def oracle_sample(seq_len: int, n_heads: int, head_dim: int, causal: bool, seed: int = 12):
+    """fp64 oracle forward + backward on one synthetic sequence; returns (seconds, counted flops)."""
+    import oracle
+    from paper_2608_07524_b200 import inputs
+    q, k, v, g = inputs.make_qkvg(seq_len, n_heads, head_dim, seed)
+    cu = [0, seq_len]
+    t0 = time.perf_counter()
+    oracle.attn_fwd(q, k, v, cu, causal)
+    oracle.attn_bwd(q, k, v, g, cu, causal)
+    dt = time.perf_counter() - t0
+    flops = 14.0 * seq_len * seq_len * head_dim * n_heads * (0.5 if causal else 1.0)
+    return dt, flops
+
+
+def run_reference(args):
+    """The oracle as the reference arm: each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    w = workload(args.workload) or workload("video")
+    L = 2048
+    sample = f"one {L}-token sequence of the {w.name} workload, {w.n_heads} heads, head_dim {w.head_dim}, fwd+bwd in fp64"
+    for _ in range(args.warmup):
+        oracle_sample(L, w.n_heads, w.head_dim, w.causal)
+    total, flops = 0.0, 0.0
+    for _ in range(args.steps):
+        dt, f = oracle_sample(L, w.n_heads, w.head_dim, w.causal)
+        total += dt
+        flops += f
+    value = flops / total / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{w.name} (bounded sample)", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ CUDA arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2608_07524_b200 import binding as B
+    from paper_2608_07524_b200 import inputs
+    from paper_2608_07524_b200.stream import StreamRunner, plan_batch
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the attention path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    B.lib()      # fail loudly here if libdcp.so is missing
+
+    if args.workload == "stream":
+        batches = inputs.stream_batches()[: args.stream_batches]
+        H, d, causal = 16, 128, False
+        name = f"stream: {len(batches)} batches of the video length mix, Lambda={args.layers}, budget {args.budget_gb} GB"
+    else:
+        w = workload(args.workload)
+        batches, H, d, causal = [w.lengths], w.n_heads, w.head_dim, w.causal
+        name = {"video": "config 3 video-DiT-like: 24 sequences, 124992 tokens, 16 heads, head_dim 128, bidirectional",
+                "text": "config 2 text-like: 32 sequences, 79299 tokens, 16 heads, head_dim 128, causal",
+                "extreme": "config 4 extreme imbalance: 131072 + 64 short, 206646 tokens, 8 heads, head_dim 128, causal"}[args.workload]
+    budget = int(args.budget_gb * 10 ** 9)
+    max_tokens = max(sum(b) for b in batches)
+    max_seqs = max(len(b) for b in batches)
+    runner = StreamRunner(max_tokens, max_seqs, H, d, causal, dev, value_seed=12 + 100 * rank)
+
+    def flops_of(lengths):
+        f = 14.0 * sum(float(L) * L for L in lengths) * d * H
+        return 0.5 * f if causal else f
+
+    def step():
+        tokens, flops = 0, 0.0
+        for lengths in batches:
+            for mb in plan_batch(lengths, budget, H, d, n_layers=args.layers):
+                tokens += runner.run_micro_batch(mb)
+                flops += flops_of(mb.lengths)
+        return tokens, flops
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    runner.check()
+
+    sampler = ClockSampler(physical_gpu_index(local))
+    B.dcp_profile_enable(True)
+    B.dcp_profile_read()
+    barrier()
+    sampler.start()
+    launches0 = B.dcp_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    tokens = flops = 0
+    for _ in range(args.steps):
+        t, f = step()
+        tokens += t
+        flops += f
+    e1.record()
+    torch.cuda.synchronize()
+    ms_total = e0.elapsed_time(e1)
+    launches = B.dcp_launch_count() - launches0
+    barrier()
+    clocks = sampler.stop()
+    prof = B.dcp_profile_read()
+    B.dcp_profile_enable(False)
+    runner.check()
+
+    t_ms = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    totals = torch.tensor([flops, float(tokens)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+        dist.all_reduce(totals, op=dist.ReduceOp.SUM)
+    ms_total = float(t_ms.item())
+    flops_all, tokens_all = float(totals[0].item()), float(totals[1].item())
+    value = flops_all / (ms_total * 1e-3) / 1e12
+
+    # ---- end-to-end: same path with HOST buffers, copies inside the timed region (single-batch workloads)
+    e2e = None
+    if args.workload != "stream":
+        T = max_tokens
+        host_in = [torch.empty((T, H, d), dtype=torch.bfloat16).pin_memory() for _ in range(4)]
+        for hbuf, dbuf in zip(host_in, (runner.q, runner.k, runner.v, runner.g)):
+            hbuf.copy_(dbuf[:T])
+        host_out = [torch.empty((T, H, d), dtype=torch.bfloat16).pin_memory() for _ in range(4)]
+        host_lse = torch.empty((H * T,), dtype=torch.float32).pin_memory()
+        n_e2e = max(1, min(args.steps, 3))
+
+        def e2e_step():
+            for hbuf, dbuf in zip(host_in, (runner.q, runner.k, runner.v, runner.g)):
+                dbuf[:T].copy_(hbuf, non_blocking=True)
+            step()
+            for hbuf, dbuf in zip(host_out, (runner.o, runner.dq, runner.dk, runner.dv)):
+                hbuf.copy_(dbuf[:T], non_blocking=True)
+            host_lse.copy_(runner.lse[: H * T], non_blocking=True)
+
+        e2e_step()
+        barrier()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        s1.record()
+        torch.cuda.synchronize()
+        e2e_ms = torch.tensor([s0.elapsed_time(s1)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+        runner.check()
+        per_step_flops = flops_all / args.steps
+        h2d = 4 * T * H * d * 2
+        d2h = 4 * T * H * d * 2 + 4 * H * T
+        e2e = {"value": per_step_flops * n_e2e / (float(e2e_ms.item()) * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e}
+        del host_in, host_out, host_lse
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    bwd_ms, bwd_n = prof["bwd_main"]
+    fwd_ms, fwd_n = prof["fwd"]
+    bwd_flops_per_launch = (flops / args.steps) * (2.5 / 3.5) / max(bwd_n / args.steps, 1)
+    achieved = bwd_flops_per_launch / (bwd_ms / max(bwd_n, 1) * 1e-3) / 1e12 if bwd_n else None
+    roofline = {"bound": "tensor", "kernel": "attn_bwd_kernel (backward main)", "achieved": achieved,
+                "peak": peaks["sustained"], "unit": UNIT, "frac": (achieved / peaks["sustained"]) if achieved else None,
+                "peak_source": f"bf16_tflops_sustained of {peaks['source']} MEASURED_PEAKS.json",
+                "traffic": BWD_MAIN_DRAM_BYTES_PER_LAUNCH,
+                "launches": bwd_n, "avg_launch_ms": bwd_ms / max(bwd_n, 1)}
+
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        Ls = 3600
+        dt, f = oracle_sample(Ls, H, d, causal)
+        cpu_baseline = {"value": f / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                        "sample": f"one {Ls}-token sequence, {H} heads, head_dim {d}, fwd+bwd in fp64, {dt:.1f} s"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": name, "l2": "inputs (2 GB+) larger than L2, no flush", "hbm_budget_bytes": budget,
+                   "n_layers": args.layers},
+        "tokens_per_s": tokens_all / (ms_total * 1e-3),
+        "frac_of_bf16_peak": {"burst": value / world / peaks["burst"], "sustained": value / world / peaks["sustained"],
+                              "source": peaks["source"]},
+        "kernel_ms_per_step": {k: v[0] / args.steps for k, v in prof.items()},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="video", choices=["video", "text", "extreme", "stream"])
+    ap.add_argument("--stream-batches", type=int, default=256)
+    ap.add_argument("--layers", type=int, default=1, help="planner's layer count Lambda")
+    ap.add_argument("--budget-gb", type=float, default=180.0, help="planner's HBM budget in decimal GB")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

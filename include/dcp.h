@@ -107,6 +107,21 @@ int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, const void*
  * DCP_ERR_CUDA. */
 int dcp_query_status(const void* workspace, void* cuda_stream);
 
+/* Measurement aid (no counterpart in the paper).  While enabled, every attention call records a
+ * pair of CUDA events around each kernel it launches, on the caller's stream.  dcp_profile_read
+ * waits for those events, adds up device time (ms) and launch counts per kernel since the previous
+ * read into ms[DCP_N_KERNELS] and launches[DCP_N_KERNELS] (host pointers), and forgets them. */
+enum {
+    DCP_KERNEL_PREP = 0,     /* work-list construction            */
+    DCP_KERNEL_FWD = 1,      /* forward attention                 */
+    DCP_KERNEL_BWD_PRE = 2,  /* D = rowsum(dO*O), zero dQ accum.  */
+    DCP_KERNEL_BWD_MAIN = 3, /* backward attention                */
+    DCP_KERNEL_BWD_POST = 4, /* dQ fp32 -> bf16                   */
+    DCP_N_KERNELS = 5
+};
+int dcp_profile_enable(int on);
+int dcp_profile_read(float* ms, int64_t* launches);
+
 /* Number of kernel launches this library has enqueued since it was loaded (all threads). */
 int64_t dcp_launch_count(void);
 

@@ -57,6 +57,10 @@ def lib():
             L.dcp_varlen_attn_bwd.restype = ctypes.c_int
             L.dcp_query_status.argtypes = [vp, vp]
             L.dcp_query_status.restype = ctypes.c_int
+            L.dcp_profile_enable.argtypes = [ctypes.c_int]
+            L.dcp_profile_enable.restype = ctypes.c_int
+            L.dcp_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int64)]
+            L.dcp_profile_read.restype = ctypes.c_int
             L.dcp_launch_count.argtypes = []
             L.dcp_launch_count.restype = ctypes.c_int64
             L.dcp_last_error.argtypes = []
@@ -68,6 +72,21 @@ def lib():
 def _check(rc: int):
     if rc != DCP_OK:
         raise DcpError(rc, lib().dcp_last_error().decode(errors="replace"))
+
+
+KERNEL_NAMES = ("prep", "fwd", "bwd_pre", "bwd_main", "bwd_post")
+
+
+def dcp_profile_enable(on: bool) -> None:
+    _check(lib().dcp_profile_enable(int(bool(on))))
+
+
+def dcp_profile_read():
+    """{kernel name: (device ms, launches)} accumulated since the previous read."""
+    ms = (ctypes.c_float * len(KERNEL_NAMES))()
+    n = (ctypes.c_int64 * len(KERNEL_NAMES))()
+    _check(lib().dcp_profile_read(ms, n))
+    return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(KERNEL_NAMES)}
 
 
 def dcp_launch_count() -> int:

@@ -9,6 +9,7 @@
 #include <cstdint>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "../../include/dcp.h"
 #include "attn_kernels.h"
@@ -25,6 +26,32 @@ char* error_buffer() {
 namespace {
 
 std::atomic<int64_t> g_launches{0};
+
+// Optional per-kernel timing: event pairs recorded on the caller's stream around every launch.
+struct TimedLaunch {
+    int kernel;
+    cudaEvent_t start, stop;
+};
+std::mutex g_prof_mu;
+std::atomic<int> g_prof_on{0};
+std::vector<TimedLaunch> g_prof_pending;
+
+struct ScopedTimer {
+    int kernel;
+    cudaStream_t stream;
+    cudaEvent_t start = nullptr, stop = nullptr;
+    ScopedTimer(int k, cudaStream_t s) : kernel(k), stream(s) {
+        if (!g_prof_on.load()) return;
+        if (cudaEventCreate(&start) != cudaSuccess || cudaEventCreate(&stop) != cudaSuccess) { start = stop = nullptr; return; }
+        cudaEventRecord(start, stream);
+    }
+    ~ScopedTimer() {
+        if (!start) return;
+        cudaEventRecord(stop, stream);
+        std::lock_guard<std::mutex> lock(g_prof_mu);
+        g_prof_pending.push_back({kernel, start, stop});
+    }
+};
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -158,7 +185,11 @@ extern "C" int dcp_varlen_attn_fwd(const void* q, const void* k, const void* v, 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
     const SchedView sched = carve_sched(workspace, n_seqs);
-    cudaError_t e = launch_prep(cu_seqlens, n_seqs, kFwdRowsPerItem, n_heads, sched, stream);
+    cudaError_t e;
+    {
+        ScopedTimer t(DCP_KERNEL_PREP, stream);
+        e = launch_prep(cu_seqlens, n_seqs, kFwdRowsPerItem, n_heads, sched, stream);
+    }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: work-list kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(1);
     if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
@@ -177,7 +208,10 @@ extern "C" int dcp_varlen_attn_fwd(const void* q, const void* k, const void* v, 
     p.total_tokens = total_tokens;
     p.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
     p.scale_log2 = p.scale * 1.4426950408889634f;
-    e = launch_attn_fwd(tq, tk, tv, p, head_dim, causal != 0, dev.sm_count, stream);
+    {
+        ScopedTimer t(DCP_KERNEL_FWD, stream);
+        e = launch_attn_fwd(tq, tk, tv, p, head_dim, causal != 0, dev.sm_count, stream);
+    }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: attention kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(1);
     return DCP_OK;
@@ -212,7 +246,11 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
     float* dsum = reinterpret_cast<float*>(base);
     float* dq_acc = reinterpret_cast<float*>(base + align256(sizeof(float) * (size_t)total_tokens * n_heads));
 
-    cudaError_t e = launch_prep(cu_seqlens, n_seqs, kTile, n_heads, sched, stream);
+    cudaError_t e;
+    {
+        ScopedTimer t(DCP_KERNEL_PREP, stream);
+        e = launch_prep(cu_seqlens, n_seqs, kTile, n_heads, sched, stream);
+    }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: work-list kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(1);
     if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
@@ -223,8 +261,11 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
     if (int rc = make_map(&tv, v, total_tokens, n_heads, head_dim)) return rc;
     if (int rc = make_map(&tg, d_o, total_tokens, n_heads, head_dim)) return rc;
 
-    e = launch_bwd_pre(static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), dsum, dq_acc,
-                       total_tokens, n_heads, head_dim, stream);
+    {
+        ScopedTimer t(DCP_KERNEL_BWD_PRE, stream);
+        e = launch_bwd_pre(static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), dsum, dq_acc,
+                           total_tokens, n_heads, head_dim, stream);
+    }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: pre kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(1);
 
@@ -240,11 +281,17 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
     p.total_tokens = total_tokens;
     p.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
     p.scale_log2 = p.scale * 1.4426950408889634f;
-    e = launch_attn_bwd(tq, tk, tv, tg, p, head_dim, causal != 0, dev.sm_count, stream);
+    {
+        ScopedTimer t(DCP_KERNEL_BWD_MAIN, stream);
+        e = launch_attn_bwd(tq, tk, tv, tg, p, head_dim, causal != 0, dev.sm_count, stream);
+    }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: main kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(1);
 
-    e = launch_bwd_post(dq_acc, static_cast<__nv_bfloat16*>(dq), (size_t)total_tokens * n_heads * head_dim, p.scale, stream);
+    {
+        ScopedTimer t(DCP_KERNEL_BWD_POST, stream);
+        e = launch_bwd_post(dq_acc, static_cast<__nv_bfloat16*>(dq), (size_t)total_tokens * n_heads * head_dim, p.scale, stream);
+    }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: post kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(1);
     return DCP_OK;
@@ -259,4 +306,30 @@ extern "C" int dcp_query_status(const void* workspace, void* cuda_stream) {
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "dcp_query_status: %s", cudaGetErrorString(e));
     if (status != 0) return fail(DCP_ERR_TIMEOUT, "a kernel abandoned a bounded wait (device status %u); results are invalid", status);
     return DCP_OK;
+}
+
+extern "C" int dcp_profile_enable(int on) {
+    g_prof_on.store(on ? 1 : 0);
+    return DCP_OK;
+}
+
+extern "C" int dcp_profile_read(float* ms, int64_t* launches) {
+    if (!ms || !launches) return fail(DCP_ERR_INVALID_ARG, "dcp_profile_read: null pointer");
+    std::vector<TimedLaunch> pending;
+    {
+        std::lock_guard<std::mutex> lock(g_prof_mu);
+        pending.swap(g_prof_pending);
+    }
+    for (int i = 0; i < DCP_N_KERNELS; ++i) { ms[i] = 0.f; launches[i] = 0; }
+    int rc = DCP_OK;
+    for (const TimedLaunch& t : pending) {
+        float one = 0.f;
+        cudaError_t e = cudaEventSynchronize(t.stop);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&one, t.start, t.stop);
+        if (e != cudaSuccess) rc = fail(DCP_ERR_CUDA, "dcp_profile_read: %s", cudaGetErrorString(e));
+        else { ms[t.kernel] += one; launches[t.kernel] += 1; }
+        cudaEventDestroy(t.start);
+        cudaEventDestroy(t.stop);
+    }
+    return rc;
 }

@@ -1,0 +1,92 @@
+"""Host loop of the end-to-end stream: plan a batch, then run every micro-batch through the kernels.
+
+Per batch (Section 3.1 of the paper: settings are re-chosen for every incoming batch):
+    dcp_plan(lengths, budget)  ->  micro-batches (gradient-accumulation steps) and recompute counts
+    for each micro-batch:      forward; forward again if its recompute count > 0 (activation
+                               recomputation re-runs the layer's forward before its backward,
+                               Section 3.4); backward.
+All arithmetic happens in libdcp; this module only slices buffers and issues calls.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List, Sequence
+
+from . import binding
+
+
+@dataclass
+class MicroBatch:
+    lengths: List[int]        # in planner order (longest first)
+    recompute: int            # layers whose forward is re-run before backward
+
+    @property
+    def total_tokens(self) -> int:
+        return sum(self.lengths)
+
+
+def plan_batch(lengths: Sequence[int], hbm_budget_bytes: int, n_heads: int, head_dim: int,
+               n_layers: int = 1, fixed_cost: int = 1 << 24) -> List[MicroBatch]:
+    mb_id, recompute, _ = binding.dcp_plan(lengths, hbm_budget_bytes, n_heads=n_heads, head_dim=head_dim,
+                                           n_layers=n_layers, fixed_cost=fixed_cost)
+    out = [MicroBatch([], r) for r in recompute]
+    # inside a micro-batch keep the planner's order: longest first, ties by input index
+    for i in sorted(range(len(lengths)), key=lambda i: (-lengths[i], i)):
+        out[mb_id[i]].lengths.append(int(lengths[i]))
+    return out
+
+
+class StreamRunner:
+    """Runs micro-batches out of pre-allocated device buffers sized for the largest micro-batch.
+
+    The synthetic stream reuses the first `tokens` rows of the q/k/v/dO buffers for every
+    micro-batch (the values are random either way); outputs go to preallocated tensors.
+    """
+
+    def __init__(self, max_tokens: int, max_seqs: int, n_heads: int, head_dim: int, causal: bool, device,
+                 value_seed: int = 20):
+        import torch
+        from . import inputs
+        self.torch = torch
+        self.H, self.d, self.causal, self.device = n_heads, head_dim, causal, device
+        self.q, self.k, self.v, self.g = inputs.make_qkvg_device(max_tokens, n_heads, head_dim, value_seed, device)
+        self.o = torch.empty_like(self.q)
+        self.dq, self.dk, self.dv = (torch.empty_like(self.q) for _ in range(3))
+        self.lse = torch.empty(n_heads * max_tokens, dtype=torch.float32, device=device)
+        _, bwd_bytes = binding.dcp_varlen_attn_workspace(max_tokens, max_seqs, n_heads, head_dim)
+        self.ws = torch.empty(bwd_bytes, dtype=torch.uint8, device=device)
+        # cu_seqlens travel through a small ring of pinned host / device slots; a slot is reused
+        # only after the copy that read it has finished (tracked by an event per slot)
+        self.n_slots = 16
+        self.cu_host = torch.empty((self.n_slots, max_seqs + 1), dtype=torch.int32).pin_memory()
+        self.cu_dev = torch.empty((self.n_slots, max_seqs + 1), dtype=torch.int32, device=device)
+        self.cu_events = [None] * self.n_slots
+        self.calls = 0
+
+    def run_micro_batch(self, mb: MicroBatch) -> int:
+        """Enqueue forward (+ recompute forward) + backward for one micro-batch; returns its tokens."""
+        torch = self.torch
+        n, T = len(mb.lengths), mb.total_tokens
+        slot = self.calls % self.n_slots
+        self.calls += 1
+        if self.cu_events[slot] is not None:
+            self.cu_events[slot].synchronize()
+        cu = self.cu_host[slot, : n + 1]
+        cu[0] = 0
+        cu[1:] = torch.tensor(mb.lengths, dtype=torch.int32).cumsum(0)
+        cu_dev = self.cu_dev[slot, : n + 1]
+        cu_dev.copy_(cu, non_blocking=True)
+        ev = torch.cuda.Event()
+        ev.record()
+        self.cu_events[slot] = ev
+        q, k, v, g, o = (x[:T] for x in (self.q, self.k, self.v, self.g, self.o))
+        lse = self.lse[: self.H * T].view(self.H, T)
+        max_len = max(mb.lengths)
+        for _ in range(1 + (1 if mb.recompute > 0 else 0)):
+            binding.dcp_varlen_attn_fwd(q, k, v, cu_dev, max_len, self.causal, out=o, lse=lse, workspace=self.ws)
+        binding.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cu_dev, max_len, self.causal, dq=self.dq[:T], dk=self.dk[:T],
+                                    dv=self.dv[:T], workspace=self.ws)
+        return T
+
+    def check(self):
+        binding.dcp_query_status(self.ws)

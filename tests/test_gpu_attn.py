@@ -1,0 +1,164 @@
+"""Parity of the CUDA attention path (through the C ABI) against the fp64 CPU oracle.
+
+Tolerances (bf16 outputs upcast to fp64, both must hold per tensor):
+    max-abs <= 5e-2  and  ||x - ref||_F / ||ref||_F <= 1e-2;   lse (fp32): max-abs <= 2e-3.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_07524_b200 import binding as B
+from paper_2608_07524_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, REL_FRO, LSE_ABS = 5e-2, 1e-2, 2e-3
+
+
+def to64(x):
+    return x.detach().double().cpu().numpy()
+
+
+def assert_close(name, got, ref):
+    got = to64(got) if torch.is_tensor(got) else got
+    assert got.shape == ref.shape, name
+    assert np.all(np.isfinite(got)), f"{name}: non-finite values"
+    max_abs = float(np.max(np.abs(got - ref))) if ref.size else 0.0
+    rel = float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)) if ref.size else 0.0
+    assert max_abs <= MAX_ABS and rel <= REL_FRO, f"{name}: max-abs {max_abs:.3e}, rel-Frobenius {rel:.3e}"
+
+
+def run_gpu(q, k, v, g, cu, causal, scale=0.0, o_override=None, lse_override=None):
+    dev = "cuda"
+    cud = torch.tensor(np.asarray(cu), dtype=torch.int32, device=dev)
+    lens = np.diff(np.asarray(cu))
+    max_len = int(lens.max()) if lens.size else 0
+    qd, kd, vd, gd = (x.to(dev) for x in (q, k, v, g))
+    T, H, d = q.shape
+    ws = B.alloc_workspace(T, len(lens), H, d, True, dev)
+    o, lse = B.dcp_varlen_attn_fwd(qd, kd, vd, cud, max_len, causal, scale, workspace=ws)
+    B.dcp_query_status(ws)
+    o_in = o if o_override is None else o_override.to(dev)
+    lse_in = lse if lse_override is None else lse_override.to(dev)
+    dq, dk, dv = B.dcp_varlen_attn_bwd(qd, kd, vd, o_in, gd, lse_in, cud, max_len, causal, scale, workspace=ws)
+    B.dcp_query_status(ws)
+    return o, lse, dq, dk, dv
+
+
+def check_full(lengths, H, d, causal, seed, scale=0.0):
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    q, k, v, g = inputs.make_qkvg(int(cu[-1]), H, d, seed)
+    o, lse, dq, dk, dv = run_gpu(q, k, v, g, cu, causal, scale)
+    O, L = oracle.attn_fwd(q, k, v, cu, causal, scale)
+    rdq, rdk, rdv = oracle.attn_bwd(q, k, v, g, cu, causal, scale)
+    assert_close("o", o, O)
+    assert float(np.max(np.abs(to64(lse) - L))) <= LSE_ABS if L.size else True
+    assert_close("dq", dq, rdq)
+    assert_close("dk", dk, rdk)
+    assert_close("dv", dv, rdv)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_config1_tiny(causal):
+    w = inputs.config(1, causal)
+    check_full(w.lengths, w.n_heads, w.head_dim, causal, w.value_seed)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("d", [64, 128])
+def test_ragged_multi_tile(causal, d):
+    # several tiles, ragged tails on both the query and the key side, tile-edge lengths
+    check_full([300, 1000, 129, 128, 1, 513, 127, 256, 257], 3, d, causal, seed=1)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_zero_length_sequences_and_single_tokens(causal):
+    check_full([0, 5, 0, 0, 1, 130, 0], 2, 64, causal, seed=2)
+
+
+def test_all_sequences_empty():
+    q = torch.empty((0, 2, 64), dtype=torch.bfloat16)
+    o, lse, dq, dk, dv = run_gpu(q, q, q, q, [0, 0, 0], False)
+    assert o.numel() == 0 and dq.numel() == 0
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_custom_softmax_scale(causal):
+    check_full([200, 77], 2, 128, causal, seed=3, scale=0.05)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_many_short_sequences(causal):
+    rng = np.random.default_rng(5)
+    check_full([int(x) for x in rng.integers(1, 200, size=300)], 2, 64, causal, seed=5)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_backward_in_isolation(causal):
+    """Backward fed with the oracle's own O (rounded to bf16) and lse (fp32) instead of the GPU
+    forward's, so a forward error cannot hide or cause a backward one."""
+    lengths = [384, 100, 250]
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    q, k, v, g = inputs.make_qkvg(int(cu[-1]), 2, 128, 7)
+    O, L = oracle.attn_fwd(q, k, v, cu, causal)
+    o_in = torch.from_numpy(O).to(torch.bfloat16)
+    lse_in = torch.from_numpy(L).to(torch.float32)
+    _, _, dq, dk, dv = run_gpu(q, k, v, g, cu, causal, o_override=o_in, lse_override=lse_in)
+    rdq, rdk, rdv = oracle.attn_bwd(q, k, v, g, cu, causal)
+    assert_close("dq", dq, rdq)
+    assert_close("dk", dk, rdk)
+    assert_close("dv", dv, rdv)
+
+
+def test_packing_independence_on_gpu():
+    """A sequence's outputs do not change when its neighbours' data change (tail tiles read the
+    next sequence's rows through TMA, so the masks must hide them completely)."""
+    lengths = [100, 200, 150]
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    q, k, v, g = inputs.make_qkvg(int(cu[-1]), 2, 128, 9)
+    a = run_gpu(q, k, v, g, cu, False)
+    q2, k2, v2, g2 = (x.clone() for x in (q, k, v, g))
+    for x in (q2, k2, v2, g2):
+        x[:100] = torch.randn_like(x[:100].float()).to(torch.bfloat16) * 3
+        x[300:] = torch.randn_like(x[300:].float()).to(torch.bfloat16) * 3
+    b = run_gpu(q2, k2, v2, g2, cu, False)
+    for i in (0, 3, 4):        # o, dk, dv: no atomics involved, bit-exact
+        assert torch.equal(a[i][100:300], b[i][100:300])
+    assert torch.equal(a[1][:, 100:300], b[1][:, 100:300])
+    # dq is summed with atomics in arbitrary order: compare within rounding
+    assert float((a[2][100:300].float() - b[2][100:300].float()).abs().max()) <= 2e-2
+
+
+def test_library_rejects_bad_arguments():
+    dev = "cuda"
+    q = torch.zeros((10, 2, 96), dtype=torch.bfloat16, device=dev)
+    cu = torch.tensor([0, 10], dtype=torch.int32, device=dev)
+    with pytest.raises(B.DcpError) as e:
+        B.dcp_varlen_attn_fwd(q, q, q, cu, 10, False)
+    assert e.value.code == B.DCP_ERR_UNSUPPORTED
+    q = torch.zeros((10, 2, 64), dtype=torch.bfloat16, device=dev)
+    small = torch.empty(16, dtype=torch.uint8, device=dev)
+    with pytest.raises(B.DcpError) as e:
+        B.dcp_varlen_attn_fwd(q, q, q, cu, 10, False, workspace=small)
+    assert e.value.code == B.DCP_ERR_WORKSPACE
+    with pytest.raises(B.DcpError) as e:
+        B.dcp_varlen_attn_fwd(q, q, q, cu, 10, False, softmax_scale=-1.0)
+    assert e.value.code == B.DCP_ERR_INVALID_ARG
+    with pytest.raises(B.DcpError) as e:
+        B.dcp_varlen_attn_fwd(q, q, q, cu, 11, False)
+    assert e.value.code == B.DCP_ERR_INVALID_ARG
+
+
+def test_launch_counter_and_profile():
+    w = inputs.config(1, False)
+    q, k, v, g = inputs.make_qkvg(w.total_tokens, w.n_heads, w.head_dim, 4)
+    B.dcp_profile_enable(True)
+    B.dcp_profile_read()
+    before = B.dcp_launch_count()
+    run_gpu(q, k, v, g, w.cu_seqlens, False)
+    assert B.dcp_launch_count() - before == 2 + 4          # forward: prep + main; backward: prep + 3
+    prof = B.dcp_profile_read()
+    B.dcp_profile_enable(False)
+    assert prof["fwd"][1] == 1 and prof["bwd_main"][1] == 1 and prof["prep"][1] == 2
+    assert prof["fwd"][0] > 0 and prof["bwd_main"][0] > 0

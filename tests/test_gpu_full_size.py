@@ -1,0 +1,117 @@
+"""Full-size benchmark configurations (2 text, 3 video, 4 extreme imbalance) in the launch
+configuration the benchmark times.  A full fp64 evaluation of these is 10^13-10^14 flop, so the
+oracle checks (a) sampled query rows (O, lse, dQ) and key columns (dK, dV), which the definition
+lets it compute one by one, (b) the shortest sequences completely, on every head, and (c) two
+whole-tensor identities that hold at any size:
+    sum_i <Q_i, dQ_i> = sum_j <K_j, dK_j>      and      sum_j dV_j = sum_i dO_i
+per (sequence, head), evaluated on the GPU results in fp64.  Their bounds have two parts: the
+independent bf16 rounding of every stored gradient element (8 sigma), and a term proportional to
+the absolute sum for the tensor cores' fp32 accumulation, which truncates instead of rounding and
+so biases sums of thousands of partial products by about 1e-4 of their magnitude.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_07524_b200 import binding as B
+from paper_2608_07524_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, REL_FRO, LSE_ABS = 5e-2, 1e-2, 2e-3
+EPS_BF16 = 2.0 ** -9
+ACC_BIAS = 5e-4
+
+
+def close(name, got, ref):
+    got = got.detach().double().cpu().numpy()
+    max_abs = float(np.max(np.abs(got - ref)))
+    rel = float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30))
+    assert np.all(np.isfinite(got)), name
+    assert max_abs <= MAX_ABS and rel <= REL_FRO, f"{name}: max-abs {max_abs:.3e}, rel-Frobenius {rel:.3e}"
+
+
+def sample_positions(L, rng, n_random=24):
+    fixed = [0, 1, 127, 128, 255, 256, L - 257, L - 256, L - 129, L - 128, L - 2, L - 1, L // 2]
+    pos = {p for p in fixed if 0 <= p < L}
+    pos.update(int(x) for x in rng.integers(0, L, size=n_random))
+    return np.array(sorted(pos), np.int32)
+
+
+@pytest.fixture(scope="module", params=[2, 3, 4])
+def full_run(request):
+    w = inputs.config(request.param)
+    dev = "cuda"
+    q, k, v, g = inputs.make_qkvg_device(w.total_tokens, w.n_heads, w.head_dim, w.value_seed, dev)
+    cud = torch.tensor(w.cu_seqlens, dtype=torch.int32, device=dev)
+    ws = B.alloc_workspace(w.total_tokens, len(w.lengths), w.n_heads, w.head_dim, True, dev)
+    o, lse = B.dcp_varlen_attn_fwd(q, k, v, cud, w.max_seqlen, w.causal, workspace=ws)
+    B.dcp_query_status(ws)
+    dq, dk, dv = B.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cud, w.max_seqlen, w.causal, workspace=ws)
+    B.dcp_query_status(ws)
+    del ws
+    host = tuple(x.cpu() for x in (q, k, v, g))
+    yield w, (q, k, v, g), host, (o, lse, dq, dk, dv)
+    torch.cuda.empty_cache()
+
+
+def test_sampled_rows_and_columns(full_run):
+    w, _, (q, k, v, g), (o, lse, dq, dk, dv) = full_run
+    rng = np.random.default_rng(100 + len(w.lengths))
+    order = np.argsort(w.lengths)
+    seqs = [int(order[-1]), int(order[len(order) // 2]), int(order[0])]      # longest, median, shortest
+    for seq in seqs:
+        L, c0 = w.lengths[seq], w.cu_seqlens[seq]
+        for head in (0, w.n_heads - 1):
+            rows = sample_positions(L, rng)
+            Or, lr, dqr = oracle.attn_rows(q, k, v, g, w.cu_seqlens, w.causal, seq, head, rows)
+            idx = torch.tensor(c0 + rows, device="cuda").long()
+            close(f"o seq {seq} head {head}", o[idx, head], Or)
+            close(f"dq seq {seq} head {head}", dq[idx, head], dqr)
+            assert float(np.max(np.abs(lse[head, idx].double().cpu().numpy() - lr))) <= LSE_ABS
+        # columns: one head per sequence.  Under a causal mask a column needs the statistics of
+        # every later row, so for very long sequences only columns near the end are sampled here
+        # (early columns are covered by the identities and by the shorter sequences).
+        head = 1
+        cols = sample_positions(L, rng, n_random=8)
+        if w.causal and L > 16384:
+            cols = cols[cols >= L - 2048]
+        dkc, dvc = oracle.attn_cols(q, k, v, g, w.cu_seqlens, w.causal, seq, head, cols)
+        idx = torch.tensor(c0 + cols, device="cuda").long()
+        close(f"dk seq {seq}", dk[idx, head], dkc)
+        close(f"dv seq {seq}", dv[idx, head], dvc)
+
+
+def test_shortest_sequences_in_full(full_run):
+    w, _, (q, k, v, g), (o, lse, dq, dk, dv) = full_run
+    order = np.argsort(w.lengths)
+    for seq in (int(order[0]), int(order[1])):
+        L, c0 = w.lengths[seq], w.cu_seqlens[seq]
+        sl = slice(c0, c0 + L)
+        O, Lse = oracle.attn_fwd(q[sl], k[sl], v[sl], [0, L], w.causal)
+        rdq, rdk, rdv = oracle.attn_bwd(q[sl], k[sl], v[sl], g[sl], [0, L], w.causal)
+        close("o", o[sl], O)
+        close("dq", dq[sl], rdq)
+        close("dk", dk[sl], rdk)
+        close("dv", dv[sl], rdv)
+        assert float(np.max(np.abs(lse[:, sl].double().cpu().numpy() - Lse))) <= LSE_ABS
+
+
+def test_whole_tensor_identities(full_run):
+    w, (q, k, v, g), _, (o, lse, dq, dk, dv) = full_run
+    for seq, L in enumerate(w.lengths):
+        sl = slice(w.cu_seqlens[seq], w.cu_seqlens[seq] + L)
+        qd = q[sl].double() * dq[sl].double()
+        kd = k[sl].double() * dk[sl].double()
+        lhs, rhs = qd.sum(dim=(0, 2)), kd.sum(dim=(0, 2))
+        # both sides carry independent bf16 rounding of every gradient element
+        bound = (8 * EPS_BF16 * torch.sqrt((qd * qd).sum(dim=(0, 2)) + (kd * kd).sum(dim=(0, 2)))
+                 + ACC_BIAS * (qd.abs().sum(dim=(0, 2)) + kd.abs().sum(dim=(0, 2))) + 1e-6)
+        assert bool(((lhs - rhs).abs() <= bound).all()), f"<Q,dQ> vs <K,dK> on sequence {seq}"
+        del qd, kd
+        dvs = dv[sl].double()
+        lhs, rhs = dvs.sum(dim=0), g[sl].double().sum(dim=0)
+        bound = 8 * EPS_BF16 * torch.sqrt((dvs * dvs).sum(dim=0)) + ACC_BIAS * dvs.abs().sum(dim=0) + 1e-6
+        assert bool(((lhs - rhs).abs() <= bound).all()), f"sum dV vs sum dO on sequence {seq}"
+    assert bool(torch.isfinite(o.float()).all()) and bool(torch.isfinite(lse).all())

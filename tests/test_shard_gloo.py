@@ -1,0 +1,61 @@
+"""Multi-rank host logic on CPU: two gloo ranks shard a batch with no data-path collective, and
+the benchmark's max-over-ranks reduction works."""
+import os
+import socket
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from paper_2608_07524_b200 import inputs
+from paper_2608_07524_b200.shard import imbalance, shard_sequences
+
+
+def test_shards_partition_and_balance():
+    lengths = inputs.video_lengths()
+    for world in (1, 2, 4, 8):
+        owned = shard_sequences(lengths, world)
+        assert sorted(i for idx in owned for i in idx) == list(range(len(lengths)))
+    # one 46800-token sequence dominates sum L^2, so two ranks cannot balance; the longest still
+    # sits alone with the short ones elsewhere
+    owned = shard_sequences(lengths, 2)
+    longest = lengths.index(max(lengths))
+    r = next(r for r in range(2) if longest in owned[r])
+    assert owned[r] == [longest]
+    assert imbalance(inputs.text_lengths(), shard_sequences(inputs.text_lengths(), 2)) < 1.05
+
+
+def _worker(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    lengths = inputs.text_lengths()
+    mine = shard_sequences(lengths, world)[rank]
+    gathered = [None] * world
+    dist.all_gather_object(gathered, mine)
+    t = torch.tensor([10.0 + rank])                      # stand-in for this rank's elapsed time
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    tokens = torch.tensor([float(sum(lengths[i] for i in mine))])
+    dist.all_reduce(tokens, op=dist.ReduceOp.SUM)
+    if rank == 0:
+        out.put((gathered, float(t), float(tokens)))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    gathered, tmax, tokens = out.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    lengths = inputs.text_lengths()
+    assert sorted(gathered[0] + gathered[1]) == list(range(len(lengths)))
+    assert tmax == 11.0 and tokens == float(sum(lengths))
