@@ -170,10 +170,13 @@ def run_ours(args):
         name = f"stream: {len(batches)} batches of the video length mix, Lambda={args.layers}, budget {args.budget_gb} GB"
     else:
         w = workload(args.workload)
-        batches, H, d, causal = [w.lengths], w.n_heads, w.head_dim, w.causal
+        lengths = [L for L in w.lengths if not args.drop_longer_than or L <= args.drop_longer_than]
+        batches, H, d, causal = [lengths], w.n_heads, w.head_dim, w.causal
         name = {"video": "config 3 video-DiT-like: 24 sequences, 124992 tokens, 16 heads, head_dim 128, bidirectional",
                 "text": "config 2 text-like: 32 sequences, 79299 tokens, 16 heads, head_dim 128, causal",
                 "extreme": "config 4 extreme imbalance: 131072 + 64 short, 206646 tokens, 8 heads, head_dim 128, causal"}[args.workload]
+        if args.drop_longer_than:
+            name += f" (profiling subset: sequences longer than {args.drop_longer_than} dropped)"
     budget = int(args.budget_gb * 10 ** 9)
     max_tokens = max(sum(b) for b in batches)
     max_seqs = max(len(b) for b in batches)
@@ -322,6 +325,8 @@ def main():
     ap.add_argument("--layers", type=int, default=1, help="planner's layer count Lambda")
     ap.add_argument("--budget-gb", type=float, default=180.0, help="planner's HBM budget in decimal GB")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--drop-longer-than", type=int, default=0,
+                    help="profiling aid: drop sequences longer than this from the workload (0 = keep all)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -8,6 +8,8 @@
 //               accumulators in tensor memory
 //   warp  9     scheduler + TMA producer (one thread): pulls work items from the global counter,
 //               streams Q once and K_j, V_j through a shared-memory ring
+//   warps 10-11 idle; they exist so that warps 8-11 form a group that can hand its registers to
+//               the softmax groups (setmaxnreg), which hold a whole 128-wide score row per thread
 // The two Q tiles alternate on the tensor pipe: while one group runs exp on its S tile, the pipe
 // computes the other tile's products.  P overwrites S in tensor memory as packed bf16 and is the
 // A operand of the second product, so probabilities never touch shared memory.
@@ -25,7 +27,7 @@
 
 namespace dcp {
 
-constexpr int kFwdThreads = 320;
+constexpr int kFwdThreads = 384;   // 8 softmax warps + a 4-warp control group (MMA, producer, 2 idle)
 constexpr int kKvStages = 4;
 constexpr float kRescaleThreshold = 8.0f;   // in log2 units
 
@@ -131,6 +133,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     tc_fence_after();
     const uint32_t tmem = sh.tmem_base;
 
+    if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (warp == 9) {
         // ---------------------------------------------------------------- scheduler + TMA producer
         if (lane == 0) {
@@ -248,7 +252,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 kv_base += 2 * nkv;
             }
         }
+    }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
         // ---------------------------------------------------------------- softmax groups
         const int t = warp >> 2;                        // Q tile of this group
         const int row_in_tile = tid & 127;
@@ -288,9 +294,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     for (int c = 0; c < 128; ++c)
                         if (c >= n_valid) s[c] = 0xff800000u;         // -inf
                 }
-                float mx = __uint_as_float(s[0]);
+                float part[8];      // eight independent chains instead of one 128-long one
 #pragma unroll
-                for (int c = 1; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
+                for (int c = 0; c < 8; ++c) part[c] = __uint_as_float(s[c]);
+#pragma unroll
+                for (int c = 8; c < 128; ++c) part[c & 7] = fmaxf(part[c & 7], __uint_as_float(s[c]));
+                const float mx = fmaxf(fmaxf(fmaxf(part[0], part[1]), fmaxf(part[2], part[3])),
+                                       fmaxf(fmaxf(part[4], part[5]), fmaxf(part[6], part[7])));
 
                 const bool need = (mx - m) * p.scale_log2 > kRescaleThreshold;
                 if (__any_sync(0xffffffffu, need)) {
@@ -311,7 +321,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     }
                 }
                 const float neg_m = -m * p.scale_log2;
-                float sum = 0.f;
+                float sum[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t pk[16];
@@ -319,12 +329,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     for (int i = 0; i < 16; ++i) {
                         const float p0 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + 2 * i]), p.scale_log2, neg_m));
                         const float p1 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + 2 * i + 1]), p.scale_log2, neg_m));
-                        sum += p0 + p1;
+                        sum[i & 3] += p0 + p1;
                         pk[i] = pack_bf16x2(p0, p1);
                     }
                     tmem_st_x16(s_tmem + c * 16, pk);
                 }
-                l += sum;
+                l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
