@@ -35,7 +35,7 @@ def _nvcc() -> str:
 
 
 def _compile(src: str, obj: str, log: str):
-    cmd = [_nvcc(), *NVCC_FLAGS, "-c", src, "-o", obj]
+    cmd = [_nvcc(), *NVCC_FLAGS, *os.environ.get("DCP_EXTRA_NVCC_FLAGS", "").split(), "-c", src, "-o", obj]
     res = subprocess.run(cmd, capture_output=True, text=True)
     with open(log, "w") as f:
         f.write(" ".join(cmd) + "\n" + res.stdout + res.stderr)

@@ -137,6 +137,7 @@ SchedView carve_sched(void* workspace, int32_t n_seqs) {
     s.hdr = reinterpret_cast<WorkspaceHeader*>(base);
     s.order = reinterpret_cast<const int32_t*>(base + sizeof(WorkspaceHeader));
     s.prefix = reinterpret_cast<const uint32_t*>(base + sizeof(WorkspaceHeader) + sizeof(int32_t) * (size_t)n_seqs);
+    s.tile_prefix = s.prefix + (size_t)n_seqs + 1;
     s.n_seqs = n_seqs;
     return s;
 }
@@ -160,7 +161,7 @@ extern "C" int dcp_varlen_attn_workspace(int32_t total_tokens, int32_t n_seqs, i
     if (fwd_bytes) *fwd_bytes = sched;
     if (bwd_bytes)
         *bwd_bytes = sched + align256(sizeof(float) * (size_t)total_tokens * n_heads) +
-                     align256(sizeof(float) * (size_t)total_tokens * n_heads * head_dim);
+                     align256(sizeof(float) * max_tiles(total_tokens, n_seqs) * kTile * n_heads * head_dim);
     return DCP_OK;
 }
 
@@ -264,7 +265,8 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
     {
         ScopedTimer t(DCP_KERNEL_BWD_PRE, stream);
         e = launch_bwd_pre(static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), dsum, dq_acc,
-                           total_tokens, n_heads, head_dim, stream);
+                           max_tiles(total_tokens, n_seqs) * kTile * n_heads * head_dim, total_tokens, n_heads, head_dim,
+                           stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: pre kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(1);
@@ -290,7 +292,8 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
 
     {
         ScopedTimer t(DCP_KERNEL_BWD_POST, stream);
-        e = launch_bwd_post(dq_acc, static_cast<__nv_bfloat16*>(dq), (size_t)total_tokens * n_heads * head_dim, p.scale, stream);
+        e = launch_bwd_post(dq_acc, static_cast<__nv_bfloat16*>(dq), cu_seqlens, sched, n_heads, head_dim, p.scale,
+                            dev.sm_count, stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: post kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(1);

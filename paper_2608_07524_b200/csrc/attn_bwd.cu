@@ -12,12 +12,16 @@
 //     dV  += P^T dO          dK += dS^T Q          dQ_tile = dS K  (dQ aliases dP^T's columns)
 //
 // dQ tiles are added into an fp32 accumulator in global memory with vector atomics because every
-// key block of a sequence contributes to the same query rows; dK and dV stay in tensor memory for
+// key block of a sequence contributes to the same query rows.  The accumulator is a workspace, so
+// its layout is chosen for the atomics: per (tile, head) a block [d/4][128 rows][4 floats], which
+// makes the 32 rows a warp holds contiguous (full 32-byte sectors, four 128-byte lines per
+// instruction instead of 32 scattered ones); a small kernel converts it to [T, H, d] bf16 later. dK and dV stay in tensor memory for
 // the whole item and are written once (dK scaled by the softmax scale).
 //
 // Roles:  warps 0-7 compute (two groups, each owns 64 of the 128 query columns, one key per thread),
-//         warp 8 MMA issue, warp 9 scheduler + TMA producer + per-row statistics staging,
-//         warps 10-13 dQ drain (tensor memory -> global atomics).
+//         warp 8 MMA issue, warp 9 scheduler + TMA producer + per-row statistics staging
+//         (warps 10-11 idle: the control group of four gives most of its registers away),
+//         warps 12-15 dQ drain (tensor memory -> global atomics).
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -26,9 +30,25 @@
 #include "sched.cuh"
 #include "sm100_ptx.cuh"
 
+// Development aid: with -DDCP_TIMING every role of CTA 0..147 accumulates the cycles it spends in
+// each of its waits and phases; dcp_debug_read_timing copies the table out.  Not part of the product build.
+#ifdef DCP_TIMING
+__device__ long long g_bwd_timing[148 * 4 * 16];
+#define TW(i, ...) do { long long _t = clock64(); __VA_ARGS__; tacc[i] += clock64() - _t; } while (0)
+#define TDECL long long tacc[16] = {0}; const long long _t_begin = clock64();
+#define TDUMP(role) do { tacc[15] = clock64() - _t_begin; for (int _i = 0; _i < 16; ++_i) g_bwd_timing[(blockIdx.x * 4 + (role)) * 16 + _i] = tacc[_i]; } while (0)
+extern "C" int dcp_debug_read_timing(long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, g_bwd_timing, sizeof(long long) * 148 * 4 * 16);
+}
+#else
+#define TW(i, ...) __VA_ARGS__
+#define TDECL
+#define TDUMP(role)
+#endif
+
 namespace dcp {
 
-constexpr int kBwdThreads = 448;
+constexpr int kBwdThreads = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int D>
@@ -40,12 +60,14 @@ struct BwdCfg {
     // shared-memory map (offsets from a 1024-byte aligned base)
     static constexpr int kOffK = 0;
     static constexpr int kOffV = kTileBytes;
-    static constexpr int kOffQ = 2 * kTileBytes;          // 2 stages
-    static constexpr int kOffDo = 4 * kTileBytes;         // 2 stages
+    static constexpr int kQStages = 3;                     // Q is needed early (S^T) and late (dK): three stages
+    static constexpr int kOffQ = 2 * kTileBytes;           // so that a load has a whole tile period to land
+    static constexpr int kOffDo = 5 * kTileBytes;          // dO lives only from dP^T to dV: one stage
     static constexpr int kOffDs = 6 * kTileBytes;
-    static constexpr int kOffStat = kOffDs + kDsBytes;    // 2 stages x (128 nlse + 128 D) floats
+    static constexpr int kOffStat = kOffDs + kDsBytes;     // 2 stages x (128 nlse + 128 D) floats
     static constexpr int kOffCtl = kOffStat + 2 * 256 * 4;
-    static constexpr int kSmemBytes = kOffCtl + 512;
+    static constexpr int kSmemBytes = kOffCtl + 320;
+    static_assert(kSmemBytes <= 232448, "exceeds the 227 KB a CTA may use");
     // tensor-memory columns
     static constexpr uint32_t kSt = 0, kDp = 128, kDv = 256, kDk = 384;
 };
@@ -53,13 +75,13 @@ struct BwdCfg {
 struct BwdControl {
     uint64_t work_full[2], work_empty[2];
     uint64_t kv_full, kv_empty;
-    uint64_t q_full[2], q_empty[2], do_full[2], do_empty[2];
+    uint64_t q_full[3], q_empty[3], do_full, do_empty, stat_full[2], stat_empty[2];
     uint64_t s_full, p_full, dp_full, ds_full, ds_free, dq_full, dq_free, dkv_full, dkv_free;
     WorkItem work[2];
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
-static_assert(sizeof(BwdControl) <= 512, "control block must fit its slot");
+static_assert(sizeof(BwdControl) <= 320, "control block must fit its slot");
 
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
@@ -102,11 +124,15 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sh.work_full[i], 1);
             mbar_init(&sh.work_empty[i], 13);   // 8 compute warps + 4 drain warps + the MMA thread
-            mbar_init(&sh.q_full[i], 2);        // TMA bytes + statistics staged
-            mbar_init(&sh.q_empty[i], 1);
-            mbar_init(&sh.do_full[i], 1);
-            mbar_init(&sh.do_empty[i], 1);
+            mbar_init(&sh.stat_full[i], 1);
+            mbar_init(&sh.stat_empty[i], 8);
         }
+        for (int i = 0; i < Cfg::kQStages; ++i) {
+            mbar_init(&sh.q_full[i], 1);
+            mbar_init(&sh.q_empty[i], 1);
+        }
+        mbar_init(&sh.do_full, 1);
+        mbar_init(&sh.do_empty, 1);
         mbar_init(&sh.kv_full, 1);
         mbar_init(&sh.kv_empty, 1);
         mbar_init(&sh.s_full, 1);
@@ -141,6 +167,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         first_q = CAUSAL ? w.blk : 0;
     };
 
+    if (warp >= 8 && warp < 12) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
     if (warp == 9) {
         // ------------------------------------------------- scheduler, TMA producer, statistics staging
         if (lane == 0) {
@@ -160,7 +188,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 if (item < n_items && !sh.abort_flag) {
                     w = decode_item(p.sched, p.cu_seqlens, item, kTile, p.n_heads, false);
                 } else {
-                    w.tok0 = 0; w.len = -1; w.head = 0; w.blk = 0;
+                    w.tok0 = 0; w.len = -1; w.head = 0; w.blk = 0; w.tile0 = 0;
                 }
                 sh.work[slot] = w;
                 mbar_arrive(&sh.work_full[slot]);
@@ -180,32 +208,40 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             }
             ++n_work;
             for (int i = first_q; i < n_q; ++i, ++g) {
-                const uint32_t stage = g & 1u;
+                const uint32_t stage = g % Cfg::kQStages, fill = g / Cfg::kQStages;
                 const int row = w.tok0 + i * kTile;
-                if (lane == 0) {
-                    if (g >= 2) {
-                        mbar_wait(&sh.q_empty[stage], ((g >> 1) - 1) & 1u, guard);
-                        mbar_wait(&sh.do_empty[stage], ((g >> 1) - 1) & 1u, guard);
-                    }
-                    mbar_expect_tx(&sh.q_full[stage], Cfg::kTileBytes);
-                    bwd_load_tile<D>(smem + Cfg::kOffQ + stage * Cfg::kTileBytes, &tmap_q, &sh.q_full[stage], w.head, row);
-                    mbar_expect_tx(&sh.do_full[stage], Cfg::kTileBytes);
-                    bwd_load_tile<D>(smem + Cfg::kOffDo + stage * Cfg::kTileBytes, &tmap_do, &sh.do_full[stage], w.head, row);
-                }
-                __syncwarp();
-                // per-row statistics of this Q tile: -lse*log2(e) (or +inf past the sequence end,
-                // which zeroes P there) and D
-                float* st = stats + stage * 256;
+                // per-row statistics of this Q tile, fetched before any wait so that their latency
+                // overlaps it: -lse*log2(e) (or -inf past the sequence end, which zeroes P there) and D
                 const size_t base = (size_t)w.head * p.total_tokens + row;
+                float nl[4], dd[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const int r = lane + 32 * e;
                     const bool ok = i * kTile + r < w.len;
-                    st[r] = ok ? -p.lse[base + r] * kLog2e : -INFINITY;
-                    st[128 + r] = ok ? p.dsum[base + r] : 0.f;
+                    nl[e] = ok ? -p.lse[base + r] * kLog2e : -INFINITY;
+                    dd[e] = ok ? p.dsum[base + r] : 0.f;
+                }
+                if (lane == 0) {
+                    if (fill >= 1) mbar_wait(&sh.q_empty[stage], (fill - 1) & 1u, guard);
+                    mbar_expect_tx(&sh.q_full[stage], Cfg::kTileBytes);
+                    bwd_load_tile<D>(smem + Cfg::kOffQ + stage * Cfg::kTileBytes, &tmap_q, &sh.q_full[stage], w.head, row);
+                }
+                // statistics ring (2 slots): slot g&1 is free once the compute warps finished tile g-2
+                if (lane == 0 && g >= 2) mbar_wait(&sh.stat_empty[g & 1u], ((g >> 1) - 1) & 1u, guard);
+                __syncwarp();
+                float* st = stats + (g & 1u) * 256;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    st[lane + 32 * e] = nl[e];
+                    st[128 + lane + 32 * e] = dd[e];
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.q_full[stage]);
+                if (lane == 0) {
+                    mbar_arrive(&sh.stat_full[g & 1u]);
+                    if (g >= 1) mbar_wait(&sh.do_empty, (g - 1) & 1u, guard);
+                    mbar_expect_tx(&sh.do_full, Cfg::kTileBytes);
+                    bwd_load_tile<D>(smem + Cfg::kOffDo, &tmap_do, &sh.do_full, w.head, row);
+                }
             }
         }
     } else if (warp == 8) {
@@ -217,6 +253,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             constexpr uint32_t idesc_nd_kb = make_idesc_bf16(128, D, false, true);   // A K-contig / tmem, B N-contig
             constexpr uint32_t idesc_nd_mm = make_idesc_bf16(128, D, true, true);    // A M-contig, B N-contig
             uint32_t n_work = 0, g = 0;
+            TDECL
             while (true) {
                 const uint32_t slot = n_work & 1u;
                 if (!mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard)) break;
@@ -226,39 +263,39 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 int first_q, n_q;
                 q_range(w, first_q, n_q);
                 const int N = n_q - first_q;
-                mbar_wait(&sh.kv_full, n_work & 1u, guard);
+                TW(0, mbar_wait(&sh.kv_full, n_work & 1u, guard));
                 // S^T and dP^T of the first tile
-                mbar_wait(&sh.q_full[g & 1u], (g >> 1) & 1u, guard);
+                TW(1, mbar_wait(&sh.q_full[g % Cfg::kQStages], (g / Cfg::kQStages) & 1u, guard));
                 tc_fence_after();
-                issue_abt<D>(tmem + Cfg::kSt, k_addr, q_addr0 + (g & 1u) * Cfg::kTileBytes);
+                issue_abt<D>(tmem + Cfg::kSt, k_addr, q_addr0 + (g % Cfg::kQStages) * Cfg::kTileBytes);
                 tc_commit(&sh.s_full);
-                mbar_wait(&sh.do_full[g & 1u], (g >> 1) & 1u, guard);
-                if (g >= 1) mbar_wait(&sh.dq_free, (g - 1) & 1u, guard);
+                TW(2, mbar_wait(&sh.do_full, g & 1u, guard));
+                if (g >= 1) TW(3, mbar_wait(&sh.dq_free, (g - 1) & 1u, guard));
                 tc_fence_after();
-                issue_abt<D>(tmem + Cfg::kDp, v_addr, do_addr0 + (g & 1u) * Cfg::kTileBytes);
+                issue_abt<D>(tmem + Cfg::kDp, v_addr, do_addr0);
                 tc_commit(&sh.dp_full);
                 for (int n = 0; n < N; ++n, ++g) {
-                    const uint32_t stage = g & 1u, nstage = stage ^ 1u;
-                    const uint32_t q_addr = q_addr0 + stage * Cfg::kTileBytes, do_addr = do_addr0 + stage * Cfg::kTileBytes;
+                    const uint32_t stage = g % Cfg::kQStages, nstage = (g + 1) % Cfg::kQStages;
+                    const uint32_t q_addr = q_addr0 + stage * Cfg::kTileBytes, do_addr = do_addr0;
                     const bool has_next = n + 1 < N;
                     // dV += P^T dO
-                    mbar_wait(&sh.p_full, g & 1u, guard);
-                    if (n == 0 && n_work >= 1) mbar_wait(&sh.dkv_free, (n_work - 1) & 1u, guard);
+                    TW(4, mbar_wait(&sh.p_full, g & 1u, guard));
+                    if (n == 0 && n_work >= 1) TW(5, mbar_wait(&sh.dkv_free, (n_work - 1) & 1u, guard));
                     tc_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < kTile / 16; ++ks)
                         tc_mma_ts(tmem + Cfg::kDv, tmem + Cfg::kSt + (ks / 4) * 64 + (ks % 4) * 8,
                                   make_sdesc_sw128(do_addr + ks * 2048, Cfg::kBoxBytes, 1024), idesc_nd_kb, n > 0 || ks > 0);
-                    tc_commit(&sh.do_empty[stage]);
+                    tc_commit(&sh.do_empty);
                     // S^T of the next tile
                     if (has_next) {
-                        mbar_wait(&sh.q_full[nstage], ((g + 1) >> 1) & 1u, guard);
+                        TW(6, mbar_wait(&sh.q_full[nstage], ((g + 1) / Cfg::kQStages) & 1u, guard));
                         tc_fence_after();
                         issue_abt<D>(tmem + Cfg::kSt, k_addr, q_addr0 + nstage * Cfg::kTileBytes);
                         tc_commit(&sh.s_full);
                     }
                     // dQ tile = dS K  (A: dS^T read M-contiguous; B: K with head_dim contiguous)
-                    mbar_wait(&sh.ds_full, g & 1u, guard);
+                    TW(7, mbar_wait(&sh.ds_full, g & 1u, guard));
                     tc_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < kTile / 16; ++ks)
@@ -276,10 +313,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     tc_commit(&sh.ds_free);
                     // dP^T of the next tile (its columns hold dQ until the drain warps have read it)
                     if (has_next) {
-                        mbar_wait(&sh.do_full[nstage], ((g + 1) >> 1) & 1u, guard);
-                        mbar_wait(&sh.dq_free, g & 1u, guard);
+                        TW(2, mbar_wait(&sh.do_full, (g + 1) & 1u, guard));
+                        TW(3, mbar_wait(&sh.dq_free, g & 1u, guard));
                         tc_fence_after();
-                        issue_abt<D>(tmem + Cfg::kDp, v_addr, do_addr0 + nstage * Cfg::kTileBytes);
+                        issue_abt<D>(tmem + Cfg::kDp, v_addr, do_addr0);
                         tc_commit(&sh.dp_full);
                     }
                 }
@@ -287,8 +324,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 tc_commit(&sh.kv_empty);
                 ++n_work;
             }
+            TDUMP(0);
         }
+    }
     } else if (warp < 8) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 152;");
         // ------------------------------------------------- compute: P^T, dS^T, final dK / dV
         const int half = warp >> 2;                                  // which 64 query columns
         const int key_in_tile = (warp & 3) * 32 + lane;              // tensor-memory lane = key
@@ -298,6 +338,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const uint32_t dp_tmem = tmem + lane_base + Cfg::kDp + half * 64;
         uint8_t* ds_row = smem + Cfg::kOffDs + half * 16384;
         uint32_t n_work = 0, g = 0;
+        TDECL
         while (true) {
             const uint32_t slot = n_work & 1u;
             const bool got = mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard);
@@ -316,68 +357,91 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 const float* st = stats + (g & 1u) * 256 + half * 64;
                 const bool diag = CAUSAL && i == w.blk;
                 float pf[64];
-                mbar_wait(&sh.q_full[g & 1u], (g >> 1) & 1u, guard);    // statistics of this tile are staged
-                mbar_wait(&sh.s_full, g & 1u, guard);
+                TW(0, mbar_wait(&sh.stat_full[g & 1u], (g >> 1) & 1u, guard));
+                TW(1, mbar_wait(&sh.s_full, g & 1u, guard));
                 tc_fence_after();
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t sr[16];
-                    tmem_ld_x16(st_tmem + c * 16, sr);
-                    float nl[16];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        *reinterpret_cast<float4*>(&nl[e * 4]) = *reinterpret_cast<const float4*>(st + c * 16 + e * 4);
+#ifdef DCP_TIMING
+                long long _tp = clock64();
+#endif
+                {
+                    // all 64 scores of this thread's key row are requested before the single wait
+                    uint32_t sr[64];
+                    tmem_ld_x32(st_tmem, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+                    tmem_ld_x32(st_tmem + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
                     tmem_wait_ld();
 #pragma unroll
-                    for (int e = 0; e < 16; ++e)
-                        pf[c * 16 + e] = fast_exp2(fmaf(__uint_as_float(sr[e]), p.scale_log2, nl[e]));
-                    if (key_tail || diag) {
-                        const int q_first = i * kTile + half * 64 + c * 16;   // query index of element 0
+                    for (int c = 0; c < 4; ++c) {
+                        float nl[16];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            *reinterpret_cast<float4*>(&nl[e * 4]) = *reinterpret_cast<const float4*>(st + c * 16 + e * 4);
 #pragma unroll
                         for (int e = 0; e < 16; ++e)
-                            if (!key_valid || (diag && key > q_first + e)) pf[c * 16 + e] = 0.f;
+                            pf[c * 16 + e] = fast_exp2(fmaf(__uint_as_float(sr[c * 16 + e]), p.scale_log2, nl[e]));
                     }
-                    uint32_t pk[8];
+                }
+                if (key_tail || diag) {
+                    const int q_first = i * kTile + half * 64;   // query index of element 0
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) pk[e] = pack_bf16x2(pf[c * 16 + 2 * e], pf[c * 16 + 2 * e + 1]);
-                    tmem_st_x8(pt_tmem + c * 8, pk);
+                    for (int e = 0; e < 64; ++e)
+                        if (!key_valid || (diag && key > q_first + e)) pf[e] = 0.f;
+                }
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) pk[e] = pack_bf16x2(pf[c * 32 + 2 * e], pf[c * 32 + 2 * e + 1]);
+                    tmem_st_x16(pt_tmem + c * 16, pk);
                 }
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.p_full);
+#ifdef DCP_TIMING
+                tacc[5] += clock64() - _tp;
+#endif
 
                 // dS^T = P^T o (dP^T - D)
-                mbar_wait(&sh.dp_full, g & 1u, guard);
-                if (g >= 1) mbar_wait(&sh.ds_free, (g - 1) & 1u, guard);
+                TW(2, mbar_wait(&sh.dp_full, g & 1u, guard));
+                if (g >= 1) TW(3, mbar_wait(&sh.ds_free, (g - 1) & 1u, guard));
                 tc_fence_after();
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t dr[16];
-                    tmem_ld_x16(dp_tmem + c * 16, dr);
-                    float dd[16];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        *reinterpret_cast<float4*>(&dd[e * 4]) = *reinterpret_cast<const float4*>(st + 128 + c * 16 + e * 4);
+#ifdef DCP_TIMING
+                _tp = clock64();
+#endif
+                {
+                    uint32_t dr[64];
+                    tmem_ld_x32(dp_tmem, *reinterpret_cast<uint32_t(*)[32]>(&dr[0]));
+                    tmem_ld_x32(dp_tmem + 32, *reinterpret_cast<uint32_t(*)[32]>(&dr[32]));
                     tmem_wait_ld();
-                    uint32_t pk[8];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const float a = pf[c * 16 + 2 * e] * (__uint_as_float(dr[2 * e]) - dd[2 * e]);
-                        const float b = pf[c * 16 + 2 * e + 1] * (__uint_as_float(dr[2 * e + 1]) - dd[2 * e + 1]);
-                        pk[e] = pack_bf16x2(a, b);
+                    for (int c = 0; c < 8; ++c) {
+                        float dd[8];
+                        *reinterpret_cast<float4*>(&dd[0]) = *reinterpret_cast<const float4*>(st + 128 + c * 8);
+                        *reinterpret_cast<float4*>(&dd[4]) = *reinterpret_cast<const float4*>(st + 128 + c * 8 + 4);
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float a = pf[c * 8 + 2 * e] * (__uint_as_float(dr[c * 8 + 2 * e]) - dd[2 * e]);
+                            const float b = pf[c * 8 + 2 * e + 1] * (__uint_as_float(dr[c * 8 + 2 * e + 1]) - dd[2 * e + 1]);
+                            pk[e] = pack_bf16x2(a, b);
+                        }
+                        *reinterpret_cast<uint4*>(ds_row + sw128_offset(key_in_tile, c)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
-                    *reinterpret_cast<uint4*>(ds_row + sw128_offset(key_in_tile, c * 2)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                    *reinterpret_cast<uint4*>(ds_row + sw128_offset(key_in_tile, c * 2 + 1)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
                 }
                 fence_async_smem();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.ds_full);
+                if (lane == 0) {
+                    mbar_arrive(&sh.ds_full);
+                    mbar_arrive(&sh.stat_empty[g & 1u]);
+                }
+#ifdef DCP_TIMING
+                tacc[6] += clock64() - _tp;
+#endif
             }
 
             // item epilogue: dV and dK rows of this key block (each group writes half the columns)
-            mbar_wait(&sh.dkv_full, n_work & 1u, guard);
+            TW(4, mbar_wait(&sh.dkv_full, n_work & 1u, guard));
             tc_fence_after();
             const size_t tok = (size_t)w.tok0 + (size_t)key;
             const size_t out_off = (tok * p.n_heads + w.head) * D + half * (D / 2);
@@ -409,11 +473,14 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             if (lane == 0) mbar_arrive(&sh.dkv_free);
             ++n_work;
         }
+        if (warp == 0 && lane == 0) TDUMP(1);
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 152;");
         // ------------------------------------------------- dQ drain: tensor memory -> fp32 atomics
-        const int q_in_tile = (warp & 3) * 32 + lane;               // warps 10-13 -> lane quarters 2,3,0,1
+        const int q_in_tile = (warp & 3) * 32 + lane;               // warps 12-15 -> lane quarters 0-3
         const uint32_t dq_tmem = tmem + ((uint32_t)((warp & 3) * 32) << 16) + Cfg::kDp;
         uint32_t n_work = 0, g = 0;
+        TDECL
         while (true) {
             const uint32_t slot = n_work & 1u;
             const bool got = mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard);
@@ -426,8 +493,17 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             int first_q, n_q;
             q_range(w, first_q, n_q);
             for (int i = first_q; i < n_q; ++i, ++g) {
-                mbar_wait(&sh.dq_full, g & 1u, guard);
+                TW(0, mbar_wait(&sh.dq_full, g & 1u, guard));
                 tc_fence_after();
+#ifdef DCP_TIMING
+                long long _tp = clock64();
+#endif
+                // accumulator block of (tile, head) is [D/4][128 rows][4]: the 32 rows of a warp are
+                // contiguous for a fixed column group, so each vector atomic covers whole sectors
+                const int qrow = i * kTile + q_in_tile;
+                float* dst = p.dq_acc + (((size_t)w.tile0 + i) * p.n_heads + w.head) * (size_t)(kTile * D) + q_in_tile * 4;
+                // read the whole tile first and release tensor memory at once: dP^T of the next tile waits
+                // on it, while the atomics below may take as long as they like
                 uint32_t acc[D];
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) tmem_ld_x32(dq_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&acc[c * 32]));
@@ -435,16 +511,18 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.dq_free);
-                const int qrow = i * kTile + q_in_tile;
                 if (qrow < w.len) {
-                    float* dst = p.dq_acc + (((size_t)w.tok0 + qrow) * p.n_heads + w.head) * D;
 #pragma unroll
                     for (int c = 0; c < D / 4; ++c)
-                        red_add_v4(dst + c * 4, __uint_as_float(acc[c * 4]), __uint_as_float(acc[c * 4 + 1]),
+                        red_add_v4(dst + c * (kTile * 4), __uint_as_float(acc[c * 4]), __uint_as_float(acc[c * 4 + 1]),
                                    __uint_as_float(acc[c * 4 + 2]), __uint_as_float(acc[c * 4 + 3]));
                 }
+#ifdef DCP_TIMING
+                tacc[1] += clock64() - _tp;
+#endif
             }
         }
+        if (warp == 12 && lane == 0) TDUMP(2);
     }
 
     tc_fence_before();

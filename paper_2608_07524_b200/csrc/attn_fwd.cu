@@ -151,7 +151,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 if (item < n_items && !sh.abort_flag) {
                     w = decode_item(p.sched, p.cu_seqlens, item, kFwdRowsPerItem, p.n_heads, CAUSAL);
                 } else {
-                    w.tok0 = 0; w.len = -1; w.head = 0; w.blk = 0;
+                    w.tok0 = 0; w.len = -1; w.head = 0; w.blk = 0; w.tile0 = 0;
                 }
                 sh.work[slot] = w;
                 mbar_arrive(&sh.work_full[slot]);

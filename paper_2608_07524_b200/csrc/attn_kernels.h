@@ -23,7 +23,7 @@ struct BwdParams {
     const int32_t* cu_seqlens;
     const float* lse;     // [H, T]
     const float* dsum;    // [H, T]   D_i = sum_c dO_ic O_ic
-    float* dq_acc;        // [T, H, d] fp32, zeroed before the main kernel
+    float* dq_acc;        // fp32, tile-blocked: [tile][head][d/4][128 rows][4]; zeroed before the main kernel
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
     SchedView sched;
@@ -40,14 +40,16 @@ cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t rows_
 cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                             int head_dim, bool causal, int n_ctas, cudaStream_t stream);
 
-// D = rowsum(dO * O) and dq_acc = 0.
+// D = rowsum(dO * O) and dq_acc[0 .. dq_acc_elems) = 0.
 cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* dsum, float* dq_acc,
-                           int32_t total_tokens, int32_t n_heads, int32_t head_dim, cudaStream_t stream);
+                           size_t dq_acc_elems, int32_t total_tokens, int32_t n_heads, int32_t head_dim,
+                           cudaStream_t stream);
 
 cudaError_t launch_attn_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
                             const BwdParams& p, int head_dim, bool causal, int n_ctas, cudaStream_t stream);
 
-// dq = bf16(scale * dq_acc)
-cudaError_t launch_bwd_post(const float* dq_acc, __nv_bfloat16* dq, size_t n_elems, float scale, cudaStream_t stream);
+// dq[T, H, d] = bf16(scale * dq_acc), undoing the tile-blocked layout
+cudaError_t launch_bwd_post(const float* dq_acc, __nv_bfloat16* dq, const int32_t* cu_seqlens, const SchedView& sched,
+                            int32_t n_heads, int32_t head_dim, float scale, int n_sms, cudaStream_t stream);
 
 }  // namespace dcp

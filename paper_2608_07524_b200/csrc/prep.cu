@@ -14,7 +14,8 @@ constexpr int kPrepThreads = 1024;
 // length L contributes ceil(L / rows_per_block) * n_heads items.
 __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __restrict__ cu, int32_t n_seqs,
                                                             int32_t rows_per_block, int32_t n_heads,
-                                                            WorkspaceHeader* hdr, int32_t* order, uint32_t* prefix) {
+                                                            WorkspaceHeader* hdr, int32_t* order, uint32_t* prefix,
+                                                            uint32_t* tile_prefix) {
     __shared__ uint32_t chunk_sum[kPrepThreads];
     const int tid = threadIdx.x;
     for (int i = tid; i < n_seqs; i += kPrepThreads) {
@@ -57,22 +58,47 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __res
         prefix[i] = run;
         run += items_of(i);
     }
+    __syncthreads();
+    // tile_prefix[b] = number of 128-row tiles of sequences 0..b-1 (input order): same two-level scan
+    auto tiles_of = [&](int b) -> uint32_t { return (uint32_t)((cu[b + 1] - cu[b] + kTile - 1) / kTile); };
+    local = 0;
+    for (int i = begin; i < end; ++i) local += tiles_of(i);
+    chunk_sum[tid] = local;
+    __syncthreads();
+    if (tid == 0) {
+        uint32_t acc = 0;
+        for (int i = 0; i < kPrepThreads; ++i) {
+            const uint32_t c = chunk_sum[i];
+            chunk_sum[i] = acc;
+            acc += c;
+        }
+        tile_prefix[n_seqs] = acc;
+    }
+    __syncthreads();
+    run = chunk_sum[tid];
+    for (int i = begin; i < end; ++i) {
+        tile_prefix[i] = run;
+        run += tiles_of(i);
+    }
 }
 
 cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t rows_per_block, int32_t n_heads,
                         const SchedView& sched, cudaStream_t stream) {
     prep_kernel<<<1, kPrepThreads, 0, stream>>>(cu_seqlens, n_seqs, rows_per_block, n_heads, sched.hdr,
-                                                const_cast<int32_t*>(sched.order), const_cast<uint32_t*>(sched.prefix));
+                                                const_cast<int32_t*>(sched.order), const_cast<uint32_t*>(sched.prefix),
+                                                const_cast<uint32_t*>(sched.tile_prefix));
     return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------------------------
-// Backward helper 1: D[h][t] = sum_c dO[t][h][c] * O[t][h][c]; dq_acc[t][h][:] = 0.
-// One warp per (token, head) row; HBM-bound: reads 2*d*2 bytes, writes d*4 + 4 bytes per row.
+// Backward helper 1: D[h][t] = sum_c dO[t][h][c] * O[t][h][c], and the fp32 dQ accumulator is zeroed.
+// One warp per (token, head) row; HBM-bound: reads 2*d*2 bytes per row, writes 4 bytes per row
+// plus the accumulator once.
 template <int D>
 __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __restrict__ o,
                                                       const __nv_bfloat16* __restrict__ d_o, float* __restrict__ dsum,
-                                                      float* __restrict__ dq_acc, int32_t total_tokens, int32_t n_heads) {
+                                                      float* __restrict__ dq_acc, size_t dq_acc_vec4,
+                                                      int32_t total_tokens, int32_t n_heads) {
     const int lane = threadIdx.x & 31;
     const size_t n_rows = (size_t)total_tokens * n_heads;
     const size_t warps = (size_t)gridDim.x * (blockDim.x >> 5);
@@ -88,13 +114,11 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
             const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.x));
             const float2 b1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.y));
             acc = a0.x * b0.x + a0.y * b0.y + a1.x * b1.x + a1.y * b1.y;
-            *reinterpret_cast<float4*>(dq_acc + row * D + lane * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
         } else {
             const uint32_t a = *reinterpret_cast<const uint32_t*>(po), b = *reinterpret_cast<const uint32_t*>(pg);
             const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a));
             const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b));
             acc = a0.x * b0.x + a0.y * b0.y;
-            *reinterpret_cast<float2*>(dq_acc + row * D + lane * 2) = make_float2(0.f, 0.f);
         }
 #pragma unroll
         for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
@@ -103,45 +127,76 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
             dsum[h * total_tokens + tok] = acc;
         }
     }
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < dq_acc_vec4; i += stride)
+        reinterpret_cast<float4*>(dq_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
 cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* dsum, float* dq_acc,
-                           int32_t total_tokens, int32_t n_heads, int32_t head_dim, cudaStream_t stream) {
+                           size_t dq_acc_elems, int32_t total_tokens, int32_t n_heads, int32_t head_dim,
+                           cudaStream_t stream) {
     const size_t n_rows = (size_t)total_tokens * n_heads;
     const int blocks = (int)min((size_t)148 * 8, (n_rows + 7) / 8);
     if (blocks == 0) return cudaSuccess;
     if (head_dim == 128)
-        bwd_pre_kernel<128><<<blocks, 256, 0, stream>>>(o, d_o, dsum, dq_acc, total_tokens, n_heads);
+        bwd_pre_kernel<128><<<blocks, 256, 0, stream>>>(o, d_o, dsum, dq_acc, dq_acc_elems / 4, total_tokens, n_heads);
     else
-        bwd_pre_kernel<64><<<blocks, 256, 0, stream>>>(o, d_o, dsum, dq_acc, total_tokens, n_heads);
+        bwd_pre_kernel<64><<<blocks, 256, 0, stream>>>(o, d_o, dsum, dq_acc, dq_acc_elems / 4, total_tokens, n_heads);
     return cudaGetLastError();
 }
 
-// Backward helper 2: dq = bf16(scale * dq_acc).  8 elements per thread.
+// Backward helper 2: dq[T, H, d] = bf16(scale * dq_acc).  dq_acc holds, per (tile, head), a block
+// [d/4][128 rows][4 floats]; a CTA reads one block with coalesced 16-byte loads, transposes it in
+// shared memory as bf16 and writes whole rows.  Rows past the sequence end are skipped.
+template <int D>
 __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict__ dq,
-                                                       size_t n_vec8, float scale) {
-    const size_t stride = (size_t)gridDim.x * blockDim.x;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec8; i += stride) {
-        const float4 a = reinterpret_cast<const float4*>(dq_acc)[2 * i];
-        const float4 b = reinterpret_cast<const float4*>(dq_acc)[2 * i + 1];
-        __nv_bfloat162 r0 = __floats2bfloat162_rn(a.x * scale, a.y * scale);
-        __nv_bfloat162 r1 = __floats2bfloat162_rn(a.z * scale, a.w * scale);
-        __nv_bfloat162 r2 = __floats2bfloat162_rn(b.x * scale, b.y * scale);
-        __nv_bfloat162 r3 = __floats2bfloat162_rn(b.z * scale, b.w * scale);
-        uint4 out;
-        out.x = *reinterpret_cast<uint32_t*>(&r0);
-        out.y = *reinterpret_cast<uint32_t*>(&r1);
-        out.z = *reinterpret_cast<uint32_t*>(&r2);
-        out.w = *reinterpret_cast<uint32_t*>(&r3);
-        reinterpret_cast<uint4*>(dq)[i] = out;
+                                                       const int32_t* __restrict__ cu, const uint32_t* __restrict__ tile_prefix,
+                                                       int32_t n_seqs, int32_t n_heads, float scale) {
+    constexpr int kRowBytes = D * 2 + 16;                    // padded row of bf16
+    __shared__ __align__(16) uint8_t tile[kTile * kRowBytes];
+    const uint32_t n_tiles = tile_prefix[n_seqs];
+    const uint32_t n_blocks = n_tiles * (uint32_t)n_heads;
+    for (uint32_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
+        const uint32_t t = blk / n_heads, h = blk % n_heads;
+        int lo = 0, hi = n_seqs;                              // sequence owning tile t
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (tile_prefix[mid] <= t) lo = mid; else hi = mid;
+        }
+        while (lo + 1 < n_seqs && tile_prefix[lo + 1] <= t) ++lo;   // skip empty sequences
+        const int row0 = (int)(t - tile_prefix[lo]) * kTile;
+        const int len = cu[lo + 1] - cu[lo];
+        const int rows = min(kTile, len - row0);
+        const float4* src = reinterpret_cast<const float4*>(dq_acc + (size_t)blk * (kTile * D));
+        for (int e = threadIdx.x; e < kTile * D / 4; e += blockDim.x) {
+            const int c4 = e / kTile, r = e % kTile;
+            const float4 v = src[e];
+            __nv_bfloat162 lo2 = __floats2bfloat162_rn(v.x * scale, v.y * scale);
+            __nv_bfloat162 hi2 = __floats2bfloat162_rn(v.z * scale, v.w * scale);
+            uint2 pk;
+            pk.x = *reinterpret_cast<uint32_t*>(&lo2);
+            pk.y = *reinterpret_cast<uint32_t*>(&hi2);
+            *reinterpret_cast<uint2*>(tile + r * kRowBytes + c4 * 8) = pk;
+        }
+        __syncthreads();
+        constexpr int kChunks = D * 2 / 16;                  // 16-byte chunks per row
+        for (int e = threadIdx.x; e < rows * kChunks; e += blockDim.x) {
+            const int r = e / kChunks, c = e % kChunks;
+            const uint4 v = *reinterpret_cast<const uint4*>(tile + r * kRowBytes + c * 16);
+            __nv_bfloat16* out = dq + (((size_t)cu[lo] + row0 + r) * n_heads + h) * D;
+            reinterpret_cast<uint4*>(out)[c] = v;
+        }
+        __syncthreads();
     }
 }
 
-cudaError_t launch_bwd_post(const float* dq_acc, __nv_bfloat16* dq, size_t n_elems, float scale, cudaStream_t stream) {
-    const size_t n_vec8 = n_elems / 8;          // head_dim is a multiple of 64
-    if (n_vec8 == 0) return cudaSuccess;
-    const int blocks = (int)min((size_t)148 * 16, (n_vec8 + 255) / 256);
-    bwd_post_kernel<<<blocks, 256, 0, stream>>>(dq_acc, dq, n_vec8, scale);
+cudaError_t launch_bwd_post(const float* dq_acc, __nv_bfloat16* dq, const int32_t* cu_seqlens, const SchedView& sched,
+                            int32_t n_heads, int32_t head_dim, float scale, int n_sms, cudaStream_t stream) {
+    const int blocks = n_sms * 4;
+    if (head_dim == 128)
+        bwd_post_kernel<128><<<blocks, 256, 0, stream>>>(dq_acc, dq, cu_seqlens, sched.tile_prefix, sched.n_seqs, n_heads, scale);
+    else
+        bwd_post_kernel<64><<<blocks, 256, 0, stream>>>(dq_acc, dq, cu_seqlens, sched.tile_prefix, sched.n_seqs, n_heads, scale);
     return cudaGetLastError();
 }
 

@@ -21,18 +21,25 @@ struct WorkspaceHeader {
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
 
-// After the header: int32 order[n_seqs] (sequence ids, longest first, ties by id) and
-// uint32 prefix[n_seqs + 1] (items before the i-th sequence of `order`).
+// After the header: int32 order[n_seqs] (sequence ids, longest first, ties by id),
+// uint32 prefix[n_seqs + 1] (items before the i-th sequence of `order`) and
+// uint32 tile_prefix[n_seqs + 1] (128-row tiles before sequence b, in input order).
 struct SchedView {
     WorkspaceHeader* hdr;
     const int32_t* order;
     const uint32_t* prefix;
+    const uint32_t* tile_prefix;
     int32_t n_seqs;
 };
 
 __host__ __device__ inline size_t sched_bytes(int32_t n_seqs) {
-    size_t b = sizeof(WorkspaceHeader) + sizeof(int32_t) * (size_t)n_seqs + sizeof(uint32_t) * ((size_t)n_seqs + 1);
+    size_t b = sizeof(WorkspaceHeader) + sizeof(int32_t) * (size_t)n_seqs + 2 * sizeof(uint32_t) * ((size_t)n_seqs + 1);
     return (b + 255) & ~(size_t)255;
+}
+
+// Upper bound on the number of 128-row tiles of a packed batch (every sequence may end in a partial tile).
+__host__ __device__ inline size_t max_tiles(int32_t total_tokens, int32_t n_seqs) {
+    return (size_t)total_tokens / kTile + (size_t)n_seqs;
 }
 
 // A decoded work item.  len < 0 marks the end of the list.
@@ -41,6 +48,7 @@ struct WorkItem {
     int32_t len;    // sequence length
     int32_t head;
     int32_t blk;    // row block inside the sequence (256 query rows forward, 128 keys backward)
+    int32_t tile0;  // index of the sequence's first 128-row tile among all tiles of the batch
 };
 
 // Map item index -> (sequence, head, block).  Within a sequence, blocks vary fastest so that CTAs
@@ -58,6 +66,7 @@ __device__ inline WorkItem decode_item(const SchedView& s, const int32_t* cu_seq
     WorkItem w;
     w.tok0 = cu_seqlens[seq];
     w.len = cu_seqlens[seq + 1] - w.tok0;
+    w.tile0 = (int32_t)s.tile_prefix[seq];
     const uint32_t local = item - s.prefix[lo];
     const uint32_t nblk = (uint32_t)(w.len + rows_per_blk - 1) / (uint32_t)rows_per_blk;
     w.head = (int32_t)(local / nblk);
