@@ -30,22 +30,6 @@
 #include "sched.cuh"
 #include "sm100_ptx.cuh"
 
-// Development aid: with -DDCP_TIMING every role of CTA 0..147 accumulates the cycles it spends in
-// each of its waits and phases; dcp_debug_read_timing copies the table out.  Not part of the product build.
-#ifdef DCP_TIMING
-__device__ long long g_bwd_timing[148 * 4 * 16];
-#define TW(i, ...) do { long long _t = clock64(); __VA_ARGS__; tacc[i] += clock64() - _t; } while (0)
-#define TDECL long long tacc[16] = {0}; const long long _t_begin = clock64();
-#define TDUMP(role) do { tacc[15] = clock64() - _t_begin; for (int _i = 0; _i < 16; ++_i) g_bwd_timing[(blockIdx.x * 4 + (role)) * 16 + _i] = tacc[_i]; } while (0)
-extern "C" int dcp_debug_read_timing(long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, g_bwd_timing, sizeof(long long) * 148 * 4 * 16);
-}
-#else
-#define TW(i, ...) __VA_ARGS__
-#define TDECL
-#define TDUMP(role)
-#endif
-
 namespace dcp {
 
 constexpr int kBwdThreads = 512;
@@ -92,17 +76,6 @@ __device__ __forceinline__ void bwd_load_tile(uint8_t* dst, const CUtensorMap* m
 #pragma unroll
     for (int b = 0; b < BwdCfg<D>::kBoxes; ++b)
         tma_load_3d(dst + b * BwdCfg<D>::kBoxBytes, map, bar, b * 64, head, row);
-}
-
-// D[128 x 128] = A B^T with A, B both [128 x D] row-major tiles (contraction over head_dim).
-template <int D>
-__device__ __forceinline__ void issue_abt(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr) {
-    constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, false);
-#pragma unroll
-    for (int ks = 0; ks < D / 16; ++ks) {
-        const uint32_t off = (ks / 4) * BwdCfg<D>::kBoxBytes + (ks % 4) * 32;
-        tc_mma_ss(d_tmem, make_sdesc_sw128(a_addr + off, 16, 1024), make_sdesc_sw128(b_addr + off, 16, 1024), idesc, ks > 0);
-    }
 }
 
 template <int D, bool CAUSAL>
@@ -168,7 +141,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     };
 
     if (warp >= 8 && warp < 12) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 104;");
     if (warp == 9) {
         // ------------------------------------------------- scheduler, TMA producer, statistics staging
         if (lane == 0) {
@@ -210,34 +183,17 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             for (int i = first_q; i < n_q; ++i, ++g) {
                 const uint32_t stage = g % Cfg::kQStages, fill = g / Cfg::kQStages;
                 const int row = w.tok0 + i * kTile;
-                // per-row statistics of this Q tile, fetched before any wait so that their latency
-                // overlaps it: -lse*log2(e) (or -inf past the sequence end, which zeroes P there) and D
-                const size_t base = (size_t)w.head * p.total_tokens + row;
-                float nl[4], dd[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int r = lane + 32 * e;
-                    const bool ok = i * kTile + r < w.len;
-                    nl[e] = ok ? -p.lse[base + r] * kLog2e : -INFINITY;
-                    dd[e] = ok ? p.dsum[base + r] : 0.f;
-                }
                 if (lane == 0) {
                     if (fill >= 1) mbar_wait(&sh.q_empty[stage], (fill - 1) & 1u, guard);
                     mbar_expect_tx(&sh.q_full[stage], Cfg::kTileBytes);
                     bwd_load_tile<D>(smem + Cfg::kOffQ + stage * Cfg::kTileBytes, &tmap_q, &sh.q_full[stage], w.head, row);
-                }
-                // statistics ring (2 slots): slot g&1 is free once the compute warps finished tile g-2
-                if (lane == 0 && g >= 2) mbar_wait(&sh.stat_empty[g & 1u], ((g >> 1) - 1) & 1u, guard);
-                __syncwarp();
-                float* st = stats + (g & 1u) * 256;
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    st[lane + 32 * e] = nl[e];
-                    st[128 + lane + 32 * e] = dd[e];
-                }
-                __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(&sh.stat_full[g & 1u]);
+                    // statistics ring (2 slots): slot g&1 is free once the compute warps finished tile g-2.
+                    // The 1 KB block of this (tile, head) comes by bulk copy, so that it does not queue
+                    // behind the dQ atomics in the load/store unit.
+                    if (g >= 2) mbar_wait(&sh.stat_empty[g & 1u], ((g >> 1) - 1) & 1u, guard);
+                    mbar_expect_tx(&sh.stat_full[g & 1u], 2 * kTile * 4);
+                    tma_load_bulk(stats + (g & 1u) * 256, p.stats + (((size_t)w.tile0 + i) * p.n_heads + w.head) * (2 * kTile),
+                                  2 * kTile * 4, &sh.stat_full[g & 1u]);
                     if (g >= 1) mbar_wait(&sh.do_empty, (g - 1) & 1u, guard);
                     mbar_expect_tx(&sh.do_full, Cfg::kTileBytes);
                     bwd_load_tile<D>(smem + Cfg::kOffDo, &tmap_do, &sh.do_full, w.head, row);
@@ -247,13 +203,31 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     } else if (warp == 8) {
         // ------------------------------------------------- MMA issue
         if (lane == 0) {
-            const uint32_t k_addr = smem_u32(smem + Cfg::kOffK), v_addr = smem_u32(smem + Cfg::kOffV);
-            const uint32_t q_addr0 = smem_u32(smem + Cfg::kOffQ), do_addr0 = smem_u32(smem + Cfg::kOffDo);
-            const uint32_t ds_addr = smem_u32(smem + Cfg::kOffDs);
+            // Shared-memory descriptors are built once; a k-step only adds a constant to the address
+            // field (the issuing thread is on the critical path: MMA issue blocks while the pipe is busy).
+            constexpr uint32_t idesc_abt = make_idesc_bf16(128, 128, false, false);  // both operands K-contiguous
             constexpr uint32_t idesc_nd_kb = make_idesc_bf16(128, D, false, true);   // A K-contig / tmem, B N-contig
             constexpr uint32_t idesc_nd_mm = make_idesc_bf16(128, D, true, true);    // A M-contig, B N-contig
+            constexpr uint32_t kStageStep = Cfg::kTileBytes >> 4;
+            const uint64_t k_km = make_sdesc_sw128(smem_u32(smem + Cfg::kOffK), 16, 1024);
+            const uint64_t k_mn = make_sdesc_sw128(smem_u32(smem + Cfg::kOffK), Cfg::kBoxBytes, 1024);
+            const uint64_t v_km = make_sdesc_sw128(smem_u32(smem + Cfg::kOffV), 16, 1024);
+            const uint64_t q_km0 = make_sdesc_sw128(smem_u32(smem + Cfg::kOffQ), 16, 1024);
+            const uint64_t q_mn0 = make_sdesc_sw128(smem_u32(smem + Cfg::kOffQ), Cfg::kBoxBytes, 1024);
+            const uint64_t do_km = make_sdesc_sw128(smem_u32(smem + Cfg::kOffDo), 16, 1024);
+            const uint64_t do_mn = make_sdesc_sw128(smem_u32(smem + Cfg::kOffDo), Cfg::kBoxBytes, 1024);
+            const uint64_t ds_km = make_sdesc_sw128(smem_u32(smem + Cfg::kOffDs), 16, 1024);
+            const uint64_t ds_mn = make_sdesc_sw128(smem_u32(smem + Cfg::kOffDs), 16384, 1024);
+            // address-field increments (16-byte units) of k-step ks
+            auto km_step = [](int ks, int box_bytes) -> uint64_t { return (uint64_t)(((ks / 4) * box_bytes + (ks % 4) * 32) >> 4); };
+            auto mn_step = [](int ks) -> uint64_t { return (uint64_t)((ks * 2048) >> 4); };
+            // D[128 x 128] = A B^T, both [128 x D] tiles with head_dim contiguous
+            auto issue_abt = [&](uint32_t d_tmem, uint64_t a, uint64_t b) {
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)
+                    tc_mma_ss(d_tmem, a + km_step(ks, Cfg::kBoxBytes), b + km_step(ks, Cfg::kBoxBytes), idesc_abt, ks > 0);
+            };
             uint32_t n_work = 0, g = 0;
-            TDECL
             while (true) {
                 const uint32_t slot = n_work & 1u;
                 if (!mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard)) break;
@@ -263,72 +237,69 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 int first_q, n_q;
                 q_range(w, first_q, n_q);
                 const int N = n_q - first_q;
-                TW(0, mbar_wait(&sh.kv_full, n_work & 1u, guard));
+                mbar_wait(&sh.kv_full, n_work & 1u, guard);
                 // S^T and dP^T of the first tile
-                TW(1, mbar_wait(&sh.q_full[g % Cfg::kQStages], (g / Cfg::kQStages) & 1u, guard));
+                uint32_t stage = g % Cfg::kQStages;
+                mbar_wait(&sh.q_full[stage], (g / Cfg::kQStages) & 1u, guard);
                 tc_fence_after();
-                issue_abt<D>(tmem + Cfg::kSt, k_addr, q_addr0 + (g % Cfg::kQStages) * Cfg::kTileBytes);
+                issue_abt(tmem + Cfg::kSt, k_km, q_km0 + stage * kStageStep);
                 tc_commit(&sh.s_full);
-                TW(2, mbar_wait(&sh.do_full, g & 1u, guard));
-                if (g >= 1) TW(3, mbar_wait(&sh.dq_free, (g - 1) & 1u, guard));
+                mbar_wait(&sh.do_full, g & 1u, guard);
+                if (g >= 1) mbar_wait(&sh.dq_free, (g - 1) & 1u, guard);
                 tc_fence_after();
-                issue_abt<D>(tmem + Cfg::kDp, v_addr, do_addr0);
+                issue_abt(tmem + Cfg::kDp, v_km, do_km);
                 tc_commit(&sh.dp_full);
                 for (int n = 0; n < N; ++n, ++g) {
-                    const uint32_t stage = g % Cfg::kQStages, nstage = (g + 1) % Cfg::kQStages;
-                    const uint32_t q_addr = q_addr0 + stage * Cfg::kTileBytes, do_addr = do_addr0;
+                    const uint32_t nstage = stage + 1 == Cfg::kQStages ? 0 : stage + 1;
                     const bool has_next = n + 1 < N;
                     // dV += P^T dO
-                    TW(4, mbar_wait(&sh.p_full, g & 1u, guard));
-                    if (n == 0 && n_work >= 1) TW(5, mbar_wait(&sh.dkv_free, (n_work - 1) & 1u, guard));
+                    mbar_wait(&sh.p_full, g & 1u, guard);
+                    if (n == 0 && n_work >= 1) mbar_wait(&sh.dkv_free, (n_work - 1) & 1u, guard);
                     tc_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < kTile / 16; ++ks)
-                        tc_mma_ts(tmem + Cfg::kDv, tmem + Cfg::kSt + (ks / 4) * 64 + (ks % 4) * 8,
-                                  make_sdesc_sw128(do_addr + ks * 2048, Cfg::kBoxBytes, 1024), idesc_nd_kb, n > 0 || ks > 0);
+                        tc_mma_ts(tmem + Cfg::kDv, tmem + Cfg::kSt + (ks / 4) * 64 + (ks % 4) * 8, do_mn + mn_step(ks),
+                                  idesc_nd_kb, n > 0 || ks > 0);
                     tc_commit(&sh.do_empty);
                     // S^T of the next tile
                     if (has_next) {
-                        TW(6, mbar_wait(&sh.q_full[nstage], ((g + 1) / Cfg::kQStages) & 1u, guard));
+                        mbar_wait(&sh.q_full[nstage], ((g + 1) / Cfg::kQStages) & 1u, guard);
                         tc_fence_after();
-                        issue_abt<D>(tmem + Cfg::kSt, k_addr, q_addr0 + nstage * Cfg::kTileBytes);
+                        issue_abt(tmem + Cfg::kSt, k_km, q_km0 + nstage * kStageStep);
                         tc_commit(&sh.s_full);
                     }
                     // dQ tile = dS K  (A: dS^T read M-contiguous; B: K with head_dim contiguous)
-                    TW(7, mbar_wait(&sh.ds_full, g & 1u, guard));
+                    mbar_wait(&sh.ds_full, g & 1u, guard);
                     tc_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < kTile / 16; ++ks)
-                        tc_mma_ss(tmem + Cfg::kDp, make_sdesc_sw128(ds_addr + ks * 2048, 16384, 1024),
-                                  make_sdesc_sw128(k_addr + ks * 2048, Cfg::kBoxBytes, 1024), idesc_nd_mm, ks > 0);
+                        tc_mma_ss(tmem + Cfg::kDp, ds_mn + mn_step(ks), k_mn + mn_step(ks), idesc_nd_mm, ks > 0);
                     tc_commit(&sh.dq_full);
                     // dK += dS^T Q
 #pragma unroll
-                    for (int ks = 0; ks < kTile / 16; ++ks) {
-                        const uint32_t offa = (ks / 4) * 16384 + (ks % 4) * 32;
-                        tc_mma_ss(tmem + Cfg::kDk, make_sdesc_sw128(ds_addr + offa, 16, 1024),
-                                  make_sdesc_sw128(q_addr + ks * 2048, Cfg::kBoxBytes, 1024), idesc_nd_kb, n > 0 || ks > 0);
-                    }
+                    for (int ks = 0; ks < kTile / 16; ++ks)
+                        tc_mma_ss(tmem + Cfg::kDk, ds_km + km_step(ks, 16384), q_mn0 + stage * kStageStep + mn_step(ks),
+                                  idesc_nd_kb, n > 0 || ks > 0);
                     tc_commit(&sh.q_empty[stage]);
                     tc_commit(&sh.ds_free);
                     // dP^T of the next tile (its columns hold dQ until the drain warps have read it)
                     if (has_next) {
-                        TW(2, mbar_wait(&sh.do_full, (g + 1) & 1u, guard));
-                        TW(3, mbar_wait(&sh.dq_free, g & 1u, guard));
+                        mbar_wait(&sh.do_full, (g + 1) & 1u, guard);
+                        mbar_wait(&sh.dq_free, g & 1u, guard);
                         tc_fence_after();
-                        issue_abt<D>(tmem + Cfg::kDp, v_addr, do_addr0);
+                        issue_abt(tmem + Cfg::kDp, v_km, do_km);
                         tc_commit(&sh.dp_full);
                     }
+                    stage = nstage;
                 }
                 tc_commit(&sh.dkv_full);
                 tc_commit(&sh.kv_empty);
                 ++n_work;
             }
-            TDUMP(0);
         }
     }
     } else if (warp < 8) {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 152;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 136;");
         // ------------------------------------------------- compute: P^T, dS^T, final dK / dV
         const int half = warp >> 2;                                  // which 64 query columns
         const int key_in_tile = (warp & 3) * 32 + lane;              // tensor-memory lane = key
@@ -338,7 +309,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const uint32_t dp_tmem = tmem + lane_base + Cfg::kDp + half * 64;
         uint8_t* ds_row = smem + Cfg::kOffDs + half * 16384;
         uint32_t n_work = 0, g = 0;
-        TDECL
         while (true) {
             const uint32_t slot = n_work & 1u;
             const bool got = mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard);
@@ -357,12 +327,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 const float* st = stats + (g & 1u) * 256 + half * 64;
                 const bool diag = CAUSAL && i == w.blk;
                 float pf[64];
-                TW(0, mbar_wait(&sh.stat_full[g & 1u], (g >> 1) & 1u, guard));
-                TW(1, mbar_wait(&sh.s_full, g & 1u, guard));
+                mbar_wait(&sh.stat_full[g & 1u], (g >> 1) & 1u, guard);
+                mbar_wait(&sh.s_full, g & 1u, guard);
                 tc_fence_after();
-#ifdef DCP_TIMING
-                long long _tp = clock64();
-#endif
                 {
                     // all 64 scores of this thread's key row are requested before the single wait
                     uint32_t sr[64];
@@ -397,17 +364,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.p_full);
-#ifdef DCP_TIMING
-                tacc[5] += clock64() - _tp;
-#endif
 
                 // dS^T = P^T o (dP^T - D)
-                TW(2, mbar_wait(&sh.dp_full, g & 1u, guard));
-                if (g >= 1) TW(3, mbar_wait(&sh.ds_free, (g - 1) & 1u, guard));
+                mbar_wait(&sh.dp_full, g & 1u, guard);
+                if (g >= 1) mbar_wait(&sh.ds_free, (g - 1) & 1u, guard);
                 tc_fence_after();
-#ifdef DCP_TIMING
-                _tp = clock64();
-#endif
                 {
                     uint32_t dr[64];
                     tmem_ld_x32(dp_tmem, *reinterpret_cast<uint32_t(*)[32]>(&dr[0]));
@@ -435,13 +396,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     mbar_arrive(&sh.ds_full);
                     mbar_arrive(&sh.stat_empty[g & 1u]);
                 }
-#ifdef DCP_TIMING
-                tacc[6] += clock64() - _tp;
-#endif
             }
 
             // item epilogue: dV and dK rows of this key block (each group writes half the columns)
-            TW(4, mbar_wait(&sh.dkv_full, n_work & 1u, guard));
+            mbar_wait(&sh.dkv_full, n_work & 1u, guard);
             tc_fence_after();
             const size_t tok = (size_t)w.tok0 + (size_t)key;
             const size_t out_off = (tok * p.n_heads + w.head) * D + half * (D / 2);
@@ -473,14 +431,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             if (lane == 0) mbar_arrive(&sh.dkv_free);
             ++n_work;
         }
-        if (warp == 0 && lane == 0) TDUMP(1);
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 152;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 136;");
         // ------------------------------------------------- dQ drain: tensor memory -> fp32 atomics
         const int q_in_tile = (warp & 3) * 32 + lane;               // warps 12-15 -> lane quarters 0-3
         const uint32_t dq_tmem = tmem + ((uint32_t)((warp & 3) * 32) << 16) + Cfg::kDp;
         uint32_t n_work = 0, g = 0;
-        TDECL
         while (true) {
             const uint32_t slot = n_work & 1u;
             const bool got = mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard);
@@ -493,11 +449,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             int first_q, n_q;
             q_range(w, first_q, n_q);
             for (int i = first_q; i < n_q; ++i, ++g) {
-                TW(0, mbar_wait(&sh.dq_full, g & 1u, guard));
+                mbar_wait(&sh.dq_full, g & 1u, guard);
                 tc_fence_after();
-#ifdef DCP_TIMING
-                long long _tp = clock64();
-#endif
                 // accumulator block of (tile, head) is [D/4][128 rows][4]: the 32 rows of a warp are
                 // contiguous for a fixed column group, so each vector atomic covers whole sectors
                 const int qrow = i * kTile + q_in_tile;
@@ -517,12 +470,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         red_add_v4(dst + c * (kTile * 4), __uint_as_float(acc[c * 4]), __uint_as_float(acc[c * 4 + 1]),
                                    __uint_as_float(acc[c * 4 + 2]), __uint_as_float(acc[c * 4 + 3]));
                 }
-#ifdef DCP_TIMING
-                tacc[1] += clock64() - _tp;
-#endif
             }
         }
-        if (warp == 12 && lane == 0) TDUMP(2);
     }
 
     tc_fence_before();

@@ -21,8 +21,8 @@ struct FwdParams {
 
 struct BwdParams {
     const int32_t* cu_seqlens;
-    const float* lse;     // [H, T]
-    const float* dsum;    // [H, T]   D_i = sum_c dO_ic O_ic
+    const float* stats;   // per (tile, head): 128 x -lse*log2(e) then 128 x D_i (D_i = sum_c dO_ic O_ic);
+                          // rows past the sequence end hold -inf and 0
     float* dq_acc;        // fp32, tile-blocked: [tile][head][d/4][128 rows][4]; zeroed before the main kernel
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
@@ -40,10 +40,10 @@ cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t rows_
 cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                             int head_dim, bool causal, int n_ctas, cudaStream_t stream);
 
-// D = rowsum(dO * O) and dq_acc[0 .. dq_acc_elems) = 0.
-cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* dsum, float* dq_acc,
-                           size_t dq_acc_elems, int32_t total_tokens, int32_t n_heads, int32_t head_dim,
-                           cudaStream_t stream);
+// Tile-aligned row statistics for the backward kernel (see BwdParams::stats) and dq_acc = 0.
+cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, const float* lse, const int32_t* cu_seqlens,
+                           const SchedView& sched, float* stats, float* dq_acc, size_t dq_acc_elems,
+                           int32_t total_tokens, int32_t n_heads, int32_t head_dim, int n_sms, cudaStream_t stream);
 
 cudaError_t launch_attn_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
                             const BwdParams& p, int head_dim, bool causal, int n_ctas, cudaStream_t stream);

@@ -91,40 +91,59 @@ cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t rows_
 }
 
 // ---------------------------------------------------------------------------------------------
-// Backward helper 1: D[h][t] = sum_c dO[t][h][c] * O[t][h][c], and the fp32 dQ accumulator is zeroed.
-// One warp per (token, head) row; HBM-bound: reads 2*d*2 bytes per row, writes 4 bytes per row
-// plus the accumulator once.
+// Backward helper 1.  For every (128-row tile, head) it writes 256 floats: -lse*log2(e) for the
+// tile's rows, then D_i = sum_c dO_ic O_ic; rows past the sequence end get -inf and 0, which makes
+// their probabilities vanish in the main kernel without any masking there.  The block is 1 KB and
+// 1 KB-aligned, so the main kernel fetches it with one bulk copy.  Also zeroes the fp32 dQ
+// accumulator.  HBM-bound: reads 2*d*2 + 4 bytes per (token, head), writes 8 bytes + the accumulator.
 template <int D>
 __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __restrict__ o,
-                                                      const __nv_bfloat16* __restrict__ d_o, float* __restrict__ dsum,
-                                                      float* __restrict__ dq_acc, size_t dq_acc_vec4,
-                                                      int32_t total_tokens, int32_t n_heads) {
-    const int lane = threadIdx.x & 31;
-    const size_t n_rows = (size_t)total_tokens * n_heads;
-    const size_t warps = (size_t)gridDim.x * (blockDim.x >> 5);
-    for (size_t row = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); row < n_rows; row += warps) {
-        constexpr int kPer = D / 32;           // elements per lane: 2 or 4
-        const __nv_bfloat16* po = o + row * D + lane * kPer;
-        const __nv_bfloat16* pg = d_o + row * D + lane * kPer;
-        float acc = 0.f;
-        if (kPer == 4) {
-            const uint2 a = *reinterpret_cast<const uint2*>(po), b = *reinterpret_cast<const uint2*>(pg);
-            const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.x));
-            const float2 a1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.y));
-            const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.x));
-            const float2 b1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.y));
-            acc = a0.x * b0.x + a0.y * b0.y + a1.x * b1.x + a1.y * b1.y;
-        } else {
-            const uint32_t a = *reinterpret_cast<const uint32_t*>(po), b = *reinterpret_cast<const uint32_t*>(pg);
-            const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a));
-            const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b));
-            acc = a0.x * b0.x + a0.y * b0.y;
+                                                      const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ lse,
+                                                      const int32_t* __restrict__ cu, const uint32_t* __restrict__ tile_prefix,
+                                                      int32_t n_seqs, float* __restrict__ stats, float* __restrict__ dq_acc,
+                                                      size_t dq_acc_vec4, int32_t total_tokens, int32_t n_heads) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t n_blocks = tile_prefix[n_seqs] * (uint32_t)n_heads;
+    for (uint32_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
+        const uint32_t t = blk / n_heads, h = blk % n_heads;
+        int lo = 0, hi = n_seqs;                              // sequence owning tile t
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (tile_prefix[mid] <= t) lo = mid; else hi = mid;
         }
+        while (lo + 1 < n_seqs && tile_prefix[lo + 1] <= t) ++lo;   // skip empty sequences
+        const int row0 = (int)(t - tile_prefix[lo]) * kTile;
+        const int len = cu[lo + 1] - cu[lo];
+        float* out = stats + (size_t)blk * (2 * kTile);
+        for (int r = warp; r < kTile; r += 8) {
+            float acc = 0.f, nl = -INFINITY;
+            if (row0 + r < len) {
+                const size_t tok = (size_t)cu[lo] + row0 + r;
+                const size_t row = tok * n_heads + h;
+                constexpr int kPer = D / 32;           // elements per lane: 2 or 4
+                const __nv_bfloat16* po = o + row * D + lane * kPer;
+                const __nv_bfloat16* pg = d_o + row * D + lane * kPer;
+                if (kPer == 4) {
+                    const uint2 a = *reinterpret_cast<const uint2*>(po), b = *reinterpret_cast<const uint2*>(pg);
+                    const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.x));
+                    const float2 a1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.y));
+                    const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.x));
+                    const float2 b1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.y));
+                    acc = a0.x * b0.x + a0.y * b0.y + a1.x * b1.x + a1.y * b1.y;
+                } else {
+                    const uint32_t a = *reinterpret_cast<const uint32_t*>(po), b = *reinterpret_cast<const uint32_t*>(pg);
+                    const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a));
+                    const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b));
+                    acc = a0.x * b0.x + a0.y * b0.y;
+                }
 #pragma unroll
-        for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-        if (lane == 0) {
-            const size_t tok = row / n_heads, h = row % n_heads;
-            dsum[h * total_tokens + tok] = acc;
+                for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+                nl = -lse[(size_t)h * total_tokens + tok] * 1.4426950408889634f;
+            }
+            if (lane == 0) {
+                out[r] = nl;
+                out[kTile + r] = acc;
+            }
         }
     }
     const size_t stride = (size_t)gridDim.x * blockDim.x;
@@ -132,16 +151,16 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
         reinterpret_cast<float4*>(dq_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
-cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* dsum, float* dq_acc,
-                           size_t dq_acc_elems, int32_t total_tokens, int32_t n_heads, int32_t head_dim,
-                           cudaStream_t stream) {
-    const size_t n_rows = (size_t)total_tokens * n_heads;
-    const int blocks = (int)min((size_t)148 * 8, (n_rows + 7) / 8);
-    if (blocks == 0) return cudaSuccess;
+cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, const float* lse, const int32_t* cu_seqlens,
+                           const SchedView& sched, float* stats, float* dq_acc, size_t dq_acc_elems,
+                           int32_t total_tokens, int32_t n_heads, int32_t head_dim, int n_sms, cudaStream_t stream) {
+    const int blocks = n_sms * 8;
     if (head_dim == 128)
-        bwd_pre_kernel<128><<<blocks, 256, 0, stream>>>(o, d_o, dsum, dq_acc, dq_acc_elems / 4, total_tokens, n_heads);
+        bwd_pre_kernel<128><<<blocks, 256, 0, stream>>>(o, d_o, lse, cu_seqlens, sched.tile_prefix, sched.n_seqs, stats,
+                                                        dq_acc, dq_acc_elems / 4, total_tokens, n_heads);
     else
-        bwd_pre_kernel<64><<<blocks, 256, 0, stream>>>(o, d_o, dsum, dq_acc, dq_acc_elems / 4, total_tokens, n_heads);
+        bwd_pre_kernel<64><<<blocks, 256, 0, stream>>>(o, d_o, lse, cu_seqlens, sched.tile_prefix, sched.n_seqs, stats,
+                                                       dq_acc, dq_acc_elems / 4, total_tokens, n_heads);
     return cudaGetLastError();
 }
 
