@@ -134,7 +134,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     const uint32_t tmem = sh.tmem_base;
 
     if (warp >= 8) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
     if (warp == 9) {
         // ---------------------------------------------------------------- scheduler + TMA producer
         if (lane == 0) {
@@ -254,7 +254,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         }
     }
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
         // ---------------------------------------------------------------- softmax groups
         const int t = warp >> 2;                        // Q tile of this group
         const int row_in_tile = tid & 127;
