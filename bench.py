@@ -26,9 +26,9 @@ sys.path.insert(0, ROOT)
 METRIC = "varlen_attn_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 HBM_BUDGET = 180 * 10 ** 9
-# DRAM traffic of one backward-main launch on the bench workload, from the ncu summary under
-# profiles/ (None until a capture exists for the current kernel).
-BWD_MAIN_DRAM_BYTES_PER_LAUNCH = None
+# DRAM traffic (bytes) of one backward-main launch on config 3, from profiles/attn_fwd_bwd_video_subset.md:
+# 3.169 GB measured by ncu on the 78192-token subset, scaled by tokens (traffic is proportional to them).
+BWD_MAIN_DRAM_BYTES_PER_LAUNCH = {"video": 3.169e9 * 124992 / 78192}
 
 
 def load_peaks():
@@ -286,7 +286,8 @@ def run_ours(args):
     roofline = {"bound": "tensor", "kernel": "attn_bwd_kernel (backward main)", "achieved": achieved,
                 "peak": peaks["sustained"], "unit": UNIT, "frac": (achieved / peaks["sustained"]) if achieved else None,
                 "peak_source": f"bf16_tflops_sustained of {peaks['source']} MEASURED_PEAKS.json",
-                "traffic": BWD_MAIN_DRAM_BYTES_PER_LAUNCH,
+                "traffic": (BWD_MAIN_DRAM_BYTES_PER_LAUNCH.get(args.workload)
+                            if not args.drop_longer_than and args.layers == 1 else None),
                 "launches": bwd_n, "avg_launch_ms": bwd_ms / max(bwd_n, 1)}
 
     cpu_baseline = None

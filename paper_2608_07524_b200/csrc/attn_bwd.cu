@@ -46,8 +46,8 @@ struct BwdCfg {
     static constexpr int kOffV = kTileBytes;
     static constexpr int kQStages = 3;                     // Q is needed early (S^T) and late (dK): three stages
     static constexpr int kOffQ = 2 * kTileBytes;           // so that a load has a whole tile period to land
-    static constexpr int kOffDo = 5 * kTileBytes;          // dO lives only from dP^T to dV: one stage
-    static constexpr int kOffDs = 6 * kTileBytes;
+    static constexpr int kOffDo = (2 + kQStages) * kTileBytes;          // dO lives only from dP^T to dV: one stage
+    static constexpr int kOffDs = (3 + kQStages) * kTileBytes;
     static constexpr int kOffStat = kOffDs + kDsBytes;     // 2 stages x (128 nlse + 128 D) floats
     static constexpr int kOffCtl = kOffStat + 2 * 256 * 4;
     static constexpr int kSmemBytes = kOffCtl + 320;
