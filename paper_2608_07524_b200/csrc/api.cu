@@ -160,7 +160,7 @@ extern "C" int dcp_varlen_attn_workspace(int32_t total_tokens, int32_t n_seqs, i
     const size_t sched = sched_bytes(n_seqs);
     if (fwd_bytes) *fwd_bytes = sched;
     if (bwd_bytes)
-        *bwd_bytes = sched + align256(sizeof(float) * max_tiles(total_tokens, n_seqs) * n_heads * 2 * kTile) +
+        *bwd_bytes = sched + align256(max_tiles(total_tokens, n_seqs) * n_heads * (size_t)(kTile * 16 * 2)) +
                      align256(sizeof(float) * max_tiles(total_tokens, n_seqs) * kTile * n_heads * head_dim);
     return DCP_OK;
 }
@@ -244,8 +244,8 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
 
     const SchedView sched = carve_sched(workspace, n_seqs);
     uint8_t* base = static_cast<uint8_t*>(workspace) + sched_bytes(n_seqs);
-    float* stats = reinterpret_cast<float*>(base);
-    float* dq_acc = reinterpret_cast<float*>(base + align256(sizeof(float) * max_tiles(total_tokens, n_seqs) * n_heads * 2 * kTile));
+    __nv_bfloat16* stats = reinterpret_cast<__nv_bfloat16*>(base);
+    float* dq_acc = reinterpret_cast<float*>(base + align256(max_tiles(total_tokens, n_seqs) * n_heads * (size_t)(kTile * 16 * 2)));
 
     cudaError_t e;
     {
@@ -266,7 +266,8 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
         ScopedTimer t(DCP_KERNEL_BWD_PRE, stream);
         e = launch_bwd_pre(static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, cu_seqlens,
                            sched, stats, dq_acc, max_tiles(total_tokens, n_seqs) * kTile * n_heads * head_dim,
-                           total_tokens, n_heads, head_dim, dev.sm_count, stream);
+                           total_tokens, n_heads, head_dim,
+                           softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim), dev.sm_count, stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: pre kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(1);

@@ -5,11 +5,17 @@
 // transposed orientation, keys on tensor-memory lanes and queries on columns, so that P^T can feed
 // the dV product straight from tensor memory:
 //
-//     S^T  = K Q^T                      (tcgen05, fp32 in tensor memory)
-//     P^T  = exp2(S^T*scale*log2e - lse*log2e), masked            -> bf16, overwrites S^T
-//     dP^T = V dO^T
-//     dS^T = P^T o (dP^T - D)                                      -> bf16, shared memory
+//     S'^T  = K Q^T - 1 (lse/scale)^T   (tcgen05, fp32 in tensor memory)
+//     P^T   = exp2(S'^T * scale*log2e), masked                     -> bf16, overwrites S'^T
+//     dP'^T = V dO^T - 1 D^T
+//     dS^T  = P^T o dP'^T                                          -> bf16, shared memory
 //     dV  += P^T dO          dK += dS^T Q          dQ_tile = dS K  (dQ aliases dP^T's columns)
+//
+// The per-query terms -lse/scale and -D are columns in this orientation; instead of every thread
+// reading them (a shared-memory broadcast costs one wavefront per value, on the port that feeds the
+// MMAs), they are added by one extra K=16 MMA per product: A = a constant tile of ones, B = a
+// [128 queries x 16] bf16 tile holding each term split into three bf16 parts (24 bits, exact sum in
+// the fp32 accumulator), prepared per (tile, head) by the pre kernel and fetched by bulk copy.
 //
 // dQ tiles are added into an fp32 accumulator in global memory with vector atomics because every
 // key block of a sequence contributes to the same query rows.  The accumulator is a workspace, so
@@ -44,12 +50,14 @@ struct BwdCfg {
     // shared-memory map (offsets from a 1024-byte aligned base)
     static constexpr int kOffK = 0;
     static constexpr int kOffV = kTileBytes;
-    static constexpr int kQStages = 3;                     // Q is needed early (S^T) and late (dK): three stages
-    static constexpr int kOffQ = 2 * kTileBytes;           // so that a load has a whole tile period to land
+    static constexpr int kQStages = 2;                     // Q is needed early (S^T) and late (dK)
+    static constexpr int kOffQ = 2 * kTileBytes;
     static constexpr int kOffDo = (2 + kQStages) * kTileBytes;          // dO lives only from dP^T to dV: one stage
     static constexpr int kOffDs = (3 + kQStages) * kTileBytes;
-    static constexpr int kOffStat = kOffDs + kDsBytes;     // 2 stages x (128 nlse + 128 D) floats
-    static constexpr int kOffCtl = kOffStat + 2 * 256 * 4;
+    static constexpr int kStatBytes = kTile * 16 * 2;      // [128 x 16] bf16 tile, K-contiguous, no swizzle
+    static constexpr int kOffOnes = kOffDs + kDsBytes;     // two constant tiles: ones in columns 0-2 / 8-10
+    static constexpr int kOffStat = kOffOnes + 2 * kStatBytes;   // 2 slots of per-query terms
+    static constexpr int kOffCtl = kOffStat + 2 * kStatBytes;
     static constexpr int kSmemBytes = kOffCtl + 320;
     static_assert(kSmemBytes <= 232448, "exceeds the 227 KB a CTA may use");
     // tensor-memory columns
@@ -59,7 +67,7 @@ struct BwdCfg {
 struct BwdControl {
     uint64_t work_full[2], work_empty[2];
     uint64_t kv_full, kv_empty;
-    uint64_t q_full[3], q_empty[3], do_full, do_empty, stat_full[2], stat_empty[2];
+    uint64_t q_full[2], q_empty[2], do_full, do_empty, stat_full[2], stat_empty[2];
     uint64_t s_full, p_full, dp_full, ds_full, ds_free, dq_full, dq_free, dkv_full, dkv_free;
     WorkItem work[2];
     uint32_t tmem_base;
@@ -86,7 +94,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     using Cfg = BwdCfg<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
     BwdControl& sh = *reinterpret_cast<BwdControl*>(smem + Cfg::kOffCtl);
-    float* stats = reinterpret_cast<float*>(smem + Cfg::kOffStat);
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -98,7 +105,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             mbar_init(&sh.work_full[i], 1);
             mbar_init(&sh.work_empty[i], 13);   // 8 compute warps + 4 drain warps + the MMA thread
             mbar_init(&sh.stat_full[i], 1);
-            mbar_init(&sh.stat_empty[i], 8);
+            mbar_init(&sh.stat_empty[i], 1);
         }
         for (int i = 0; i < Cfg::kQStages; ++i) {
             mbar_init(&sh.q_full[i], 1);
@@ -128,6 +135,18 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     if (warp == 0) {
         tmem_alloc(&sh.tmem_base, 512);
         tmem_relinquish();
+    }
+    {   // constant A operands of the rank-1 MMAs: [128 keys x 16] with ones in columns 0-2 (adds the lse
+        // term to S^T) and in columns 8-10 (adds the D term to dP^T).  Layout: 8x8 core matrices of
+        // 128 bytes, row groups 128 bytes apart, the two column halves 2048 bytes apart.
+        uint32_t* ones = reinterpret_cast<uint32_t*>(smem + Cfg::kOffOnes);
+        for (int i = tid; i < 2 * Cfg::kStatBytes / 4; i += kBwdThreads) {
+            const int tile = i / (Cfg::kStatBytes / 4), w32 = i % (Cfg::kStatBytes / 4);
+            const int half = w32 / 512, in_row = w32 % 4;            // 32-bit word inside a 16-byte row chunk
+            const bool on = half == tile;                            // tile 0: first column half, tile 1: second
+            ones[i] = !on ? 0u : in_row == 0 ? 0x3f803f80u : in_row == 1 ? 0x00003f80u : 0u;   // 1,1 | 1,0 | 0..
+        }
+        fence_async_smem();
     }
     tc_fence_before();
     __syncthreads();
@@ -187,13 +206,13 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     if (fill >= 1) mbar_wait(&sh.q_empty[stage], (fill - 1) & 1u, guard);
                     mbar_expect_tx(&sh.q_full[stage], Cfg::kTileBytes);
                     bwd_load_tile<D>(smem + Cfg::kOffQ + stage * Cfg::kTileBytes, &tmap_q, &sh.q_full[stage], w.head, row);
-                    // statistics ring (2 slots): slot g&1 is free once the compute warps finished tile g-2.
-                    // The 1 KB block of this (tile, head) comes by bulk copy, so that it does not queue
-                    // behind the dQ atomics in the load/store unit.
+                    // per-query terms (2 slots): slot g&1 is free once the rank-1 MMAs of tile g-2 are done.
+                    // The 4 KB block of this (tile, head) comes by bulk copy in the layout the MMA reads.
                     if (g >= 2) mbar_wait(&sh.stat_empty[g & 1u], ((g >> 1) - 1) & 1u, guard);
-                    mbar_expect_tx(&sh.stat_full[g & 1u], 2 * kTile * 4);
-                    tma_load_bulk(stats + (g & 1u) * 256, p.stats + (((size_t)w.tile0 + i) * p.n_heads + w.head) * (2 * kTile),
-                                  2 * kTile * 4, &sh.stat_full[g & 1u]);
+                    mbar_expect_tx(&sh.stat_full[g & 1u], Cfg::kStatBytes);
+                    tma_load_bulk(smem + Cfg::kOffStat + (g & 1u) * Cfg::kStatBytes,
+                                  p.stats + (((size_t)w.tile0 + i) * p.n_heads + w.head) * (Cfg::kStatBytes / 2),
+                                  Cfg::kStatBytes, &sh.stat_full[g & 1u]);
                     if (g >= 1) mbar_wait(&sh.do_empty, (g - 1) & 1u, guard);
                     mbar_expect_tx(&sh.do_full, Cfg::kTileBytes);
                     bwd_load_tile<D>(smem + Cfg::kOffDo, &tmap_do, &sh.do_full, w.head, row);
@@ -218,6 +237,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             const uint64_t do_mn = make_sdesc_sw128(smem_u32(smem + Cfg::kOffDo), Cfg::kBoxBytes, 1024);
             const uint64_t ds_km = make_sdesc_sw128(smem_u32(smem + Cfg::kOffDs), 16, 1024);
             const uint64_t ds_mn = make_sdesc_sw128(smem_u32(smem + Cfg::kOffDs), 16384, 1024);
+            const uint64_t ones_s = make_sdesc_nosw(smem_u32(smem + Cfg::kOffOnes), 2048, 128);
+            const uint64_t ones_d = make_sdesc_nosw(smem_u32(smem + Cfg::kOffOnes + Cfg::kStatBytes), 2048, 128);
+            const uint64_t stat0 = make_sdesc_nosw(smem_u32(smem + Cfg::kOffStat), 2048, 128);
+            constexpr uint32_t kStatStep = Cfg::kStatBytes >> 4;
             // address-field increments (16-byte units) of k-step ks
             auto km_step = [](int ks, int box_bytes) -> uint64_t { return (uint64_t)(((ks / 4) * box_bytes + (ks % 4) * 32) >> 4); };
             auto mn_step = [](int ks) -> uint64_t { return (uint64_t)((ks * 2048) >> 4); };
@@ -242,13 +265,17 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 uint32_t stage = g % Cfg::kQStages;
                 mbar_wait(&sh.q_full[stage], (g / Cfg::kQStages) & 1u, guard);
                 tc_fence_after();
+                mbar_wait(&sh.stat_full[g & 1u], (g >> 1) & 1u, guard);
                 issue_abt(tmem + Cfg::kSt, k_km, q_km0 + stage * kStageStep);
+                tc_mma_ss(tmem + Cfg::kSt, ones_s, stat0 + (g & 1u) * kStatStep, idesc_abt, true);
                 tc_commit(&sh.s_full);
                 mbar_wait(&sh.do_full, g & 1u, guard);
                 if (g >= 1) mbar_wait(&sh.dq_free, (g - 1) & 1u, guard);
                 tc_fence_after();
                 issue_abt(tmem + Cfg::kDp, v_km, do_km);
+                tc_mma_ss(tmem + Cfg::kDp, ones_d, stat0 + (g & 1u) * kStatStep, idesc_abt, true);
                 tc_commit(&sh.dp_full);
+                tc_commit(&sh.stat_empty[g & 1u]);
                 for (int n = 0; n < N; ++n, ++g) {
                     const uint32_t nstage = stage + 1 == Cfg::kQStages ? 0 : stage + 1;
                     const bool has_next = n + 1 < N;
@@ -264,8 +291,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     // S^T of the next tile
                     if (has_next) {
                         mbar_wait(&sh.q_full[nstage], ((g + 1) / Cfg::kQStages) & 1u, guard);
+                        mbar_wait(&sh.stat_full[(g + 1) & 1u], ((g + 1) >> 1) & 1u, guard);
                         tc_fence_after();
                         issue_abt(tmem + Cfg::kSt, k_km, q_km0 + nstage * kStageStep);
+                        tc_mma_ss(tmem + Cfg::kSt, ones_s, stat0 + ((g + 1) & 1u) * kStatStep, idesc_abt, true);
                         tc_commit(&sh.s_full);
                     }
                     // dQ tile = dS K  (A: dS^T read M-contiguous; B: K with head_dim contiguous)
@@ -288,7 +317,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         mbar_wait(&sh.dq_free, g & 1u, guard);
                         tc_fence_after();
                         issue_abt(tmem + Cfg::kDp, v_km, do_km);
+                        tc_mma_ss(tmem + Cfg::kDp, ones_d, stat0 + ((g + 1) & 1u) * kStatStep, idesc_abt, true);
                         tc_commit(&sh.dp_full);
+                        tc_commit(&sh.stat_empty[(g + 1) & 1u]);
                     }
                     stage = nstage;
                 }
@@ -324,10 +355,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             const bool key_tail = (w.blk + 1) * kTile > w.len;
 
             for (int i = first_q; i < n_q; ++i, ++g) {
-                const float* st = stats + (g & 1u) * 256 + half * 64;
                 const bool diag = CAUSAL && i == w.blk;
                 float pf[64];
-                mbar_wait(&sh.stat_full[g & 1u], (g >> 1) & 1u, guard);
                 mbar_wait(&sh.s_full, g & 1u, guard);
                 tc_fence_after();
                 {
@@ -337,15 +366,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     tmem_ld_x32(st_tmem + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
                     tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        float nl[16];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            *reinterpret_cast<float4*>(&nl[e * 4]) = *reinterpret_cast<const float4*>(st + c * 16 + e * 4);
-#pragma unroll
-                        for (int e = 0; e < 16; ++e)
-                            pf[c * 16 + e] = fast_exp2(fmaf(__uint_as_float(sr[c * 16 + e]), p.scale_log2, nl[e]));
-                    }
+                    for (int e = 0; e < 64; ++e) pf[e] = fast_exp2(__uint_as_float(sr[e]) * p.scale_log2);
                 }
                 if (key_tail || diag) {
                     const int q_first = i * kTile + half * 64;   // query index of element 0
@@ -376,26 +397,18 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     tmem_wait_ld();
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
-                        float dd[8];
-                        *reinterpret_cast<float4*>(&dd[0]) = *reinterpret_cast<const float4*>(st + 128 + c * 8);
-                        *reinterpret_cast<float4*>(&dd[4]) = *reinterpret_cast<const float4*>(st + 128 + c * 8 + 4);
                         uint32_t pk[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float a = pf[c * 8 + 2 * e] * (__uint_as_float(dr[c * 8 + 2 * e]) - dd[2 * e]);
-                            const float b = pf[c * 8 + 2 * e + 1] * (__uint_as_float(dr[c * 8 + 2 * e + 1]) - dd[2 * e + 1]);
-                            pk[e] = pack_bf16x2(a, b);
-                        }
+                        for (int e = 0; e < 4; ++e)
+                            pk[e] = pack_bf16x2(pf[c * 8 + 2 * e] * __uint_as_float(dr[c * 8 + 2 * e]),
+                                                pf[c * 8 + 2 * e + 1] * __uint_as_float(dr[c * 8 + 2 * e + 1]));
                         *reinterpret_cast<uint4*>(ds_row + sw128_offset(key_in_tile, c)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
                 }
                 fence_async_smem();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(&sh.ds_full);
-                    mbar_arrive(&sh.stat_empty[g & 1u]);
-                }
+                if (lane == 0) mbar_arrive(&sh.ds_full);
             }
 
             // item epilogue: dV and dK rows of this key block (each group writes half the columns)

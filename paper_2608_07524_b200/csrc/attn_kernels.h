@@ -21,8 +21,9 @@ struct FwdParams {
 
 struct BwdParams {
     const int32_t* cu_seqlens;
-    const float* stats;   // per (tile, head): 128 x -lse*log2(e) then 128 x D_i (D_i = sum_c dO_ic O_ic);
-                          // rows past the sequence end hold -inf and 0
+    const __nv_bfloat16* stats;   // per (tile, head) a [128 queries x 16] bf16 tile in the layout the MMA reads:
+                                  // columns 0-2 = -lse/scale split in three bf16 parts, 8-10 = -D likewise
+                                  // (D_i = sum_c dO_ic O_ic); rows past the sequence end hold -1e30 and 0
     float* dq_acc;        // fp32, tile-blocked: [tile][head][d/4][128 rows][4]; zeroed before the main kernel
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
@@ -42,8 +43,9 @@ cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const 
 
 // Tile-aligned row statistics for the backward kernel (see BwdParams::stats) and dq_acc = 0.
 cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, const float* lse, const int32_t* cu_seqlens,
-                           const SchedView& sched, float* stats, float* dq_acc, size_t dq_acc_elems,
-                           int32_t total_tokens, int32_t n_heads, int32_t head_dim, int n_sms, cudaStream_t stream);
+                           const SchedView& sched, __nv_bfloat16* stats, float* dq_acc, size_t dq_acc_elems,
+                           int32_t total_tokens, int32_t n_heads, int32_t head_dim, float scale, int n_sms,
+                           cudaStream_t stream);
 
 cudaError_t launch_attn_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
                             const BwdParams& p, int head_dim, bool causal, int n_ctas, cudaStream_t stream);

@@ -91,17 +91,20 @@ cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t rows_
 }
 
 // ---------------------------------------------------------------------------------------------
-// Backward helper 1.  For every (128-row tile, head) it writes 256 floats: -lse*log2(e) for the
-// tile's rows, then D_i = sum_c dO_ic O_ic; rows past the sequence end get -inf and 0, which makes
-// their probabilities vanish in the main kernel without any masking there.  The block is 1 KB and
-// 1 KB-aligned, so the main kernel fetches it with one bulk copy.  Also zeroes the fp32 dQ
-// accumulator.  HBM-bound: reads 2*d*2 + 4 bytes per (token, head), writes 8 bytes + the accumulator.
+// Backward helper 1.  For every (128-row tile, head) it writes a [128 rows x 16] bf16 tile holding,
+// per query row, -lse/scale (columns 0-2) and -D_i = -sum_c dO_ic O_ic (columns 8-10), each split
+// into three bf16 parts whose sum carries 24 bits; the main kernel adds them to its score and dP
+// accumulators with a K=16 MMA against a tile of ones.  Rows past the sequence end get -1e30 and 0,
+// which makes their probabilities vanish without masking.  The tile is stored in the MMA's shared-
+// memory layout (8x8 core matrices; column halves 2048 bytes apart) and is 4 KB-aligned, so one bulk
+// copy fetches it.  Also zeroes the fp32 dQ accumulator.  HBM-bound.
 template <int D>
 __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __restrict__ o,
                                                       const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ lse,
                                                       const int32_t* __restrict__ cu, const uint32_t* __restrict__ tile_prefix,
-                                                      int32_t n_seqs, float* __restrict__ stats, float* __restrict__ dq_acc,
-                                                      size_t dq_acc_vec4, int32_t total_tokens, int32_t n_heads) {
+                                                      int32_t n_seqs, __nv_bfloat16* __restrict__ stats,
+                                                      float* __restrict__ dq_acc, size_t dq_acc_vec4,
+                                                      int32_t total_tokens, int32_t n_heads, float inv_scale) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t n_blocks = tile_prefix[n_seqs] * (uint32_t)n_heads;
     for (uint32_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
@@ -114,9 +117,9 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
         while (lo + 1 < n_seqs && tile_prefix[lo + 1] <= t) ++lo;   // skip empty sequences
         const int row0 = (int)(t - tile_prefix[lo]) * kTile;
         const int len = cu[lo + 1] - cu[lo];
-        float* out = stats + (size_t)blk * (2 * kTile);
+        uint8_t* out = reinterpret_cast<uint8_t*>(stats) + (size_t)blk * (kTile * 16 * 2);
         for (int r = warp; r < kTile; r += 8) {
-            float acc = 0.f, nl = -INFINITY;
+            float acc = 0.f, nl = -1e30f;
             if (row0 + r < len) {
                 const size_t tok = (size_t)cu[lo] + row0 + r;
                 const size_t row = tok * n_heads + h;
@@ -138,11 +141,20 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
                 }
 #pragma unroll
                 for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-                nl = -lse[(size_t)h * total_tokens + tok] * 1.4426950408889634f;
+                nl = -lse[(size_t)h * total_tokens + tok] * inv_scale;
             }
-            if (lane == 0) {
-                out[r] = nl;
-                out[kTile + r] = acc;
+            if (lane < 2) {     // lane 0: the lse term into column half 0; lane 1: the D term into half 1
+                const float x = lane == 0 ? nl : -acc;
+                const __nv_bfloat16 b0 = __float2bfloat16(x);
+                const float r1 = x - __bfloat162float(b0);
+                const __nv_bfloat16 b1 = __float2bfloat16(r1);
+                const __nv_bfloat16 b2 = __float2bfloat16(r1 - __bfloat162float(b1));
+                uint4 v;
+                v.x = (uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16);
+                v.y = (uint32_t)__bfloat16_as_ushort(b2);
+                v.z = 0u;
+                v.w = 0u;
+                *reinterpret_cast<uint4*>(out + lane * 2048 + (r / 8) * 128 + (r % 8) * 16) = v;
             }
         }
     }
@@ -152,15 +164,16 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
 }
 
 cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, const float* lse, const int32_t* cu_seqlens,
-                           const SchedView& sched, float* stats, float* dq_acc, size_t dq_acc_elems,
-                           int32_t total_tokens, int32_t n_heads, int32_t head_dim, int n_sms, cudaStream_t stream) {
+                           const SchedView& sched, __nv_bfloat16* stats, float* dq_acc, size_t dq_acc_elems,
+                           int32_t total_tokens, int32_t n_heads, int32_t head_dim, float scale, int n_sms,
+                           cudaStream_t stream) {
     const int blocks = n_sms * 8;
     if (head_dim == 128)
         bwd_pre_kernel<128><<<blocks, 256, 0, stream>>>(o, d_o, lse, cu_seqlens, sched.tile_prefix, sched.n_seqs, stats,
-                                                        dq_acc, dq_acc_elems / 4, total_tokens, n_heads);
+                                                        dq_acc, dq_acc_elems / 4, total_tokens, n_heads, 1.0f / scale);
     else
         bwd_pre_kernel<64><<<blocks, 256, 0, stream>>>(o, d_o, lse, cu_seqlens, sched.tile_prefix, sched.n_seqs, stats,
-                                                       dq_acc, dq_acc_elems / 4, total_tokens, n_heads);
+                                                       dq_acc, dq_acc_elems / 4, total_tokens, n_heads, 1.0f / scale);
     return cudaGetLastError();
 }
 

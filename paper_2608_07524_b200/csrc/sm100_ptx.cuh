@@ -149,6 +149,14 @@ __device__ __forceinline__ uint64_t make_sdesc_sw128(uint32_t smem_addr, uint32_
            ((uint64_t)((stride_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
 }
 
+// Same, without swizzle, for a K-contiguous operand made of 8-row x 16-byte core matrices (128
+// contiguous bytes each): leading offset = distance between the two 8-element column halves of a
+// K=16 step, stride offset = distance between 8-row groups.
+__device__ __forceinline__ uint64_t make_sdesc_nosw(uint32_t smem_addr, uint32_t leading_bytes, uint32_t stride_bytes) {
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)((leading_bytes >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((stride_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                           bool accumulate) {
