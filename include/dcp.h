@@ -102,6 +102,27 @@ int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, const void*
                         float softmax_scale, void* dq, void* dk, void* dv, void* workspace,
                         size_t workspace_bytes, void* cuda_stream);
 
+/* Forward attention without a workspace argument (the paper has no counterpart; this exists for
+ * callers that must not allocate device memory - code running inside a memory-pool callback or a
+ * real-time loop, a plug-in handed fixed buffers by its host program, a process whose allocator is
+ * locked down after start-up).  Same operation, arguments, layouts and error codes as
+ * dcp_varlen_attn_fwd, but the work-list scratch is a fixed array inside the library's device
+ * image (about 50 KB, held by every GPU that loads the library until the process exits) instead of
+ * a caller buffer.  Limits and rules:
+ *   - n_seqs <= DCP_NOALLOC_MAX_SEQS, else DCP_ERR_UNSUPPORTED and nothing is enqueued;
+ *   - the call allocates nothing on the device and frees nothing;
+ *   - the first call on each device looks up the array's device address (a synchronous runtime
+ *     query); make that first call before starting any stream capture on that device;
+ *   - all calls on a device share the one array, which keeps the previous call's contents; the
+ *     library re-initialises what it needs at the start of every call, but two calls whose kernels
+ *     may overlap on the GPU (different streams) race on it - serialise them;
+ *   - the device status word of this variant lives in that array and is not readable through
+ *     dcp_query_status; the kernels' waits are bounded all the same. */
+#define DCP_NOALLOC_MAX_SEQS 4096
+int dcp_varlen_attn_fwd_noalloc(const void* q, const void* k, const void* v, const int32_t* cu_seqlens, int32_t n_seqs,
+                                int32_t total_tokens, int32_t max_seqlen, int32_t n_heads, int32_t head_dim,
+                                int32_t causal, float softmax_scale, void* o, float* lse, void* cuda_stream);
+
 /* Synchronises `cuda_stream`, then reads the status word at the start of `workspace`.
  * Returns DCP_OK, DCP_ERR_TIMEOUT (a kernel abandoned a bounded wait; results are invalid) or
  * DCP_ERR_CUDA. */

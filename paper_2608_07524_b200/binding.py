@@ -55,6 +55,8 @@ def lib():
             L.dcp_varlen_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32,
                                               vp, vp, vp, vp, ctypes.c_size_t, vp]
             L.dcp_varlen_attn_bwd.restype = ctypes.c_int
+            L.dcp_varlen_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, vp, vp, vp]
+            L.dcp_varlen_attn_fwd_noalloc.restype = ctypes.c_int
             L.dcp_query_status.argtypes = [vp, vp]
             L.dcp_query_status.restype = ctypes.c_int
             L.dcp_profile_enable.argtypes = [ctypes.c_int]
@@ -155,6 +157,27 @@ def dcp_varlen_attn_fwd(q, k, v, cu_seqlens, max_seqlen: int, causal: bool, soft
                                      int(bool(causal)), float(softmax_scale), _ptr(o), _ptr(lse), _ptr(ws),
                                      ws.numel(), _stream(stream)))
     return o, lse
+
+
+NOALLOC_MAX_SEQS = 4096
+
+
+def dcp_varlen_attn_fwd_noalloc(q, k, v, cu_seqlens, max_seqlen: int, causal: bool, out, lse,
+                                softmax_scale: float = 0.0, stream=None):
+    """Forward attention for callers that cannot allocate device memory: the caller supplies `out`
+    [T,H,d] bf16 and `lse` [H,T] fp32; the work-list scratch is a fixed array inside the library (at
+    most NOALLOC_MAX_SEQS sequences).  This wrapper allocates nothing either.  Calls on one device
+    share that array, so do not let two of them overlap on the GPU."""
+    import torch
+    for name, t in (("q", q), ("k", k), ("v", v), ("out", out)):
+        _require(t, torch.bfloat16, name)
+    _require(lse, torch.float32, "lse")
+    _require(cu_seqlens, torch.int32, "cu_seqlens")
+    T, H, d = q.shape
+    _check(lib().dcp_varlen_attn_fwd_noalloc(_ptr(q), _ptr(k), _ptr(v), _ptr(cu_seqlens), cu_seqlens.numel() - 1, T,
+                                             int(max_seqlen), H, d, int(bool(causal)), float(softmax_scale),
+                                             _ptr(out), _ptr(lse), _stream(stream)))
+    return out, lse
 
 
 def dcp_varlen_attn_bwd(q, k, v, o, d_o, lse, cu_seqlens, max_seqlen: int, causal: bool,

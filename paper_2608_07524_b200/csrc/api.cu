@@ -300,6 +300,54 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
     return DCP_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Forward attention for callers that cannot allocate device memory.
+//
+// The forward kernel needs scratch for its work list (header, sequence order, prefix sums).  Here
+// that scratch is a fixed array in the library's own device image, so the caller passes inputs and
+// outputs only.  Every GPU that loads this library holds the array until the process exits.
+#define DCP_NOALLOC_MAX_SEQS_VALUE 4096
+namespace {
+constexpr size_t kNoAllocScratchBytes =
+    (sizeof(dcp::WorkspaceHeader) + sizeof(int32_t) * DCP_NOALLOC_MAX_SEQS_VALUE +
+     2 * sizeof(uint32_t) * (DCP_NOALLOC_MAX_SEQS_VALUE + 1) + 255) / 256 * 256;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+}  // namespace
+
+extern "C" int dcp_varlen_attn_fwd_noalloc(const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
+                                           int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen, int32_t n_heads,
+                                           int32_t head_dim, int32_t causal, float softmax_scale, void* o, float* lse,
+                                           void* cuda_stream) {
+    const char* fn = "dcp_varlen_attn_fwd_noalloc";
+    if (n_seqs > DCP_NOALLOC_MAX_SEQS_VALUE)
+        return fail(DCP_ERR_UNSUPPORTED, "%s: %d sequences exceed the built-in scratch (at most %d per call)", fn, n_seqs,
+                    DCP_NOALLOC_MAX_SEQS_VALUE);
+    if (n_seqs < 0) return fail(DCP_ERR_INVALID_ARG, "%s: negative n_seqs", fn);
+    // In host code the array's name is only a handle, not a device address: ask the runtime for the
+    // address once per device, with that device current, and hand the kernels that pointer.
+    static std::mutex mu;
+    static void* scratch_of_device[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
+        return fail(DCP_ERR_CUDA, "%s: cudaGetDevice failed or device index out of range", fn);
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!scratch_of_device[dev]) {
+            void* ptr = nullptr;
+            const cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+            if (e != cudaSuccess || !ptr)
+                return fail(DCP_ERR_CUDA, "%s: cudaGetSymbolAddress: %s", fn, cudaGetErrorString(e));
+            scratch_of_device[dev] = ptr;
+        }
+        scratch = scratch_of_device[dev];
+    }
+    if (sched_bytes(n_seqs) > kNoAllocScratchBytes)      // cannot happen for n_seqs <= the maximum; kept as a guard
+        return fail(DCP_ERR_UNSUPPORTED, "%s: built-in scratch too small", fn);
+    return dcp_varlen_attn_fwd(q, k, v, cu_seqlens, n_seqs, total_tokens, max_seqlen, n_heads, head_dim, causal,
+                               softmax_scale, o, lse, scratch, kNoAllocScratchBytes, cuda_stream);
+}
+
 extern "C" int dcp_query_status(const void* workspace, void* cuda_stream) {
     if (!workspace) return fail(DCP_ERR_INVALID_ARG, "dcp_query_status: workspace is null");
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

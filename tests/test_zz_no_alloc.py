@@ -1,0 +1,59 @@
+"""The no-allocation forward entry point gives the same result as the regular one.
+
+Some callers of this library may not allocate device memory at the moment they need attention (a
+memory-pool callback, a real-time loop, a host program that hands a plug-in fixed buffers).  For
+them dcp_varlen_attn_fwd_noalloc keeps its work-list scratch in a fixed array inside the library.
+This file runs last (its name sorts after every other test file) so that a failure here cannot hide
+the results of the other tests; it must also pass when run alone in a fresh process.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_07524_b200 import binding as B
+from paper_2608_07524_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _regular(q, k, v, cu, max_len, causal):
+    ws = B.alloc_workspace(q.shape[0], cu.numel() - 1, q.shape[1], q.shape[2], False, q.device)
+    o, lse = B.dcp_varlen_attn_fwd(q, k, v, cu, max_len, causal, workspace=ws)
+    B.dcp_query_status(ws)
+    return o, lse
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_two_calls_in_a_row_match_the_regular_entry_point(causal):
+    dev = "cuda"
+    # two different batches back to back: the second call finds the first call's work list in the
+    # shared scratch and must not be affected by it
+    batches = [([300, 1000, 129, 128, 1, 513], 3, 128, 31), ([17, 64, 100, 255, 700], 2, 64, 32)]
+    for lengths, H, d, seed in batches:
+        cu_host = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+        q, k, v, _ = (x.to(dev) for x in inputs.make_qkvg(int(cu_host[-1]), H, d, seed))
+        cu = torch.tensor(cu_host, device=dev)
+        ref_o, ref_lse = _regular(q, k, v, cu, max(lengths), causal)
+        out = torch.full_like(q, float("nan"))
+        lse = torch.full((H, q.shape[0]), float("nan"), dtype=torch.float32, device=dev)
+        B.dcp_varlen_attn_fwd_noalloc(q, k, v, cu, max(lengths), causal, out, lse)
+        torch.cuda.synchronize()
+        # same kernels, same inputs: within the tolerance the parity tests use (in fact identical)
+        diff = (out.double() - ref_o.double()).abs()
+        rel = float(torch.linalg.norm(out.double() - ref_o.double()) / torch.linalg.norm(ref_o.double()))
+        assert float(diff.max()) <= 5e-2 and rel <= 1e-2
+        assert float((lse.double() - ref_lse.double()).abs().max()) <= 2e-3
+        assert bool(torch.isfinite(out.float()).all()) and bool(torch.isfinite(lse).all())
+
+
+def test_rejects_more_sequences_than_the_built_in_scratch_holds():
+    dev = "cuda"
+    n = B.NOALLOC_MAX_SEQS + 1
+    q = torch.zeros((n, 1, 64), dtype=torch.bfloat16, device=dev)
+    cu = torch.arange(n + 1, dtype=torch.int32, device=dev)
+    out = torch.zeros_like(q)
+    lse = torch.zeros((1, n), dtype=torch.float32, device=dev)
+    with pytest.raises(B.DcpError) as e:
+        B.dcp_varlen_attn_fwd_noalloc(q, q, q, cu, 1, False, out, lse)
+    assert e.value.code == B.DCP_ERR_UNSUPPORTED
+    assert "4096" in str(e.value)
