@@ -67,6 +67,20 @@ typedef struct {
 int dcp_plan(const int32_t* lengths, int32_t n, int64_t hbm_budget_bytes, const dcp_plan_params* params,
              int32_t* mb_id, int32_t* n_mb, int32_t* recompute, int64_t* cost);
 
+/* DCP-inter: accumulation-step counts that balance n batches running side by side.
+ *
+ * Paper: Section 3.3, Eq. 3, and Appendix C (G_min, G_max).  Batch i takes times[i] (any positive
+ * integer unit: modelled cost, measured microseconds) per accumulation step on its worker group.
+ * Chooses g[i] >= 1 minimising the idle time sum_i (max_j g_j T_j - g_i T_i) subject to
+ * g_i T_i <= G_max * max_j T_j.  Ties: shorter iteration max_j g_j T_j, then the lexicographically
+ * smallest g.  Afterwards, if max_i g_i < G_min, every g_i is multiplied by ceil(G_min / max_i g_i).
+ * On a single GPU this is a planning/simulation aid (the n worker groups are virtual); nothing here
+ * touches the device.  Host pointers; outputs g [n], idle and iteration_time (both nullable, after
+ * the G_min scaling).  Errors: DCP_ERR_INVALID_ARG, DCP_ERR_OVERFLOW, DCP_ERR_UNSUPPORTED (more than
+ * 4e6 candidate iteration times, i.e. times differing by many orders of magnitude). */
+int dcp_inter_plan(const int64_t* times, int32_t n, int32_t g_min, int32_t g_max, int32_t* g, int64_t* idle,
+                   int64_t* iteration_time);
+
 /* ---------------------------------------------------------------------------------------------
  * Attention.
  *

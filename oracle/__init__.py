@@ -16,7 +16,8 @@ import threading
 import numpy as np
 
 _DIR = os.path.dirname(os.path.abspath(__file__))
-_SOURCES = [os.path.join(_DIR, "attn_oracle.c"), os.path.join(_DIR, "plan_oracle.c")]
+_SOURCES = [os.path.join(_DIR, "attn_oracle.c"), os.path.join(_DIR, "plan_oracle.c"),
+            os.path.join(_DIR, "inter_oracle.c")]
 _LIB_PATH = os.path.join(_DIR, "liboracle.so")
 _lock = threading.Lock()
 _lib = None
@@ -60,6 +61,9 @@ def _load():
                                              ci, i32p, f64p, f64p]
             lib.oracle_plan_bruteforce.argtypes = [
                 i32p, ctypes.c_int32, ctypes.c_int64, ctypes.POINTER(PlanParams), i32p, i32p, i32p,
+                ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)]
+            lib.oracle_inter_bruteforce.argtypes = [
+                ctypes.POINTER(ctypes.c_int64), ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, i32p,
                 ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)]
             _lib = lib
     return _lib
@@ -197,3 +201,17 @@ def plan_bruteforce(lengths, budget: int, n_heads=16, head_dim=128, elt_bytes=2,
         raise ValueError(f"oracle_plan_bruteforce rejected its arguments ({rc})")
     K = n_mb.value
     return mb[:n].tolist(), rec[:K].tolist(), (hi.value << 64) | lo.value
+
+
+def inter_bruteforce(times, g_min: int = 1, g_max: int = 4):
+    """Best accumulation-step vector by enumeration of every vector within the G_max bound.
+    Returns (g list[n], idle int).  Raises ValueError when the search space exceeds 5e7 vectors."""
+    t = np.ascontiguousarray(times, dtype=np.int64)
+    n = int(t.size)
+    g = np.zeros(max(n, 1), np.int32)
+    lo, hi = ctypes.c_uint64(0), ctypes.c_uint64(0)
+    rc = _load().oracle_inter_bruteforce(_p(t, ctypes.c_int64), n, int(g_min), int(g_max), _p(g, ctypes.c_int32),
+                                         ctypes.byref(lo), ctypes.byref(hi))
+    if rc:
+        raise ValueError(f"oracle_inter_bruteforce rejected its arguments or the space is too large ({rc})")
+    return g[:n].tolist(), (hi.value << 64) | lo.value

@@ -47,6 +47,9 @@ def lib():
             L.dcp_plan.argtypes = [i32p, i32, i64, ctypes.POINTER(PlanParams), i32p, i32p, i32p,
                                    ctypes.POINTER(ctypes.c_int64)]
             L.dcp_plan.restype = ctypes.c_int
+            i64p = ctypes.POINTER(ctypes.c_int64)
+            L.dcp_inter_plan.argtypes = [i64p, i32, i32, i32, i32p, i64p, i64p]
+            L.dcp_inter_plan.restype = ctypes.c_int
             L.dcp_varlen_attn_workspace.argtypes = [i32, i32, i32, i32, szp, szp]
             L.dcp_varlen_attn_workspace.restype = ctypes.c_int
             L.dcp_varlen_attn_fwd.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, vp, vp, vp,
@@ -109,6 +112,16 @@ def dcp_plan(lengths, hbm_budget_bytes: int, n_heads: int = 16, head_dim: int = 
     _check(lib().dcp_plan(arr, n, int(hbm_budget_bytes), ctypes.byref(params), mb, ctypes.byref(n_mb), rec,
                           ctypes.byref(cost)))
     return list(mb[:n]), list(rec[:n_mb.value]), int(cost.value)
+
+
+def dcp_inter_plan(times, g_min: int = 1, g_max: int = 4) -> Tuple[List[int], int, int]:
+    """(g [n], idle, iteration_time): accumulation steps balancing n side-by-side batches (Eq. 3)."""
+    n = len(times)
+    arr = (ctypes.c_int64 * max(n, 1))(*[int(x) for x in times])
+    g = (ctypes.c_int32 * max(n, 1))()
+    idle, it = ctypes.c_int64(0), ctypes.c_int64(0)
+    _check(lib().dcp_inter_plan(arr, n, int(g_min), int(g_max), g, ctypes.byref(idle), ctypes.byref(it)))
+    return list(g[:n]), int(idle.value), int(it.value)
 
 
 def dcp_varlen_attn_workspace(total_tokens: int, n_seqs: int, n_heads: int, head_dim: int) -> Tuple[int, int]:
