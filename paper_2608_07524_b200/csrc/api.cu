@@ -192,7 +192,7 @@ extern "C" int dcp_varlen_attn_fwd(const void* q, const void* k, const void* v, 
         e = launch_prep(cu_seqlens, n_seqs, kFwdRowsPerItem, n_heads, sched, stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: work-list kernel: %s", fn, cudaGetErrorString(e));
-    g_launches.fetch_add(1);
+    g_launches.fetch_add(prep_launches(n_seqs));
     if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
 
     CUtensorMap tq, tk, tv;
@@ -253,7 +253,7 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
         e = launch_prep(cu_seqlens, n_seqs, kTile, n_heads, sched, stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: work-list kernel: %s", fn, cudaGetErrorString(e));
-    g_launches.fetch_add(1);
+    g_launches.fetch_add(prep_launches(n_seqs));
     if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
 
     CUtensorMap tq, tk, tv, tg;

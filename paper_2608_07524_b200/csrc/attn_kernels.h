@@ -35,6 +35,7 @@ struct BwdParams {
 };
 
 // Builds the work list (longest sequence first) and resets the work counter and status word.
+int prep_launches(int32_t n_seqs);   // kernels launch_prep enqueues for a batch of n_seqs sequences (1 or 2)
 cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t rows_per_block, int32_t n_heads,
                         const SchedView& sched, cudaStream_t stream);
 

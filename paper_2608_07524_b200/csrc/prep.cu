@@ -9,23 +9,47 @@ namespace dcp {
 
 constexpr int kPrepThreads = 1024;
 
-// One CTA.  order[] = sequence ids sorted by (length descending, id ascending) via a rank sort;
-// prefix[i] = number of work items of the first i sequences in that order, where a sequence of
-// length L contributes ceil(L / rows_per_block) * n_heads items.
+// Rank sort, one thread per sequence over as many CTAs as needed: order[] = sequence ids sorted by
+// (length descending, id ascending).  Used on its own for batches of more than kPrepThreads
+// sequences; small batches do the same loop inside prep_kernel and save the launch.
+__global__ void __launch_bounds__(256) rank_kernel(const int32_t* __restrict__ cu, int32_t n_seqs, int32_t* order) {
+    __shared__ int32_t len_tile[256];
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    const int32_t len_i = i < n_seqs ? cu[i + 1] - cu[i] : 0;
+    int rank = 0;
+    for (int j0 = 0; j0 < n_seqs; j0 += 256) {
+        const int j = j0 + threadIdx.x;
+        __syncthreads();
+        len_tile[threadIdx.x] = j < n_seqs ? cu[j + 1] - cu[j] : -1;     // -1 never outranks anything
+        __syncthreads();
+        const int cnt = min(256, n_seqs - j0);
+        for (int t = 0; t < cnt; ++t) {
+            const int32_t len_j = len_tile[t];
+            rank += (len_j > len_i) || (len_j == len_i && j0 + t < i);
+        }
+    }
+    if (i < n_seqs) order[rank] = i;
+}
+
+// One CTA.  order[] as above (computed here unless `ranked`); prefix[i] = number of work items of the
+// first i sequences in that order, where a sequence of length L contributes
+// ceil(L / rows_per_block) * n_heads items; tile_prefix[b] = 128-row tiles before sequence b.
 __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __restrict__ cu, int32_t n_seqs,
                                                             int32_t rows_per_block, int32_t n_heads,
                                                             WorkspaceHeader* hdr, int32_t* order, uint32_t* prefix,
-                                                            uint32_t* tile_prefix) {
+                                                            uint32_t* tile_prefix, int ranked) {
     __shared__ uint32_t chunk_sum[kPrepThreads];
     const int tid = threadIdx.x;
-    for (int i = tid; i < n_seqs; i += kPrepThreads) {
-        const int32_t len_i = cu[i + 1] - cu[i];
-        int rank = 0;
-        for (int j = 0; j < n_seqs; ++j) {
-            const int32_t len_j = cu[j + 1] - cu[j];
-            rank += (len_j > len_i) || (len_j == len_i && j < i);
+    if (!ranked) {
+        for (int i = tid; i < n_seqs; i += kPrepThreads) {
+            const int32_t len_i = cu[i + 1] - cu[i];
+            int rank = 0;
+            for (int j = 0; j < n_seqs; ++j) {
+                const int32_t len_j = cu[j + 1] - cu[j];
+                rank += (len_j > len_i) || (len_j == len_i && j < i);
+            }
+            order[rank] = i;
         }
-        order[rank] = i;
     }
     __syncthreads();
     // exclusive scan of item counts over the sorted order: contiguous chunk per thread
@@ -82,11 +106,18 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __res
     }
 }
 
+int prep_launches(int32_t n_seqs) { return n_seqs > kPrepThreads ? 2 : 1; }
+
 cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t rows_per_block, int32_t n_heads,
                         const SchedView& sched, cudaStream_t stream) {
+    const int ranked = n_seqs > kPrepThreads;
+    if (ranked) {
+        rank_kernel<<<(n_seqs + 255) / 256, 256, 0, stream>>>(cu_seqlens, n_seqs, const_cast<int32_t*>(sched.order));
+        if (cudaError_t e = cudaGetLastError()) return e;
+    }
     prep_kernel<<<1, kPrepThreads, 0, stream>>>(cu_seqlens, n_seqs, rows_per_block, n_heads, sched.hdr,
                                                 const_cast<int32_t*>(sched.order), const_cast<uint32_t*>(sched.prefix),
-                                                const_cast<uint32_t*>(sched.tile_prefix));
+                                                const_cast<uint32_t*>(sched.tile_prefix), ranked);
     return cudaGetLastError();
 }
 
@@ -106,45 +137,63 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
                                                       float* __restrict__ dq_acc, size_t dq_acc_vec4,
                                                       int32_t total_tokens, int32_t n_heads, float inv_scale) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t n_blocks = tile_prefix[n_seqs] * (uint32_t)n_heads;
-    for (uint32_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
-        const uint32_t t = blk / n_heads, h = blk % n_heads;
-        int lo = 0, hi = n_seqs;                              // sequence owning tile t
-        while (hi - lo > 1) {
+    const uint32_t n_tiles = tile_prefix[n_seqs];
+    for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        int lo = 0, hi = n_seqs;                              // sequence owning tile t (one search per tile,
+        while (hi - lo > 1) {                                 // shared by all heads)
             const int mid = (lo + hi) >> 1;
             if (tile_prefix[mid] <= t) lo = mid; else hi = mid;
         }
         while (lo + 1 < n_seqs && tile_prefix[lo + 1] <= t) ++lo;   // skip empty sequences
         const int row0 = (int)(t - tile_prefix[lo]) * kTile;
         const int len = cu[lo + 1] - cu[lo];
-        uint8_t* out = reinterpret_cast<uint8_t*>(stats) + (size_t)blk * (kTile * 16 * 2);
-        for (int r = warp; r < kTile; r += 8) {
-            float acc = 0.f, nl = -1e30f;
-            if (row0 + r < len) {
-                const size_t tok = (size_t)cu[lo] + row0 + r;
-                const size_t row = tok * n_heads + h;
-                constexpr int kPer = D / 32;           // elements per lane: 2 or 4
-                const __nv_bfloat16* po = o + row * D + lane * kPer;
-                const __nv_bfloat16* pg = d_o + row * D + lane * kPer;
-                if (kPer == 4) {
-                    const uint2 a = *reinterpret_cast<const uint2*>(po), b = *reinterpret_cast<const uint2*>(pg);
-                    const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.x));
-                    const float2 a1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.y));
-                    const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.x));
-                    const float2 b1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.y));
-                    acc = a0.x * b0.x + a0.y * b0.y + a1.x * b1.x + a1.y * b1.y;
-                } else {
-                    const uint32_t a = *reinterpret_cast<const uint32_t*>(po), b = *reinterpret_cast<const uint32_t*>(pg);
-                    const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a));
-                    const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b));
-                    acc = a0.x * b0.x + a0.y * b0.y;
-                }
+        for (uint32_t h = 0; h < (uint32_t)n_heads; ++h) {
+        uint8_t* out = reinterpret_cast<uint8_t*>(stats) + ((size_t)t * n_heads + h) * (kTile * 16 * 2);
+        // a warp takes rows warp, warp+8, ...; four rows per pass so that eight loads are in flight per lane
+        constexpr int kPer = D / 32;           // elements per lane: 2 or 4
+        for (int r0 = warp; r0 < kTile; r0 += 32) {
+            float acc[4], nl[4];
+            uint2 a[4], b[4];
 #pragma unroll
-                for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-                nl = -lse[(size_t)h * total_tokens + tok] * inv_scale;
+            for (int u = 0; u < 4; ++u) {
+                const int r = r0 + 8 * u;
+                a[u] = make_uint2(0u, 0u);
+                b[u] = make_uint2(0u, 0u);
+                nl[u] = -1e30f;
+                if (row0 + r < len) {
+                    const size_t tok = (size_t)cu[lo] + row0 + r;
+                    const size_t row = tok * n_heads + h;
+                    if (kPer == 4) {
+                        a[u] = *reinterpret_cast<const uint2*>(o + row * D + lane * 4);
+                        b[u] = *reinterpret_cast<const uint2*>(d_o + row * D + lane * 4);
+                    } else {
+                        a[u].x = *reinterpret_cast<const uint32_t*>(o + row * D + lane * 2);
+                        b[u].x = *reinterpret_cast<const uint32_t*>(d_o + row * D + lane * 2);
+                    }
+                    if (lane == 0) nl[u] = -lse[(size_t)h * total_tokens + tok] * inv_scale;
+                }
             }
-            if (lane < 2) {     // lane 0: the lse term into column half 0; lane 1: the D term into half 1
-                const float x = lane == 0 ? nl : -acc;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a[u].x));
+                const float2 a1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a[u].y));
+                const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b[u].x));
+                const float2 b1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b[u].y));
+                acc[u] = a0.x * b0.x + a0.y * b0.y + a1.x * b1.x + a1.y * b1.y;     // unused halves are zero
+#pragma unroll
+                for (int sft = 16; sft > 0; sft >>= 1) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], sft);
+            }
+            // lane 0 holds the lse terms; lanes 0..3 write the lse chunk of row u, lanes 4..7 its D chunk
+            const int u = lane & 3;
+            float nl_b[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) nl_b[t] = __shfl_sync(0xffffffffu, nl[t], 0);
+            const float nl_u = u == 0 ? nl_b[0] : u == 1 ? nl_b[1] : u == 2 ? nl_b[2] : nl_b[3];
+            if (lane < 8) {
+                const int r = r0 + 8 * u;
+                const float acc_u = u == 0 ? acc[0] : u == 1 ? acc[1] : u == 2 ? acc[2] : acc[3];
+                const int which = lane >> 2;                      // 0: lse term -> column half 0, 1: D term -> half 1
+                const float x = which == 0 ? nl_u : -acc_u;
                 const __nv_bfloat16 b0 = __float2bfloat16(x);
                 const float r1 = x - __bfloat162float(b0);
                 const __nv_bfloat16 b1 = __float2bfloat16(r1);
@@ -154,8 +203,9 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
                 v.y = (uint32_t)__bfloat16_as_ushort(b2);
                 v.z = 0u;
                 v.w = 0u;
-                *reinterpret_cast<uint4*>(out + lane * 2048 + (r / 8) * 128 + (r % 8) * 16) = v;
+                *reinterpret_cast<uint4*>(out + which * 2048 + (r / 8) * 128 + (r % 8) * 16) = v;
             }
+        }
         }
     }
     const size_t stride = (size_t)gridDim.x * blockDim.x;
@@ -187,9 +237,7 @@ __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__
     constexpr int kRowBytes = D * 2 + 16;                    // padded row of bf16
     __shared__ __align__(16) uint8_t tile[kTile * kRowBytes];
     const uint32_t n_tiles = tile_prefix[n_seqs];
-    const uint32_t n_blocks = n_tiles * (uint32_t)n_heads;
-    for (uint32_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
-        const uint32_t t = blk / n_heads, h = blk % n_heads;
+    for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
         int lo = 0, hi = n_seqs;                              // sequence owning tile t
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
@@ -199,7 +247,8 @@ __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__
         const int row0 = (int)(t - tile_prefix[lo]) * kTile;
         const int len = cu[lo + 1] - cu[lo];
         const int rows = min(kTile, len - row0);
-        const float4* src = reinterpret_cast<const float4*>(dq_acc + (size_t)blk * (kTile * D));
+        for (uint32_t h = 0; h < (uint32_t)n_heads; ++h) {
+        const float4* src = reinterpret_cast<const float4*>(dq_acc + ((size_t)t * n_heads + h) * (kTile * D));
         for (int e = threadIdx.x; e < kTile * D / 4; e += blockDim.x) {
             const int c4 = e / kTile, r = e % kTile;
             const float4 v = src[e];
@@ -219,6 +268,7 @@ __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__
             reinterpret_cast<uint4*>(out)[c] = v;
         }
         __syncthreads();
+        }
     }
 }
 

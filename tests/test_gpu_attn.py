@@ -94,6 +94,12 @@ def test_many_short_sequences(causal):
     check_full([int(x) for x in rng.integers(1, 200, size=300)], 2, 64, causal, seed=5)
 
 
+def test_more_sequences_than_one_sorting_block():
+    # above 1024 sequences the work list is ranked by a separate multi-CTA kernel
+    rng = np.random.default_rng(6)
+    check_full([int(x) for x in rng.integers(0, 60, size=1500)], 1, 64, True, seed=6)
+
+
 @pytest.mark.parametrize("causal", [False, True])
 def test_backward_in_isolation(causal):
     """Backward fed with the oracle's own O (rounded to bf16) and lse (fp32) instead of the GPU
