@@ -25,6 +25,21 @@
 #include "sched.cuh"
 #include "sm100_ptx.cuh"
 
+// Development aid (-DDCP_TIMING, not part of the product build): cycles spent in waits and phases.
+#ifdef DCP_TIMING
+__device__ long long g_fwd_timing[148 * 3 * 8];
+#define FTW(i, ...) do { long long _t = clock64(); __VA_ARGS__; tacc[i] += clock64() - _t; } while (0)
+#define FTDECL long long tacc[8] = {0}; const long long _t_begin = clock64();
+#define FTDUMP(role) do { tacc[7] = clock64() - _t_begin; for (int _i = 0; _i < 8; ++_i) g_fwd_timing[(blockIdx.x * 3 + (role)) * 8 + _i] = tacc[_i]; } while (0)
+extern "C" int dcp_debug_read_timing_fwd(long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, g_fwd_timing, sizeof(long long) * 148 * 3 * 8);
+}
+#else
+#define FTW(i, ...) __VA_ARGS__
+#define FTDECL
+#define FTDUMP(role)
+#endif
+
 namespace dcp {
 
 constexpr int kFwdThreads = 384;   // 8 softmax warps + a 4-warp control group (MMA, producer, 2 idle)
@@ -68,26 +83,30 @@ __device__ __forceinline__ void load_tile(uint8_t* dst, const CUtensorMap* map, 
         tma_load_3d(dst + b * FwdCfg<D>::kBoxBytes, map, bar, b * 64, head, row);
 }
 
+// The MMA warp runs its loop with all 32 lanes in lock step and only `leader` issues: every operand
+// below is then warp-uniform, the descriptors are built once outside the loops, and a k-step costs
+// one add per operand.  (tcgen05.mma issue blocks while the pipe is busy, and a lone thread executes
+// dependent instructions several cycles apart, so each instruction between two MMAs is pipe idle time.)
+
 // S = Q K^T for one 128x128 tile: both operands K-contiguous in shared memory.
 template <int D>
-__device__ __forceinline__ void issue_qk(uint32_t d_tmem, uint32_t q_addr, uint32_t k_addr) {
+__device__ __forceinline__ void issue_qk(uint32_t d_tmem, uint64_t q_desc, uint64_t k_desc, bool leader) {
     constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, false);
 #pragma unroll
     for (int ks = 0; ks < D / 16; ++ks) {
-        const uint32_t off = (ks / 4) * FwdCfg<D>::kBoxBytes + (ks % 4) * 32;
-        tc_mma_ss(d_tmem, make_sdesc_sw128(q_addr + off, 16, 1024), make_sdesc_sw128(k_addr + off, 16, 1024), idesc,
-                  ks > 0);
+        constexpr int kBox = FwdCfg<D>::kBoxBytes;
+        const uint64_t off = (uint64_t)(((ks / 4) * kBox + (ks % 4) * 32) >> 4);
+        if (leader) tc_mma_ss(d_tmem, q_desc + off, k_desc + off, idesc, ks > 0);
     }
 }
 
 // O (+)= P V: P from tensor memory (bf16 pairs per column), V with head_dim contiguous.
 template <int D>
-__device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint32_t v_addr, bool accumulate) {
+__device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint64_t v_desc, bool accumulate, bool leader) {
     constexpr uint32_t idesc = make_idesc_bf16(128, D, false, true);
 #pragma unroll
     for (int ks = 0; ks < kTile / 16; ++ks)
-        tc_mma_ts(d_tmem, p_tmem + ks * 8, make_sdesc_sw128(v_addr + ks * 2048, FwdCfg<D>::kBoxBytes, 1024), idesc,
-                  accumulate || ks > 0);
+        if (leader) tc_mma_ts(d_tmem, p_tmem + ks * 8, v_desc + (uint64_t)((ks * 2048) >> 4), idesc, accumulate || ks > 0);
 }
 
 template <int D, bool CAUSAL>
@@ -102,7 +121,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     __shared__ FwdShared sh;
 
     const int tid = threadIdx.x;
-    const int warp = tid >> 5;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);     // via a shuffle: provably uniform within the warp
     const int lane = tid & 31;
     const WaitGuard guard{&sh.abort_flag, &p.sched.hdr->status};
 
@@ -182,21 +201,28 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         }
     } else if (warp == 8) {
         // ---------------------------------------------------------------- MMA issue
-        if (lane == 0) {
+        {
+            const bool leader = elect_one();
             uint32_t n_work = 0, kv_base = 0, use[2] = {0, 0}, n_p[2] = {0, 0};
-            const uint32_t q_addr[2] = {smem_u32(sQ), smem_u32(sQ) + Cfg::kTileBytes};
-            const uint32_t kv_addr = smem_u32(sKV);
+            FTDECL
+            const uint64_t q_desc[2] = {make_sdesc_sw128(smem_u32(sQ), 16, 1024),
+                                        make_sdesc_sw128(smem_u32(sQ) + Cfg::kTileBytes, 16, 1024)};
+            const uint64_t kv_km0 = make_sdesc_sw128(smem_u32(sKV), 16, 1024);                 // K: head_dim contiguous
+            const uint64_t kv_mn0 = make_sdesc_sw128(smem_u32(sKV), Cfg::kBoxBytes, 1024);     // V: head_dim contiguous = N
+            constexpr uint32_t kStageStep = Cfg::kTileBytes >> 4;
             const uint32_t s_tmem[2] = {tmem + Cfg::kS0, tmem + Cfg::kS1};
             const uint32_t o_tmem[2] = {tmem + Cfg::kO0, tmem + Cfg::kO1};
             auto kv_wait = [&](uint32_t idx) {
-                mbar_wait(&sh.kv_full[idx % kKvStages], (idx / kKvStages) & 1u, guard);
+                FTW(0, mbar_wait(&sh.kv_full[idx % kKvStages], (idx / kKvStages) & 1u, guard));
             };
-            auto kv_smem = [&](uint32_t idx) { return kv_addr + (idx % kKvStages) * Cfg::kTileBytes; };
+            auto commit = [&](uint64_t* bar) { if (leader) tc_commit(bar); };
             while (true) {
                 const uint32_t slot = n_work & 1u;
-                if (!mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard)) break;
+                const bool got = mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard);
+                if (!__all_sync(0xffffffffu, got)) break;
                 const WorkItem w = sh.work[slot];
-                mbar_arrive(&sh.work_empty[slot]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.work_empty[slot]);
                 ++n_work;
                 if (w.len < 0) break;
                 const int r0 = w.blk * kFwdRowsPerItem;
@@ -210,13 +236,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     if (nkv_t[t] == 0) continue;
                     mbar_wait(&sh.q_full[t], use[t] & 1u, guard);
                     tc_fence_after();
-                    issue_qk<D>(s_tmem[t], q_addr[t], kv_smem(kv_base));
-                    tc_commit(&sh.s_full[t]);
+                    issue_qk<D>(s_tmem[t], q_desc[t], kv_km0 + (kv_base % kKvStages) * kStageStep, leader);
+                    commit(&sh.s_full[t]);
                 }
-                tc_commit(&sh.kv_empty[kv_base % kKvStages]);
+                commit(&sh.kv_empty[kv_base % kKvStages]);
 
                 for (int j = 0; j < nkv; ++j) {
                     const uint32_t iv = kv_base + 2 * j + 1, ik = kv_base + 2 * j + 2;
+                    const uint32_t st_v = iv % kKvStages, st_k = ik % kKvStages;
                     const bool has_next = j + 1 < nkv;
                     kv_wait(iv);
 #pragma unroll
@@ -224,33 +251,34 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         if (t == 1 && has_next) kv_wait(ik);
                         if (t == 1 && j + 1 < nkv_t[0]) {      // S_0(j+1) goes between the two PV products
                             tc_fence_after();
-                            issue_qk<D>(s_tmem[0], q_addr[0], kv_smem(ik));
-                            tc_commit(&sh.s_full[0]);
+                            issue_qk<D>(s_tmem[0], q_desc[0], kv_km0 + st_k * kStageStep, leader);
+                            commit(&sh.s_full[0]);
                         }
                         if (j < nkv_t[t]) {
-                            mbar_wait(&sh.p_full[t], n_p[t] & 1u, guard);
+                            FTW(1 + t, mbar_wait(&sh.p_full[t], n_p[t] & 1u, guard));
                             ++n_p[t];
                             if (j == 0 && use[t] >= 1) mbar_wait(&sh.o_free[t], (use[t] - 1) & 1u, guard);
                             tc_fence_after();
-                            issue_pv<D>(o_tmem[t], s_tmem[t], kv_smem(iv), j > 0);
-                            if (j == nkv_t[t] - 1) tc_commit(&sh.o_full[t]);
+                            issue_pv<D>(o_tmem[t], s_tmem[t], kv_mn0 + st_v * kStageStep, j > 0, leader);
+                            if (j == nkv_t[t] - 1) commit(&sh.o_full[t]);
                         }
                     }
-                    tc_commit(&sh.kv_empty[iv % kKvStages]);
+                    commit(&sh.kv_empty[st_v]);
                     if (j + 1 < nkv_t[1]) {
-                        issue_qk<D>(s_tmem[1], q_addr[1], kv_smem(ik));
-                        tc_commit(&sh.s_full[1]);
+                        issue_qk<D>(s_tmem[1], q_desc[1], kv_km0 + st_k * kStageStep, leader);
+                        commit(&sh.s_full[1]);
                     }
-                    if (has_next) tc_commit(&sh.kv_empty[ik % kKvStages]);
+                    if (has_next) commit(&sh.kv_empty[st_k]);
                 }
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     if (nkv_t[t] == 0) continue;
-                    tc_commit(&sh.q_empty[t]);
+                    commit(&sh.q_empty[t]);
                     ++use[t];
                 }
                 kv_base += 2 * nkv;
             }
+            if (lane == 0) FTDUMP(0);
         }
     }
     } else {
@@ -262,6 +290,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const uint32_t s_tmem = tmem + lane_base + (t == 0 ? Cfg::kS0 : Cfg::kS1);
         const uint32_t o_tmem = tmem + lane_base + (t == 0 ? Cfg::kO0 : Cfg::kO1);
         uint32_t n_work = 0, n_s = 0, use = 0;
+        FTDECL
         while (true) {
             const uint32_t slot = n_work & 1u;
             const bool got = mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard);
@@ -278,8 +307,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 
             float m = -INFINITY, l = 0.f;
             for (int j = 0; j < nkv; ++j) {
-                mbar_wait(&sh.s_full[t], n_s & 1u, guard);
+                FTW(0, mbar_wait(&sh.s_full[t], n_s & 1u, guard));
                 ++n_s;
+#ifdef DCP_TIMING
+                const long long _tp = clock64();
+#endif
                 tc_fence_after();
                 uint32_t s[128];
 #pragma unroll
@@ -339,6 +371,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.p_full[t]);
+#ifdef DCP_TIMING
+                tacc[1] += clock64() - _tp;
+#endif
             }
 
             // epilogue: O = acc / l, lse = m*scale + ln l
@@ -371,6 +406,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.o_free[t]);
         }
+        if ((warp == 0 || warp == 4) && lane == 0) FTDUMP(1 + t);
     }
 
     tc_fence_before();
