@@ -112,7 +112,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     BwdControl& sh = *reinterpret_cast<BwdControl*>(smem + Cfg::kOffCtl);
 
     const int tid = threadIdx.x;
-    const int warp = tid >> 5;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);     // via a shuffle: provably uniform within the warp
     const int lane = tid & 31;
     const WaitGuard guard{&sh.abort_flag, &p.sched.hdr->status};
 
@@ -237,7 +237,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         }
     } else if (warp == 8) {
         // ------------------------------------------------- MMA issue
-        if (lane == 0) {
+        // All 32 lanes run the loop in lock step and only `leader` issues, so that every operand is
+        // warp-uniform and an MMA costs a couple of adds: each instruction between two MMAs is pipe idle time.
+        {
+            const bool leader = elect_one();
             // Shared-memory descriptors are built once; a k-step only adds a constant to the address
             // field (the issuing thread is on the critical path: MMA issue blocks while the pipe is busy).
             constexpr uint32_t idesc_abt = make_idesc_bf16(128, 128, false, false);  // both operands K-contiguous
@@ -264,15 +267,17 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             auto issue_abt = [&](uint32_t d_tmem, uint64_t a, uint64_t b) {
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks)
-                    tc_mma_ss(d_tmem, a + km_step(ks, Cfg::kBoxBytes), b + km_step(ks, Cfg::kBoxBytes), idesc_abt, ks > 0);
+                    if (leader) tc_mma_ss(d_tmem, a + km_step(ks, Cfg::kBoxBytes), b + km_step(ks, Cfg::kBoxBytes), idesc_abt, ks > 0);
             };
             uint32_t n_work = 0, g = 0;
             TDECL
             while (true) {
                 const uint32_t slot = n_work & 1u;
-                if (!mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard)) break;
+                const bool got = mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard);
+                if (!__all_sync(0xffffffffu, got)) break;
                 const WorkItem w = sh.work[slot];
-                mbar_arrive(&sh.work_empty[slot]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.work_empty[slot]);
                 if (w.len < 0) break;
                 int first_q, n_q;
                 q_range(w, first_q, n_q);
@@ -284,15 +289,15 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 tc_fence_after();
                 mbar_wait(&sh.stat_full[g & 1u], (g >> 1) & 1u, guard);
                 issue_abt(tmem + Cfg::kSt, k_km, q_km0 + stage * kStageStep);
-                tc_mma_ss(tmem + Cfg::kSt, ones_s, stat0 + (g & 1u) * kStatStep, idesc_abt, true);
-                tc_commit(&sh.s_full);
+                if (leader) tc_mma_ss(tmem + Cfg::kSt, ones_s, stat0 + (g & 1u) * kStatStep, idesc_abt, true);
+                if (leader) tc_commit(&sh.s_full);
                 mbar_wait(&sh.do_full, g & 1u, guard);
                 if (g >= 1) mbar_wait(&sh.dq_free, (g - 1) & 1u, guard);
                 tc_fence_after();
                 issue_abt(tmem + Cfg::kDp, v_km, do_km);
-                tc_mma_ss(tmem + Cfg::kDp, ones_d, stat0 + (g & 1u) * kStatStep, idesc_abt, true);
-                tc_commit(&sh.dp_full);
-                tc_commit(&sh.stat_empty[g & 1u]);
+                if (leader) tc_mma_ss(tmem + Cfg::kDp, ones_d, stat0 + (g & 1u) * kStatStep, idesc_abt, true);
+                if (leader) tc_commit(&sh.dp_full);
+                if (leader) tc_commit(&sh.stat_empty[g & 1u]);
                 for (int n = 0; n < N; ++n, ++g) {
                     const uint32_t nstage = stage + 1 == Cfg::kQStages ? 0 : stage + 1;
                     const bool has_next = n + 1 < N;
@@ -303,17 +308,17 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     TW(6,
 #pragma unroll
                     for (int ks = 0; ks < kTile / 16; ++ks)
-                        tc_mma_ts(tmem + Cfg::kDv, tmem + Cfg::kSt + (ks / 4) * 64 + (ks % 4) * 8, do_mn + mn_step(ks),
+                        if (leader) tc_mma_ts(tmem + Cfg::kDv, tmem + Cfg::kSt + (ks / 4) * 64 + (ks % 4) * 8, do_mn + mn_step(ks),
                                   idesc_nd_kb, n > 0 || ks > 0);
-                    tc_commit(&sh.do_empty));
+                    if (leader) tc_commit(&sh.do_empty));
                     // S^T of the next tile
                     if (has_next) {
                         TW(2, mbar_wait(&sh.q_full[nstage], ((g + 1) / Cfg::kQStages) & 1u, guard);
                         mbar_wait(&sh.stat_full[(g + 1) & 1u], ((g + 1) >> 1) & 1u, guard));
                         tc_fence_after();
                         TW(7, issue_abt(tmem + Cfg::kSt, k_km, q_km0 + nstage * kStageStep);
-                        tc_mma_ss(tmem + Cfg::kSt, ones_s, stat0 + ((g + 1) & 1u) * kStatStep, idesc_abt, true);
-                        tc_commit(&sh.s_full));
+                        if (leader) tc_mma_ss(tmem + Cfg::kSt, ones_s, stat0 + ((g + 1) & 1u) * kStatStep, idesc_abt, true);
+                        if (leader) tc_commit(&sh.s_full));
                     }
                     // dQ tile = dS K  (A: dS^T read M-contiguous; B: K with head_dim contiguous)
                     TW(3, mbar_wait(&sh.ds_full, g & 1u, guard));
@@ -321,33 +326,33 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     TW(8,
 #pragma unroll
                     for (int ks = 0; ks < kTile / 16; ++ks)
-                        tc_mma_ss(tmem + Cfg::kDp, ds_mn + mn_step(ks), k_mn + mn_step(ks), idesc_nd_mm, ks > 0);
-                    tc_commit(&sh.dq_full));
+                        if (leader) tc_mma_ss(tmem + Cfg::kDp, ds_mn + mn_step(ks), k_mn + mn_step(ks), idesc_nd_mm, ks > 0);
+                    if (leader) tc_commit(&sh.dq_full));
                     // dK += dS^T Q
                     TW(9,
 #pragma unroll
                     for (int ks = 0; ks < kTile / 16; ++ks)
-                        tc_mma_ss(tmem + Cfg::kDk, ds_km + km_step(ks, 16384), q_mn0 + stage * kStageStep + mn_step(ks),
+                        if (leader) tc_mma_ss(tmem + Cfg::kDk, ds_km + km_step(ks, 16384), q_mn0 + stage * kStageStep + mn_step(ks),
                                   idesc_nd_kb, n > 0 || ks > 0);
-                    tc_commit(&sh.q_empty[stage]);
-                    tc_commit(&sh.ds_free));
+                    if (leader) tc_commit(&sh.q_empty[stage]);
+                    if (leader) tc_commit(&sh.ds_free));
                     // dP^T of the next tile (its columns hold dQ until the drain warps have read it)
                     if (has_next) {
                         TW(4, mbar_wait(&sh.do_full, (g + 1) & 1u, guard));
                         TW(5, mbar_wait(&sh.dq_free, g & 1u, guard));
                         tc_fence_after();
                         TW(10, issue_abt(tmem + Cfg::kDp, v_km, do_km);
-                        tc_mma_ss(tmem + Cfg::kDp, ones_d, stat0 + ((g + 1) & 1u) * kStatStep, idesc_abt, true);
-                        tc_commit(&sh.dp_full);
-                        tc_commit(&sh.stat_empty[(g + 1) & 1u]));
+                        if (leader) tc_mma_ss(tmem + Cfg::kDp, ones_d, stat0 + ((g + 1) & 1u) * kStatStep, idesc_abt, true);
+                        if (leader) tc_commit(&sh.dp_full);
+                        if (leader) tc_commit(&sh.stat_empty[(g + 1) & 1u]));
                     }
                     stage = nstage;
                 }
-                tc_commit(&sh.dkv_full);
-                tc_commit(&sh.kv_empty);
+                if (leader) tc_commit(&sh.dkv_full);
+                if (leader) tc_commit(&sh.kv_empty);
                 ++n_work;
             }
-            TDUMP(0);
+            if (lane == 0) TDUMP(0);
         }
     }
     } else if (warp < 8) {
