@@ -137,17 +137,18 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
                                                       float* __restrict__ dq_acc, size_t dq_acc_vec4,
                                                       int32_t total_tokens, int32_t n_heads, float inv_scale) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t n_tiles = tile_prefix[n_seqs];
-    for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-        int lo = 0, hi = n_seqs;                              // sequence owning tile t (one search per tile,
-        while (hi - lo > 1) {                                 // shared by all heads)
+    const uint32_t n_blocks = tile_prefix[n_seqs] * (uint32_t)n_heads;
+    for (uint32_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
+        const uint32_t t = blk / n_heads, h = blk % n_heads;
+        int lo = 0, hi = n_seqs;                              // sequence owning tile t
+        while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
             if (tile_prefix[mid] <= t) lo = mid; else hi = mid;
         }
         while (lo + 1 < n_seqs && tile_prefix[lo + 1] <= t) ++lo;   // skip empty sequences
         const int row0 = (int)(t - tile_prefix[lo]) * kTile;
         const int len = cu[lo + 1] - cu[lo];
-        for (uint32_t h = 0; h < (uint32_t)n_heads; ++h) {
+        {
         uint8_t* out = reinterpret_cast<uint8_t*>(stats) + ((size_t)t * n_heads + h) * (kTile * 16 * 2);
         // a warp takes rows warp, warp+8, ...; four rows per pass so that eight loads are in flight per lane
         constexpr int kPer = D / 32;           // elements per lane: 2 or 4
@@ -236,8 +237,9 @@ __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__
                                                        int32_t n_seqs, int32_t n_heads, float scale) {
     constexpr int kRowBytes = D * 2 + 16;                    // padded row of bf16
     __shared__ __align__(16) uint8_t tile[kTile * kRowBytes];
-    const uint32_t n_tiles = tile_prefix[n_seqs];
-    for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+    const uint32_t n_blocks = tile_prefix[n_seqs] * (uint32_t)n_heads;
+    for (uint32_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
+        const uint32_t t = blk / n_heads, h = blk % n_heads;
         int lo = 0, hi = n_seqs;                              // sequence owning tile t
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
@@ -247,7 +249,7 @@ __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__
         const int row0 = (int)(t - tile_prefix[lo]) * kTile;
         const int len = cu[lo + 1] - cu[lo];
         const int rows = min(kTile, len - row0);
-        for (uint32_t h = 0; h < (uint32_t)n_heads; ++h) {
+        {
         const float4* src = reinterpret_cast<const float4*>(dq_acc + ((size_t)t * n_heads + h) * (kTile * D));
         for (int e = threadIdx.x; e < kTile * D / 4; e += blockDim.x) {
             const int c4 = e / kTile, r = e % kTile;
