@@ -49,7 +49,7 @@ constexpr float kRescaleThreshold = 8.0f;   // in log2 units
 struct FwdShared {
     uint64_t q_full[2], q_empty[2];
     uint64_t kv_full[kKvStages], kv_empty[kKvStages];
-    uint64_t s_full[2], p_half[2], p_full[2], o_full[2], o_free[2];
+    uint64_t s_full[2], p_part[2][4], o_full[2], o_free[2];
     uint64_t work_full[2], work_empty[2];
     WorkItem work[2];
     uint32_t tmem_base;
@@ -101,15 +101,15 @@ __device__ __forceinline__ void issue_qk(uint32_t d_tmem, uint64_t q_desc, uint6
 }
 
 // O (+)= P V: P from tensor memory (bf16 pairs per column), V with head_dim contiguous.
-// `half` selects keys 0-63 or 64-127: the product starts on the first half of P while the softmax
-// group is still producing the second, which shortens the chain S -> softmax -> PV -> next S.
+// `part` selects 32 of the tile's 128 keys: the product starts on the first part of P while the softmax
+// group is still producing the rest, which shortens the chain S -> softmax -> PV -> next S.
 template <int D>
 __device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint64_t v_desc, bool accumulate, bool leader,
-                                         int half) {
+                                         int part) {
     constexpr uint32_t idesc = make_idesc_bf16(128, D, false, true);
 #pragma unroll
-    for (int k4 = 0; k4 < kTile / 32; ++k4) {
-        const int ks = half * (kTile / 32) + k4;
+    for (int k4 = 0; k4 < 2; ++k4) {
+        const int ks = part * 2 + k4;
         if (leader) tc_mma_ts(d_tmem, p_tmem + ks * 8, v_desc + (uint64_t)((ks * 2048) >> 4), idesc, accumulate || ks > 0);
     }
 }
@@ -135,8 +135,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             mbar_init(&sh.q_full[i], 1);
             mbar_init(&sh.q_empty[i], 1);
             mbar_init(&sh.s_full[i], 1);
-            mbar_init(&sh.p_half[i], 4);       // one arrival per softmax warp: keys 0-63 of P written
-            mbar_init(&sh.p_full[i], 4);       // ... all 128 keys written
+            for (int k = 0; k < 4; ++k) mbar_init(&sh.p_part[i][k], 4);   // one arrival per softmax warp per 32 keys of P
             mbar_init(&sh.o_full[i], 1);
             mbar_init(&sh.o_free[i], 4);
             mbar_init(&sh.work_full[i], 1);
@@ -261,14 +260,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                             commit(&sh.s_full[0]);
                         }
                         if (j < nkv_t[t]) {
-                            FTW(1 + t, mbar_wait(&sh.p_half[t], n_p[t] & 1u, guard));
                             if (j == 0 && use[t] >= 1) mbar_wait(&sh.o_free[t], (use[t] - 1) & 1u, guard);
-                            tc_fence_after();
-                            issue_pv<D>(o_tmem[t], s_tmem[t], kv_mn0 + st_v * kStageStep, j > 0, leader, 0);
-                            FTW(1 + t, mbar_wait(&sh.p_full[t], n_p[t] & 1u, guard));
+#pragma unroll
+                            for (int part = 0; part < 4; ++part) {
+                                FTW(1 + t, mbar_wait(&sh.p_part[t][part], n_p[t] & 1u, guard));
+                                tc_fence_after();
+                                issue_pv<D>(o_tmem[t], s_tmem[t], kv_mn0 + st_v * kStageStep, j > 0, leader, part);
+                            }
                             ++n_p[t];
-                            tc_fence_after();
-                            issue_pv<D>(o_tmem[t], s_tmem[t], kv_mn0 + st_v * kStageStep, j > 0, leader, 1);
                             if (j == nkv_t[t] - 1) commit(&sh.o_full[t]);
                         }
                     }
@@ -374,18 +373,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         pk[i] = pack_bf16x2(p0, p1);
                     }
                     tmem_st_x16(s_tmem + c * 16, pk);
-                    if (c == 1) {       // keys 0-63 of P are in tensor memory: the PV product may start
-                        tmem_wait_st();
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&sh.p_half[t]);
-                    }
+                    // these 32 keys of P are in tensor memory: the PV product may use them
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sh.p_part[t][c]);
                 }
                 l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
-                tmem_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.p_full[t]);
 #ifdef DCP_TIMING
                 tacc[1] += clock64() - _tp;
 #endif
