@@ -27,8 +27,8 @@ METRIC = "varlen_attn_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 HBM_BUDGET = 180 * 10 ** 9
 # DRAM traffic (bytes) of one backward-main launch on config 3, from profiles/attn_fwd_bwd_video_subset.md:
-# 3.169 GB measured by ncu on the 78192-token subset, scaled by tokens (traffic is proportional to them).
-BWD_MAIN_DRAM_BYTES_PER_LAUNCH = {"video": 3.169e9 * 124992 / 78192}
+# 3.201 GB measured by ncu on the 78192-token subset, scaled by tokens (traffic is proportional to them).
+BWD_MAIN_DRAM_BYTES_PER_LAUNCH = {"video": 3.201e9 * 124992 / 78192}
 
 
 def load_peaks():
