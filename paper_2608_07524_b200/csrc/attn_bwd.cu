@@ -84,7 +84,7 @@ struct BwdControl {
     uint64_t work_full[2], work_empty[2];
     uint64_t kv_full, kv_empty;
     uint64_t q_full[2], q_empty[2], do_full, do_empty, stat_full[2], stat_empty[2];
-    uint64_t s_full, p_full, dp_full, ds_full, ds_free, dq_full, dq_free, dkv_full, dkv_free;
+    uint64_t s_full, p_half, p_full, dp_full, ds_full, ds_free, dq_full, dq_free, dkv_full, dkv_free;
     WorkItem work[2];
     uint32_t tmem_base;
     uint32_t abort_flag;
@@ -132,6 +132,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         mbar_init(&sh.kv_full, 1);
         mbar_init(&sh.kv_empty, 1);
         mbar_init(&sh.s_full, 1);
+        mbar_init(&sh.p_half, 8);     // first 32 query columns of each group's P^T written
         mbar_init(&sh.p_full, 8);
         mbar_init(&sh.dp_full, 1);
         mbar_init(&sh.ds_full, 8);
@@ -302,14 +303,23 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     const uint32_t nstage = stage + 1 == Cfg::kQStages ? 0 : stage + 1;
                     const bool has_next = n + 1 < N;
                     // dV += P^T dO
-                    TW(1, mbar_wait(&sh.p_full, g & 1u, guard));
+                    TW(1, mbar_wait(&sh.p_half, g & 1u, guard));
                     if (n == 0 && n_work >= 1) mbar_wait(&sh.dkv_free, (n_work - 1) & 1u, guard);
                     tc_fence_after();
                     TW(6,
 #pragma unroll
-                    for (int ks = 0; ks < kTile / 16; ++ks)
-                        if (leader) tc_mma_ts(tmem + Cfg::kDv, tmem + Cfg::kSt + (ks / 4) * 64 + (ks % 4) * 8, do_mn + mn_step(ks),
-                                  idesc_nd_kb, n > 0 || ks > 0);
+                    for (int part = 0; part < 2; ++part) {
+                        if (part == 1) {
+                            mbar_wait(&sh.p_full, g & 1u, guard);
+                            tc_fence_after();
+                        }
+#pragma unroll
+                        for (int k4 = 0; k4 < 4; ++k4) {
+                            const int ks = (k4 / 2) * 4 + part * 2 + (k4 % 2);     // k-steps {0,1,4,5} then {2,3,6,7}
+                            if (leader) tc_mma_ts(tmem + Cfg::kDv, tmem + Cfg::kSt + (ks / 4) * 64 + (ks % 4) * 8, do_mn + mn_step(ks),
+                                      idesc_nd_kb, n > 0 || part > 0 || k4 > 0);
+                        }
+                    }
                     if (leader) tc_commit(&sh.do_empty));
                     // S^T of the next tile
                     if (has_next) {
@@ -399,24 +409,29 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     tacc[7] += clock64() - _tp;
 #endif
 #pragma unroll
-                    for (int e = 0; e < 64; ++e) pf[e] = fast_exp2(__uint_as_float(sr[e]) * p.scale_log2);
-                }
-                if (key_tail || diag) {
-                    const int q_first = i * kTile + half * 64;   // query index of element 0
+                    for (int c = 0; c < 2; ++c) {
+                        // 32 query columns at a time: the dV product starts on the first chunk while the
+                        // second is still being exponentiated
 #pragma unroll
-                    for (int e = 0; e < 64; ++e)
-                        if (!key_valid || (diag && key > q_first + e)) pf[e] = 0.f;
-                }
+                        for (int e = 0; e < 32; ++e) pf[c * 32 + e] = fast_exp2(__uint_as_float(sr[c * 32 + e]) * p.scale_log2);
+                        if (key_tail || diag) {
+                            const int q_first = i * kTile + half * 64 + c * 32;   // query index of element 0
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t pk[16];
+                            for (int e = 0; e < 32; ++e)
+                                if (!key_valid || (diag && key > q_first + e)) pf[c * 32 + e] = 0.f;
+                        }
+                        uint32_t pk[16];
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) pk[e] = pack_bf16x2(pf[c * 32 + 2 * e], pf[c * 32 + 2 * e + 1]);
-                    tmem_st_x16(pt_tmem + c * 16, pk);
+                        for (int e = 0; e < 16; ++e) pk[e] = pack_bf16x2(pf[c * 32 + 2 * e], pf[c * 32 + 2 * e + 1]);
+                        tmem_st_x16(pt_tmem + c * 16, pk);
+                        if (c == 0) {
+                            tmem_wait_st();
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&sh.p_half);
+                        }
+                    }
                 }
-#ifdef DCP_TIMING
-                tacc[8] += clock64() - _tp;
-#endif
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
