@@ -21,8 +21,21 @@
 // key block of a sequence contributes to the same query rows.  The accumulator is a workspace, so
 // its layout is chosen for the atomics: per (tile, head) a block [d/4][128 rows][4 floats], which
 // makes the 32 rows a warp holds contiguous (full 32-byte sectors, four 128-byte lines per
-// instruction instead of 32 scattered ones); a small kernel converts it to [T, H, d] bf16 later. dK and dV stay in tensor memory for
-// the whole item and are written once (dK scaled by the softmax scale).
+// instruction instead of 32 scattered ones); a small kernel converts it to [T, H, d] bf16 later.
+// These 64 KB per (Q tile, K tile) pair are what bounds the kernel: the SM's path to L2 moves about
+// 15-25 bytes per clock for reductions, per-thread atomics and shared-memory bulk reductions alike,
+// and the atomics share the load/store unit with the compute warps' dS^T stores; with the atomics
+// compiled out the same kernel runs a third faster.  Measured and rejected: pacing the atomics,
+// bulk reductions from a 16 KB staging buffer, atomics into an L2-hot block (same time, so the
+// limit is on the SM's side), dK before dQ, and staggering the Q walk of neighbouring key blocks.
+// dK and dV stay in tensor memory for the whole item and are written once (dK scaled by the
+// softmax scale).
+//
+// The MMA warp runs its loop warp-uniformly and an elected lane issues: a tcgen05.mma issue blocks,
+// and a lone diverged thread that also computes descriptors pays 80-100 cycles per instruction, so
+// descriptors are built once per item and a k-step is a constant add.  P^T is published in two
+// parts (the first 32 query columns of each column group first), so the dV product starts on
+// those while the rest is still being exponentiated.
 //
 // Roles:  warps 0-7 compute (two groups, each owns 64 of the 128 query columns, one key per thread),
 //         warp 8 MMA issue, warp 9 scheduler + TMA producer + per-row statistics staging
