@@ -186,10 +186,22 @@ def run_ours(args):
         f = 14.0 * sum(float(L) * L for L in lengths) * d * H
         return 0.5 * f if causal else f
 
+    profile, plan_kw = None, {}
+    if args.plan == "profiled":
+        # Section 3.5: measure t_f, t_b per length bucket on this GPU (second of two runs) and let the
+        # planner use the table instead of its L^2 stand-in; T_C is then in nanoseconds
+        from paper_2608_07524_b200.profiler import dual_layer_profile
+        buckets = sorted(set(L for b in batches for L in b))
+        if len(buckets) > 16:
+            buckets = [buckets[i * (len(buckets) - 1) // 15] for i in range(16)]
+        profile = dual_layer_profile(buckets, H, d, causal, device=dev)
+        plan_kw = dict(profile=profile, fixed_cost=args.fixed_cost_ns)
+        name += f", planner fed by a {len(buckets)}-bucket dual-layer profile (T_C = {args.fixed_cost_ns} ns)"
+
     def step():
         tokens, flops = 0, 0.0
         for lengths in batches:
-            for mb in plan_batch(lengths, budget, H, d, n_layers=args.layers):
+            for mb in plan_batch(lengths, budget, H, d, n_layers=args.layers, **plan_kw):
                 tokens += runner.run_micro_batch(mb)
                 flops += flops_of(mb.lengths)
         return tokens, flops
@@ -324,6 +336,9 @@ def main():
     ap.add_argument("--workload", default="video", choices=["video", "text", "extreme", "stream"])
     ap.add_argument("--stream-batches", type=int, default=256)
     ap.add_argument("--layers", type=int, default=1, help="planner's layer count Lambda")
+    ap.add_argument("--plan", default="model", choices=["model", "profiled"],
+                    help="planner's forward-time source: the L^2 model or a dual-layer profile measured first")
+    ap.add_argument("--fixed-cost-ns", type=int, default=20000, help="T_C per micro-batch for --plan profiled")
     ap.add_argument("--budget-gb", type=float, default=180.0, help="planner's HBM budget in decimal GB")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--drop-longer-than", type=int, default=0,

@@ -67,6 +67,19 @@ typedef struct {
 int dcp_plan(const int32_t* lengths, int32_t n, int64_t hbm_budget_bytes, const dcp_plan_params* params,
              int32_t* mb_id, int32_t* n_mb, int32_t* recompute, int64_t* cost);
 
+/* The same planner fed by profiled times instead of the L^2 model.
+ *
+ * Paper: Section 3.5 (dual-layer profiling: the forward time t_f of one layer is measured per
+ * candidate and the whole model is extrapolated from it) and Eq. 5 (recomputing r layers costs
+ * r * t_f).  fwd_time [n] (host, each >= 0) is the measured or interpolated per-layer forward time
+ * of sequence i in any integer unit (nanoseconds, say); T_C (params->fixed_cost) is in the same
+ * unit.  Memory model, ordering, tie rules, outputs and errors are those of dcp_plan; the cost is
+ * K*T_C + sum_k r*_k * sum_{i in block k} fwd_time[i].  With fwd_time[i] = 2 * lengths[i]^2 the
+ * result equals dcp_plan's. */
+int dcp_plan_profiled(const int32_t* lengths, const int64_t* fwd_time, int32_t n, int64_t hbm_budget_bytes,
+                      const dcp_plan_params* params, int32_t* mb_id, int32_t* n_mb, int32_t* recompute,
+                      int64_t* cost);
+
 /* DCP-inter: accumulation-step counts that balance n batches running side by side.
  *
  * Paper: Section 3.3, Eq. 3, and Appendix C (G_min, G_max).  Batch i takes times[i] (any positive

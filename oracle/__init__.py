@@ -59,9 +59,9 @@ def _load():
                                              ci, i32p, f64p, f64p, f64p]
             lib.oracle_attn_cols.argtypes = [u16p, u16p, u16p, u16p, i32p, ci, ci, ci, cd, ci, ci,
                                              ci, i32p, f64p, f64p]
-            lib.oracle_plan_bruteforce.argtypes = [
-                i32p, ctypes.c_int32, ctypes.c_int64, ctypes.POINTER(PlanParams), i32p, i32p, i32p,
-                ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)]
+            lib.oracle_plan_bruteforce_weighted.argtypes = [
+                i32p, ctypes.POINTER(ctypes.c_int64), ctypes.c_int32, ctypes.c_int64, ctypes.POINTER(PlanParams),
+                i32p, i32p, i32p, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)]
             lib.oracle_inter_bruteforce.argtypes = [
                 ctypes.POINTER(ctypes.c_int64), ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, i32p,
                 ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)]
@@ -182,19 +182,24 @@ class Infeasible(Exception):
 
 
 def plan_bruteforce(lengths, budget: int, n_heads=16, head_dim=128, elt_bytes=2, n_layers=1,
-                    const_bytes=0, fixed_cost=1 << 24):
+                    const_bytes=0, fixed_cost=1 << 24, fwd_time=None):
     """Best plan by enumeration of all 2^(n-1) contiguous splits of the length-sorted list.
+    fwd_time (optional, one integer per sequence) replaces the 2 L^2 forward-time model (Section 3.5).
     Returns (mb_id list[n], recompute list[K], cost int)."""
     lengths = np.ascontiguousarray(lengths, dtype=np.int32)
     n = int(lengths.size)
+    wt = None if fwd_time is None else np.ascontiguousarray(fwd_time, dtype=np.int64)
+    if wt is not None and wt.size != n:
+        raise ValueError("fwd_time needs one entry per sequence")
     params = PlanParams(n_heads, head_dim, elt_bytes, n_layers, const_bytes, fixed_cost)
     mb = np.zeros(max(n, 1), np.int32)
     rec = np.zeros(max(n, 1), np.int32)
     n_mb = ctypes.c_int32(0)
     lo, hi = ctypes.c_uint64(0), ctypes.c_uint64(0)
-    rc = _load().oracle_plan_bruteforce(_p(lengths, ctypes.c_int32), n, int(budget), ctypes.byref(params),
-                                        _p(mb, ctypes.c_int32), ctypes.byref(n_mb), _p(rec, ctypes.c_int32),
-                                        ctypes.byref(lo), ctypes.byref(hi))
+    rc = _load().oracle_plan_bruteforce_weighted(_p(lengths, ctypes.c_int32),
+                                                 None if wt is None else _p(wt, ctypes.c_int64), n, int(budget),
+                                                 ctypes.byref(params), _p(mb, ctypes.c_int32), ctypes.byref(n_mb),
+                                                 _p(rec, ctypes.c_int32), ctypes.byref(lo), ctypes.byref(hi))
     if rc == 3:
         raise Infeasible()
     if rc:

@@ -22,6 +22,11 @@
  *   ties: smaller cost, then smaller K, then the lexicographically LARGEST vector of block
  *   sizes (the first block takes as many sequences as it can).
  *
+ * Profiled variant (Section 3.5: the per-layer forward time t_f comes from a measurement, not
+ * from a model): the caller passes t_f of every sequence as weight[i]; a block's recompute term
+ * is then r* * sum(weight) (Eq. 5) and the cost  K * T_C + sum_k r*_k sum_{i in k} weight[i].
+ * weight == NULL means weight[i] = 2 s_i^2, which is the model above.
+ *
  * All arithmetic is exact: unsigned __int128, far beyond what int64 inputs can reach.
  */
 #include <stdint.h>
@@ -59,16 +64,16 @@ static int min_recompute(u128 tok, const oracle_plan_params* p, u128 budget)
  *   cost_lo/hi    the 128-bit cost split into two 64-bit halves
  * n <= 24 (2^(n-1) plans are enumerated).
  */
-int oracle_plan_bruteforce(const int32_t* lengths, int32_t n, int64_t budget,
-                           const oracle_plan_params* p, int32_t* mb_id, int32_t* n_mb,
-                           int32_t* recompute, uint64_t* cost_lo, uint64_t* cost_hi)
+int oracle_plan_bruteforce_weighted(const int32_t* lengths, const int64_t* weight, int32_t n, int64_t budget,
+                                    const oracle_plan_params* p, int32_t* mb_id, int32_t* n_mb,
+                                    int32_t* recompute, uint64_t* cost_lo, uint64_t* cost_hi)
 {
     if (!lengths || !p || n < 1 || n > 24 || budget < 0 || p->n_layers < 1 || p->n_heads < 1 ||
         p->head_dim < 1 || p->elt_bytes < 1 || p->const_bytes < 0 || p->fixed_cost < 0)
         return 1;
     int64_t pairs[24][2];
     for (int i = 0; i < n; ++i) {
-        if (lengths[i] < 1) return 1;
+        if (lengths[i] < 1 || (weight && weight[i] < 0)) return 1;
         pairs[i][0] = lengths[i]; pairs[i][1] = i;
     }
     qsort(pairs, n, sizeof pairs[0], cmp_desc);
@@ -84,12 +89,12 @@ int oracle_plan_bruteforce(const int32_t* lengths, int32_t n, int64_t budget,
                 u128 tok = 0, W = 0;
                 for (int a = begin; a <= t; ++a) {
                     tok += (u128)pairs[a][0];
-                    W += (u128)pairs[a][0] * (u128)pairs[a][0];
+                    W += weight ? (u128)weight[pairs[a][1]] : 2 * (u128)pairs[a][0] * (u128)pairs[a][0];
                 }
                 int r = min_recompute(tok, p, (u128)budget);
                 if (r < 0) { feasible = 0; break; }
                 sizes[K] = t - begin + 1; rs[K] = r; ++K;
-                cost += (u128)p->fixed_cost + 2 * (u128)r * W;
+                cost += (u128)p->fixed_cost + (u128)r * W;
                 begin = t + 1;
             }
         }
@@ -117,4 +122,11 @@ int oracle_plan_bruteforce(const int32_t* lengths, int32_t n, int64_t budget,
     if (cost_lo) *cost_lo = (uint64_t)best_cost;
     if (cost_hi) *cost_hi = (uint64_t)(best_cost >> 64);
     return 0;
+}
+
+int oracle_plan_bruteforce(const int32_t* lengths, int32_t n, int64_t budget,
+                           const oracle_plan_params* p, int32_t* mb_id, int32_t* n_mb,
+                           int32_t* recompute, uint64_t* cost_lo, uint64_t* cost_hi)
+{
+    return oracle_plan_bruteforce_weighted(lengths, NULL, n, budget, p, mb_id, n_mb, recompute, cost_lo, cost_hi);
 }

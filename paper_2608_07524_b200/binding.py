@@ -44,10 +44,13 @@ def lib():
             i32, i64, vp, f32 = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float
             i32p = ctypes.POINTER(ctypes.c_int32)
             szp = ctypes.POINTER(ctypes.c_size_t)
+            i64p = ctypes.POINTER(ctypes.c_int64)
             L.dcp_plan.argtypes = [i32p, i32, i64, ctypes.POINTER(PlanParams), i32p, i32p, i32p,
                                    ctypes.POINTER(ctypes.c_int64)]
             L.dcp_plan.restype = ctypes.c_int
-            i64p = ctypes.POINTER(ctypes.c_int64)
+            L.dcp_plan_profiled.argtypes = [i32p, i64p, i32, i64, ctypes.POINTER(PlanParams), i32p, i32p, i32p,
+                                            ctypes.POINTER(ctypes.c_int64)]
+            L.dcp_plan_profiled.restype = ctypes.c_int
             L.dcp_inter_plan.argtypes = [i64p, i32, i32, i32, i32p, i64p, i64p]
             L.dcp_inter_plan.restype = ctypes.c_int
             L.dcp_varlen_attn_workspace.argtypes = [i32, i32, i32, i32, szp, szp]
@@ -111,6 +114,26 @@ def dcp_plan(lengths, hbm_budget_bytes: int, n_heads: int = 16, head_dim: int = 
     params = PlanParams(n_heads, head_dim, elt_bytes, n_layers, const_bytes, fixed_cost)
     _check(lib().dcp_plan(arr, n, int(hbm_budget_bytes), ctypes.byref(params), mb, ctypes.byref(n_mb), rec,
                           ctypes.byref(cost)))
+    return list(mb[:n]), list(rec[:n_mb.value]), int(cost.value)
+
+
+def dcp_plan_profiled(lengths, fwd_time, hbm_budget_bytes: int, n_heads: int = 16, head_dim: int = 128,
+                      elt_bytes: int = 2, n_layers: int = 1, const_bytes: int = 0, fixed_cost: int = 0
+                      ) -> Tuple[List[int], List[int], int]:
+    """dcp_plan with a profiled per-layer forward time per sequence (Section 3.5) instead of the L^2 model;
+    fixed_cost is in the unit of fwd_time."""
+    n = len(lengths)
+    if len(fwd_time) != n:
+        raise ValueError("fwd_time needs one entry per sequence")
+    arr = (ctypes.c_int32 * max(n, 1))(*[int(x) for x in lengths])
+    wt = (ctypes.c_int64 * max(n, 1))(*[int(x) for x in fwd_time])
+    mb = (ctypes.c_int32 * max(n, 1))()
+    rec = (ctypes.c_int32 * max(n, 1))()
+    n_mb = ctypes.c_int32(0)
+    cost = ctypes.c_int64(0)
+    params = PlanParams(n_heads, head_dim, elt_bytes, n_layers, const_bytes, fixed_cost)
+    _check(lib().dcp_plan_profiled(arr, wt, n, int(hbm_budget_bytes), ctypes.byref(params), mb, ctypes.byref(n_mb),
+                                   rec, ctypes.byref(cost)))
     return list(mb[:n]), list(rec[:n_mb.value]), int(cost.value)
 
 

@@ -43,33 +43,40 @@ int min_recompute(u128 tok, const dcp_plan_params& p, u128 budget) {
 
 }  // namespace
 
-extern "C" int dcp_plan(const int32_t* lengths, int32_t n, int64_t hbm_budget_bytes, const dcp_plan_params* params,
-                        int32_t* mb_id, int32_t* n_mb, int32_t* recompute, int64_t* cost) {
+namespace {
+
+// Shared body of dcp_plan and dcp_plan_profiled.  weight[i] is the per-layer forward time of
+// sequence i in the caller's unit (nullptr: the analytic stand-in 2 * length^2), so a block with
+// r recomputed layers adds r * sum(weight) to the objective (Eq. 5).
+int plan_impl(const char* who, const int32_t* lengths, const int64_t* weight, int32_t n, int64_t hbm_budget_bytes,
+              const dcp_plan_params* params, int32_t* mb_id, int32_t* n_mb, int32_t* recompute, int64_t* cost) {
     static const dcp_plan_params kDefaults = {16, 128, 2, 1, 0, (int64_t)1 << 24};
     const dcp_plan_params p = params ? *params : kDefaults;
-    if (!lengths || !mb_id || !n_mb || !recompute) return dcp::fail(DCP_ERR_INVALID_ARG, "dcp_plan: null pointer");
-    if (n < 1) return dcp::fail(DCP_ERR_INVALID_ARG, "dcp_plan: n = %d, need n >= 1", n);
-    if (hbm_budget_bytes < 0) return dcp::fail(DCP_ERR_INVALID_ARG, "dcp_plan: negative budget");
+    if (!lengths || !mb_id || !n_mb || !recompute) return dcp::fail(DCP_ERR_INVALID_ARG, "%s: null pointer", who);
+    if (n < 1) return dcp::fail(DCP_ERR_INVALID_ARG, "%s: n = %d, need n >= 1", who, n);
+    if (hbm_budget_bytes < 0) return dcp::fail(DCP_ERR_INVALID_ARG, "%s: negative budget", who);
     if (p.n_heads < 1 || p.head_dim < 1 || p.elt_bytes < 1 || p.n_layers < 1 || p.const_bytes < 0 || p.fixed_cost < 0)
-        return dcp::fail(DCP_ERR_INVALID_ARG, "dcp_plan: bad params (H, d, e, Lambda >= 1; M_C, T_C >= 0)");
-    for (int32_t i = 0; i < n; ++i)
-        if (lengths[i] < 1) return dcp::fail(DCP_ERR_INVALID_ARG, "dcp_plan: lengths[%d] = %d, need >= 1", i, lengths[i]);
+        return dcp::fail(DCP_ERR_INVALID_ARG, "%s: bad params (H, d, e, Lambda >= 1; M_C, T_C >= 0)", who);
+    for (int32_t i = 0; i < n; ++i) {
+        if (lengths[i] < 1) return dcp::fail(DCP_ERR_INVALID_ARG, "%s: lengths[%d] = %d, need >= 1", who, i, lengths[i]);
+        if (weight && weight[i] < 0) return dcp::fail(DCP_ERR_INVALID_ARG, "%s: fwd_time[%d] is negative", who, i);
+    }
 
     std::vector<int32_t> order(n);
     std::iota(order.begin(), order.end(), 0);
     std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return lengths[a] > lengths[b]; });
 
     // prefix sums over the sorted order
-    std::vector<u128> tok(n + 1, 0), sq(n + 1, 0);
+    std::vector<u128> tok(n + 1, 0), w(n + 1, 0);
     for (int32_t i = 0; i < n; ++i) {
         const u128 L = (u128)lengths[order[i]];
         tok[i + 1] = tok[i] + L;
-        sq[i + 1] = sq[i] + L * L;
+        w[i + 1] = w[i] + (weight ? (u128)weight[order[i]] : 2 * L * L);
     }
     const u128 budget = (u128)hbm_budget_bytes;
     if (min_recompute(tok[1] - tok[0], p, budget) < 0)
         return dcp::fail(DCP_ERR_INFEASIBLE,
-                         "dcp_plan: the longest sequence (%d tokens) exceeds the budget even with every layer recomputed",
+                         "%s: the longest sequence (%d tokens) exceeds the budget even with every layer recomputed", who,
                          lengths[order[0]]);
 
     // best[i] = optimum for the sorted suffix i..n-1; cut[i] = end of its first block (largest on ties)
@@ -81,14 +88,14 @@ extern "C" int dcp_plan(const int32_t* lengths, int32_t n, int64_t hbm_budget_by
         for (int32_t j = i + 1; j <= n; ++j) {
             const int r = min_recompute(tok[j] - tok[i], p, budget);
             if (r < 0) break;                                  // larger blocks only need more memory
-            const Key cand = {best[j].cost + (u128)p.fixed_cost + 2 * (u128)r * (sq[j] - sq[i]), best[j].blocks + 1};
+            const Key cand = {best[j].cost + (u128)p.fixed_cost + (u128)r * (w[j] - w[i]), best[j].blocks + 1};
             if (!have || cand < best[i] || cand == best[i]) {  // '==' keeps the LARGEST j among ties
                 best[i] = cand; cut[i] = j; rec[i] = r; have = true;
             }
         }
         // a single sequence always fits here: the longest one does and memory grows with length
     }
-    if (best[0].cost > kInt64Max) return dcp::fail(DCP_ERR_OVERFLOW, "dcp_plan: cost does not fit in int64");
+    if (best[0].cost > kInt64Max) return dcp::fail(DCP_ERR_OVERFLOW, "%s: cost does not fit in int64", who);
 
     int32_t k = 0;
     for (int32_t i = 0; i < n; i = cut[i], ++k) {
@@ -98,4 +105,18 @@ extern "C" int dcp_plan(const int32_t* lengths, int32_t n, int64_t hbm_budget_by
     *n_mb = k;
     if (cost) *cost = (int64_t)best[0].cost;
     return DCP_OK;
+}
+
+}  // namespace
+
+extern "C" int dcp_plan(const int32_t* lengths, int32_t n, int64_t hbm_budget_bytes, const dcp_plan_params* params,
+                        int32_t* mb_id, int32_t* n_mb, int32_t* recompute, int64_t* cost) {
+    return plan_impl("dcp_plan", lengths, nullptr, n, hbm_budget_bytes, params, mb_id, n_mb, recompute, cost);
+}
+
+extern "C" int dcp_plan_profiled(const int32_t* lengths, const int64_t* fwd_time, int32_t n, int64_t hbm_budget_bytes,
+                                 const dcp_plan_params* params, int32_t* mb_id, int32_t* n_mb, int32_t* recompute,
+                                 int64_t* cost) {
+    if (!fwd_time) return dcp::fail(DCP_ERR_INVALID_ARG, "dcp_plan_profiled: null pointer");
+    return plan_impl("dcp_plan_profiled", lengths, fwd_time, n, hbm_budget_bytes, params, mb_id, n_mb, recompute, cost);
 }

@@ -26,9 +26,17 @@ class MicroBatch:
 
 
 def plan_batch(lengths: Sequence[int], hbm_budget_bytes: int, n_heads: int, head_dim: int,
-               n_layers: int = 1, fixed_cost: int = 1 << 24) -> List[MicroBatch]:
-    mb_id, recompute, _ = binding.dcp_plan(lengths, hbm_budget_bytes, n_heads=n_heads, head_dim=head_dim,
-                                           n_layers=n_layers, fixed_cost=fixed_cost)
+               n_layers: int = 1, fixed_cost: int = 1 << 24, profile=None) -> List[MicroBatch]:
+    """Micro-batches of one batch.  With `profile` (a profiler.ProfileTable) the per-layer forward
+    time of every sequence comes from the measured table (Section 3.5) and fixed_cost is in
+    nanoseconds; without it the planner uses its L^2 stand-in and fixed_cost is in its units."""
+    if profile is None:
+        mb_id, recompute, _ = binding.dcp_plan(lengths, hbm_budget_bytes, n_heads=n_heads, head_dim=head_dim,
+                                               n_layers=n_layers, fixed_cost=fixed_cost)
+    else:
+        fwd_time = [profile.fwd_time(int(L)) for L in lengths]
+        mb_id, recompute, _ = binding.dcp_plan_profiled(lengths, fwd_time, hbm_budget_bytes, n_heads=n_heads,
+                                                        head_dim=head_dim, n_layers=n_layers, fixed_cost=fixed_cost)
     out = [MicroBatch([], r) for r in recompute]
     # inside a micro-batch keep the planner's order: longest first, ties by input index
     for i in sorted(range(len(lengths)), key=lambda i: (-lengths[i], i)):

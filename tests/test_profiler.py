@@ -1,0 +1,135 @@
+"""Profiled planning (Section 3.5 feeding Eq. 5): the planner with measured per-sequence forward
+times against the brute-force oracle, and the host logic of the dual-layer profiler."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2608_07524_b200 import binding as B
+from paper_2608_07524_b200.profiler import ProfileTable, dual_layer_profile
+from paper_2608_07524_b200.stream import plan_batch
+
+
+def both(lengths, fwd_time, budget, **kw):
+    try:
+        ref = oracle.plan_bruteforce(lengths, budget, fwd_time=fwd_time, **kw)
+    except oracle.Infeasible:
+        ref = None
+    try:
+        got = B.dcp_plan_profiled(lengths, fwd_time, budget, **kw)
+    except B.DcpError as e:
+        assert e.code == B.DCP_ERR_INFEASIBLE
+        got = None
+    return got, ref
+
+
+def test_profiled_planner_matches_bruteforce_on_random_cases():
+    rng = np.random.default_rng(5)
+    for _ in range(3000):
+        n = int(rng.integers(1, 11))
+        lengths = [int(x) for x in rng.integers(1, 500, size=n)]
+        # times unrelated to length on purpose: the planner may not assume any shape of t_f(L)
+        fwd_time = [int(x) for x in rng.integers(0, 10 ** int(rng.integers(1, 12)), size=n)]
+        lam = int(rng.choice([1, 2, 4, 28]))
+        TC = int(rng.choice([0, 1, 50, 10 ** 5, 1 << 24, 1 << 40]))
+        unit = 2 * 8 * 2
+        budget = int(rng.integers(max(lam * unit * max(lengths) - 40, 0), 5 * lam * unit * sum(lengths) + 2))
+        got, ref = both(lengths, fwd_time, budget, n_heads=2, head_dim=8, n_layers=lam, fixed_cost=TC)
+        assert got == ref, (lengths, fwd_time, budget, lam, TC)
+
+
+def test_profiled_with_model_times_equals_model_planner():
+    rng = np.random.default_rng(6)
+    for _ in range(500):
+        n = int(rng.integers(1, 20))
+        lengths = [int(x) for x in rng.integers(1, 3000, size=n)]
+        lam = int(rng.choice([1, 3, 28]))
+        budget = int(rng.integers(lam * 32 * max(lengths), 5 * lam * 32 * sum(lengths) + 2))
+        kw = dict(n_heads=2, head_dim=8, n_layers=lam, fixed_cost=12345)
+        assert B.dcp_plan_profiled(lengths, [2 * L * L for L in lengths], budget, **kw) == B.dcp_plan(lengths, budget, **kw)
+
+
+def test_hand_worked_case():
+    # two sequences of 10 tokens, H = d = e = 1, Lambda = 1: mem(r) of a block = (1 - r) 4 tok + tok.
+    # budget 60: both together need 100 at r = 0 and 20 at r = 1, so r = 1; alone each needs 50, r = 0.
+    # together costs T_C + 1 * (7 + 5), split costs 2 T_C: split wins iff T_C < 12, a tie goes to fewer blocks.
+    kw = dict(n_heads=1, head_dim=1, elt_bytes=1, n_layers=1)
+    assert B.dcp_plan_profiled([10, 10], [7, 5], 60, fixed_cost=11, **kw) == ([0, 1], [0, 0], 22)
+    assert B.dcp_plan_profiled([10, 10], [7, 5], 60, fixed_cost=13, **kw) == ([0, 0], [1], 25)
+    assert B.dcp_plan_profiled([10, 10], [7, 5], 60, fixed_cost=12, **kw) == ([0, 0], [1], 24)   # tie: fewer blocks
+    assert oracle.plan_bruteforce([10, 10], 60, fixed_cost=12, fwd_time=[7, 5], **kw) == ([0, 0], [1], 24)
+
+
+def test_profiled_argument_errors():
+    with pytest.raises(B.DcpError) as e:
+        B.dcp_plan_profiled([5, 6], [1, -1], 10 ** 9)
+    assert e.value.code == B.DCP_ERR_INVALID_ARG
+    with pytest.raises(ValueError):
+        B.dcp_plan_profiled([5, 6], [1], 10 ** 9)
+    with pytest.raises(B.DcpError) as e:
+        B.dcp_plan_profiled([5, 6], [2 ** 62, 2 ** 62], 16 * 128 * 2 * 11 + 1, n_layers=2, fixed_cost=2 ** 62)
+    assert e.value.code in (B.DCP_ERR_OVERFLOW, B.DCP_ERR_INFEASIBLE)
+
+
+def test_interpolation_rule():
+    t = ProfileTable([100, 200, 400], [1000, 3000, 11000], [2000, 7000, 30000], [1, 2, 4])
+    assert [t.fwd_time(L) for L in (100, 200, 400)] == [1000, 3000, 11000]
+    assert t.fwd_time(50) == 500 and t.fwd_time(1) == 10            # linear below the first bucket
+    assert t.fwd_time(150) == 2000 and t.fwd_time(201) == 3040      # linear between, floor
+    assert t.fwd_time(800) == 44000 and t.fwd_time(401) == 11000 * 401 * 401 // 160000   # quadratic above
+    assert t.bwd_time(300) == 18500
+    xs = [t.fwd_time(L) for L in range(1, 1000)]
+    assert all(b >= a for a, b in zip(xs, xs[1:]))
+    # Eq. 4-5: Lambda (t_f + t_b) + r t_f + T_C
+    assert t.model_time([100, 200], 3, 2, 7) == 3 * (4000 + 9000) + 2 * 4000 + 7
+    with pytest.raises(ValueError):
+        ProfileTable([100, 100], [1, 2], [1, 2], [1, 2])
+    with pytest.raises(ValueError):
+        t.fwd_time(0)
+
+
+def test_dual_layer_profile_keeps_the_second_run():
+    calls = []
+
+    def fake_layer(lengths):
+        calls.append(list(lengths))
+        first = sum(1 for c in calls if c == list(lengths)) == 1
+        L, n = lengths[0], len(lengths)
+        return (999.0, 999.0) if first else (n * L * L * 1e-6, n * L * L * 3e-6)   # ms
+
+    t = dual_layer_profile([256, 64, 1024], n_heads=4, head_dim=32, causal=False, fill_tokens=1024, run_layer=fake_layer)
+    assert t.lengths == [64, 256, 1024]
+    assert [len(c) for c in calls] == [16, 16, 4, 4, 1, 1]          # batches hold about fill_tokens tokens
+    assert t.t_f_ns == [64 * 64, 256 * 256, 1024 * 1024]            # per sequence, ns; warm-up discarded
+    assert t.t_b_ns == [3 * x for x in t.t_f_ns]
+    assert t.m_bytes == [4 * L * 4 * 32 * 2 for L in t.lengths]
+
+
+def test_plan_batch_with_profile_uses_measured_times():
+    # a table in which recomputing is nearly free makes one micro-batch with recompute the best plan;
+    # one in which it is expensive makes the planner split instead
+    lengths = [4000, 3000, 2000, 1000]
+    unit = 16 * 128 * 2
+    budget = 3 * unit * sum(lengths)              # all four together only fit when recomputed
+    cheap = ProfileTable([1000, 4000], [1, 4], [1, 4], [1, 1])
+    dear = ProfileTable([1000, 4000], [10 ** 6, 16 * 10 ** 6], [1, 4], [1, 1])
+    one = plan_batch(lengths, budget, 16, 128, n_layers=1, fixed_cost=1000, profile=cheap)
+    assert [m.lengths for m in one] == [lengths] and one[0].recompute == 1
+    many = plan_batch(lengths, budget, 16, 128, n_layers=1, fixed_cost=1000, profile=dear)
+    assert len(many) == 2 and all(m.recompute == 0 for m in many)
+    assert sorted(sum((m.lengths for m in many), [])) == sorted(lengths)
+
+
+@pytest.mark.gpu
+def test_profile_on_device_and_plan():
+    t = dual_layer_profile([512, 2048, 8192], n_heads=16, head_dim=128, causal=False, fill_tokens=1 << 15)
+    assert all(x > 0 for x in t.t_f_ns + t.t_b_ns)
+    assert t.t_f_ns[0] < t.t_f_ns[1] < t.t_f_ns[2] and t.t_b_ns[0] < t.t_b_ns[1] < t.t_b_ns[2]
+    # the kernels are quadratic in length once tensor-bound: 4x the length costs 8-20x the time
+    assert 8 < t.t_f_ns[2] / t.t_f_ns[1] < 20
+    assert all(b > f for f, b in zip(t.t_f_ns, t.t_b_ns))
+    lengths = [9600, 9600, 3600, 2048, 1024, 256]
+    mbs = plan_batch(lengths, 5 * 16 * 128 * 2 * 14000, 16, 128, n_layers=1, fixed_cost=20000, profile=t)
+    assert sorted(sum((m.lengths for m in mbs), [])) == sorted(lengths)
+    ref = oracle.plan_bruteforce(lengths, 5 * 16 * 128 * 2 * 14000, fixed_cost=20000,
+                                 fwd_time=[t.fwd_time(L) for L in lengths])
+    assert [m.recompute for m in mbs] == ref[1]
