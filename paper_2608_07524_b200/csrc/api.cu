@@ -138,6 +138,7 @@ SchedView carve_sched(void* workspace, int32_t n_seqs) {
     s.order = reinterpret_cast<const int32_t*>(base + sizeof(WorkspaceHeader));
     s.prefix = reinterpret_cast<const uint32_t*>(base + sizeof(WorkspaceHeader) + sizeof(int32_t) * (size_t)n_seqs);
     s.tile_prefix = s.prefix + (size_t)n_seqs + 1;
+    s.vcu = reinterpret_cast<const int32_t*>(s.tile_prefix + (size_t)n_seqs + 1);
     s.n_seqs = n_seqs;
     return s;
 }
@@ -157,7 +158,7 @@ extern "C" int dcp_varlen_attn_workspace(int32_t total_tokens, int32_t n_seqs, i
                                          size_t* fwd_bytes, size_t* bwd_bytes) {
     if (total_tokens < 0 || n_seqs < 0 || n_heads < 1 || head_dim < 1)
         return fail(DCP_ERR_INVALID_ARG, "dcp_varlen_attn_workspace: bad sizes");
-    const size_t sched = sched_bytes(n_seqs);
+    const size_t sched = sched_bytes(n_seqs) + bounds_bytes(total_tokens);
     if (fwd_bytes) *fwd_bytes = sched;
     if (bwd_bytes)
         *bwd_bytes = sched + align256(max_tiles(total_tokens, n_seqs) * n_heads * (size_t)(kTile * 16 * 2)) +
@@ -165,18 +166,21 @@ extern "C" int dcp_varlen_attn_workspace(int32_t total_tokens, int32_t n_seqs, i
     return DCP_OK;
 }
 
-extern "C" int dcp_varlen_attn_fwd(const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
-                                   int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen, int32_t n_heads,
-                                   int32_t head_dim, int32_t causal, float softmax_scale, void* o, float* lse,
-                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
-    const char* fn = "dcp_varlen_attn_fwd";
+// `merge` = false builds the work list over cu_seqlens itself and needs only sched_bytes of workspace
+// (the entry point with built-in scratch, whose size cannot depend on the token count, uses it);
+// the results are the same either way.
+static int attn_fwd_impl(const char* fn, bool merge, const void* q, const void* k, const void* v,
+                         const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen,
+                         int32_t n_heads, int32_t head_dim, int32_t causal, float softmax_scale, void* o, float* lse,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
     if (int rc = check_shape(fn, n_seqs, total_tokens, max_seqlen, n_heads, head_dim, softmax_scale)) return rc;
     if (!cu_seqlens) return fail(DCP_ERR_INVALID_ARG, "%s: cu_seqlens is null", fn);
     if (!workspace) return fail(DCP_ERR_WORKSPACE, "%s: workspace is null", fn);
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
         return fail(DCP_ERR_WORKSPACE, "%s: workspace must be 256-byte aligned", fn);
-    if (workspace_bytes < sched_bytes(n_seqs))
-        return fail(DCP_ERR_WORKSPACE, "%s: workspace has %zu bytes, needs %zu", fn, workspace_bytes, sched_bytes(n_seqs));
+    const size_t need = sched_bytes(n_seqs) + (merge ? bounds_bytes(total_tokens) : 0);
+    if (workspace_bytes < need)
+        return fail(DCP_ERR_WORKSPACE, "%s: workspace has %zu bytes, needs %zu", fn, workspace_bytes, need);
     if (total_tokens > 0 && (!q || !k || !v || !o || !lse)) return fail(DCP_ERR_INVALID_ARG, "%s: null tensor pointer", fn);
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o))
         return fail(DCP_ERR_INVALID_ARG, "%s: tensor pointers must be 16-byte aligned", fn);
@@ -186,13 +190,14 @@ extern "C" int dcp_varlen_attn_fwd(const void* q, const void* k, const void* v, 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
     const SchedView sched = carve_sched(workspace, n_seqs);
+    uint16_t* bounds = merge ? reinterpret_cast<uint16_t*>(static_cast<uint8_t*>(workspace) + sched_bytes(n_seqs)) : nullptr;
     cudaError_t e;
     {
         ScopedTimer t(DCP_KERNEL_PREP, stream);
-        e = launch_prep(cu_seqlens, n_seqs, kFwdRowsPerItem, n_heads, sched, stream);
+        e = launch_prep(cu_seqlens, n_seqs, total_tokens, max_seqlen, kFwdRowsPerItem, n_heads, sched, bounds, stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: work-list kernel: %s", fn, cudaGetErrorString(e));
-    g_launches.fetch_add(prep_launches(n_seqs));
+    g_launches.fetch_add(prep_launches(n_seqs, merge));
     if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
 
     CUtensorMap tq, tk, tv;
@@ -201,7 +206,8 @@ extern "C" int dcp_varlen_attn_fwd(const void* q, const void* k, const void* v, 
     if (int rc = make_map(&tv, v, total_tokens, n_heads, head_dim)) return rc;
 
     FwdParams p;
-    p.cu_seqlens = cu_seqlens;
+    p.cu_seqlens = merge ? sched.vcu : cu_seqlens;
+    p.bounds = bounds;
     p.o = static_cast<__nv_bfloat16*>(o);
     p.lse = lse;
     p.sched = sched;
@@ -216,6 +222,14 @@ extern "C" int dcp_varlen_attn_fwd(const void* q, const void* k, const void* v, 
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: attention kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(1);
     return DCP_OK;
+}
+
+extern "C" int dcp_varlen_attn_fwd(const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
+                                   int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen, int32_t n_heads,
+                                   int32_t head_dim, int32_t causal, float softmax_scale, void* o, float* lse,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return attn_fwd_impl("dcp_varlen_attn_fwd", true, q, k, v, cu_seqlens, n_seqs, total_tokens, max_seqlen, n_heads,
+                         head_dim, causal, softmax_scale, o, lse, workspace, workspace_bytes, cuda_stream);
 }
 
 extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
@@ -243,17 +257,19 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
     const SchedView sched = carve_sched(workspace, n_seqs);
-    uint8_t* base = static_cast<uint8_t*>(workspace) + sched_bytes(n_seqs);
+    uint16_t* bounds = reinterpret_cast<uint16_t*>(static_cast<uint8_t*>(workspace) + sched_bytes(n_seqs));
+    uint8_t* base = static_cast<uint8_t*>(workspace) + sched_bytes(n_seqs) + bounds_bytes(total_tokens);
     __nv_bfloat16* stats = reinterpret_cast<__nv_bfloat16*>(base);
     float* dq_acc = reinterpret_cast<float*>(base + align256(max_tiles(total_tokens, n_seqs) * n_heads * (size_t)(kTile * 16 * 2)));
 
     cudaError_t e;
     {
         ScopedTimer t(DCP_KERNEL_PREP, stream);
-        e = launch_prep(cu_seqlens, n_seqs, kTile, n_heads, sched, stream);
+        e = launch_prep(cu_seqlens, n_seqs, total_tokens, max_seqlen, kTile, n_heads, sched, bounds, stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: work-list kernel: %s", fn, cudaGetErrorString(e));
-    g_launches.fetch_add(prep_launches(n_seqs));
+    g_launches.fetch_add(prep_launches(n_seqs, true));
+    const int32_t* vcu = sched.vcu;      // every later kernel works on the virtual sequences
     if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
 
     CUtensorMap tq, tk, tv, tg;
@@ -264,7 +280,7 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
 
     {
         ScopedTimer t(DCP_KERNEL_BWD_PRE, stream);
-        e = launch_bwd_pre(static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, cu_seqlens,
+        e = launch_bwd_pre(static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, vcu,
                            sched, stats, dq_acc, max_tiles(total_tokens, n_seqs) * kTile * n_heads * head_dim,
                            total_tokens, n_heads, head_dim,
                            softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim), dev.sm_count, stream);
@@ -273,7 +289,8 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
     g_launches.fetch_add(1);
 
     BwdParams p;
-    p.cu_seqlens = cu_seqlens;
+    p.cu_seqlens = vcu;
+    p.bounds = bounds;
     p.stats = stats;
     p.dq_acc = dq_acc;
     p.dk = static_cast<__nv_bfloat16*>(dk);
@@ -292,7 +309,7 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
 
     {
         ScopedTimer t(DCP_KERNEL_BWD_POST, stream);
-        e = launch_bwd_post(dq_acc, static_cast<__nv_bfloat16*>(dq), cu_seqlens, sched, n_heads, head_dim, p.scale,
+        e = launch_bwd_post(dq_acc, static_cast<__nv_bfloat16*>(dq), vcu, sched, n_heads, head_dim, p.scale,
                             dev.sm_count, stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: post kernel: %s", fn, cudaGetErrorString(e));
@@ -308,9 +325,7 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
 // outputs only.  Every GPU that loads this library holds the array until the process exits.
 #define DCP_NOALLOC_MAX_SEQS_VALUE 4096
 namespace {
-constexpr size_t kNoAllocScratchBytes =
-    (sizeof(dcp::WorkspaceHeader) + sizeof(int32_t) * DCP_NOALLOC_MAX_SEQS_VALUE +
-     2 * sizeof(uint32_t) * (DCP_NOALLOC_MAX_SEQS_VALUE + 1) + 255) / 256 * 256;
+constexpr size_t kNoAllocScratchBytes = dcp::sched_bytes(DCP_NOALLOC_MAX_SEQS_VALUE);
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
 }  // namespace
 
@@ -344,8 +359,9 @@ extern "C" int dcp_varlen_attn_fwd_noalloc(const void* q, const void* k, const v
     }
     if (sched_bytes(n_seqs) > kNoAllocScratchBytes)      // cannot happen for n_seqs <= the maximum; kept as a guard
         return fail(DCP_ERR_UNSUPPORTED, "%s: built-in scratch too small", fn);
-    return dcp_varlen_attn_fwd(q, k, v, cu_seqlens, n_seqs, total_tokens, max_seqlen, n_heads, head_dim, causal,
-                               softmax_scale, o, lse, scratch, kNoAllocScratchBytes, cuda_stream);
+    // short sequences are not merged here: the table that needs is sized by the token count
+    return attn_fwd_impl(fn, false, q, k, v, cu_seqlens, n_seqs, total_tokens, max_seqlen, n_heads, head_dim, causal,
+                         softmax_scale, o, lse, scratch, kNoAllocScratchBytes, cuda_stream);
 }
 
 extern "C" int dcp_query_status(const void* workspace, void* cuda_stream) {

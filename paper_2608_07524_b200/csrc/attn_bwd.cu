@@ -403,6 +403,15 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             const int key = w.blk * kTile + key_in_tile;
             const bool key_valid = key < w.len;
             const bool key_tail = (w.blk + 1) * kTile > w.len;
+            // in a virtual sequence of merged sequences a key is seen only by the queries at positions
+            // [q_lo, q_hi) of its own sequence
+            const bool merged = p.bounds != nullptr && w.len <= kTile;
+            int q_lo = 0, q_hi = 0x7fffffff;
+            if (merged && key_valid) {
+                const uint32_t b = p.bounds[(size_t)w.tok0 + key];
+                q_lo = (int)(b & 0xffu);
+                q_hi = (int)(b >> 8);
+            }
 
             for (int i = first_q; i < n_q; ++i, ++g) {
                 const bool diag = CAUSAL && i == w.blk;
@@ -427,11 +436,13 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         // second is still being exponentiated
 #pragma unroll
                         for (int e = 0; e < 32; ++e) pf[c * 32 + e] = fast_exp2(__uint_as_float(sr[c * 32 + e]) * p.scale_log2);
-                        if (key_tail || diag) {
+                        if (key_tail || diag || merged) {
                             const int q_first = i * kTile + half * 64 + c * 32;   // query index of element 0
 #pragma unroll
-                            for (int e = 0; e < 32; ++e)
-                                if (!key_valid || (diag && key > q_first + e)) pf[c * 32 + e] = 0.f;
+                            for (int e = 0; e < 32; ++e) {
+                                const int qi = q_first + e;
+                                if (!key_valid || (diag && key > qi) || qi < q_lo || qi >= q_hi) pf[c * 32 + e] = 0.f;
+                            }
                         }
                         uint32_t pk[16];
 #pragma unroll

@@ -312,6 +312,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             const int nkv = kv_tiles_for<CAUSAL>(r_tile, w.len);
             if (nkv == 0) continue;
             const int row = r_tile + row_in_tile;       // row inside the sequence (may be >= len)
+            // a virtual sequence of at most one tile may hold several merged sequences: the row then
+            // sees only the positions [lo_key, hi_key) of its own sequence
+            const bool merged = p.bounds != nullptr && w.len <= kTile;
+            int lo_key = 0, hi_key = w.len;
+            if (merged && row < w.len) {
+                const uint32_t b = p.bounds[(size_t)w.tok0 + row];
+                lo_key = (int)(b & 0xffu);
+                hi_key = (int)(b >> 8);
+            }
 
             float m = -INFINITY, l = 0.f;
             for (int j = 0; j < nkv; ++j) {
@@ -326,13 +335,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 for (int c = 0; c < 4; ++c) tmem_ld_x32(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
                 tmem_wait_ld();
 
-                const bool boundary = (j == nkv - 1) && (CAUSAL || (w.len & (kTile - 1)) != 0);
+                const bool boundary = (j == nkv - 1) && (CAUSAL || merged || (w.len & (kTile - 1)) != 0);
                 if (boundary) {
-                    const int last_key = CAUSAL ? (row < w.len - 1 ? row : w.len - 1) : w.len - 1;
+                    const int last_key = CAUSAL ? (row < hi_key - 1 ? row : hi_key - 1) : hi_key - 1;
                     const int n_valid = last_key - j * kTile + 1;     // >= 1
+                    const int n_before = lo_key - j * kTile;          // > 0 only in a merged tile
 #pragma unroll
                     for (int c = 0; c < 128; ++c)
-                        if (c >= n_valid) s[c] = 0xff800000u;         // -inf
+                        if (c >= n_valid || c < n_before) s[c] = 0xff800000u;         // -inf
                 }
                 float part[8];      // eight independent chains instead of one 128-long one
 #pragma unroll

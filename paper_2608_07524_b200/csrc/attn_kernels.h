@@ -9,7 +9,8 @@
 namespace dcp {
 
 struct FwdParams {
-    const int32_t* cu_seqlens;
+    const int32_t* cu_seqlens;    // boundaries of the (virtual) sequences the work list was built over
+    const uint16_t* bounds;       // per-token table of the merged path (see sched.cuh), or null
     __nv_bfloat16* o;
     float* lse;
     SchedView sched;
@@ -20,7 +21,8 @@ struct FwdParams {
 };
 
 struct BwdParams {
-    const int32_t* cu_seqlens;
+    const int32_t* cu_seqlens;    // as in FwdParams
+    const uint16_t* bounds;
     const __nv_bfloat16* stats;   // per (tile, head) a [128 queries x 16] bf16 tile in the layout the MMA reads:
                                   // columns 0-2 = -lse/scale split in three bf16 parts, 8-10 = -D likewise
                                   // (D_i = sum_c dO_ic O_ic); rows past the sequence end hold -1e30 and 0
@@ -35,9 +37,13 @@ struct BwdParams {
 };
 
 // Builds the work list (longest sequence first) and resets the work counter and status word.
-int prep_launches(int32_t n_seqs);   // kernels launch_prep enqueues for a batch of n_seqs sequences (1 or 2)
-cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t rows_per_block, int32_t n_heads,
-                        const SchedView& sched, cudaStream_t stream);
+// With `bounds` non-null, short sequences are first merged into virtual sequences: sched.vcu and
+// `bounds` are written and the list is built over sched.vcu, which the later kernels must then be
+// given as their boundary array; with `bounds` null the list is built over cu_seqlens itself.
+int prep_launches(int32_t n_seqs, bool merge);   // kernels launch_prep enqueues (1 to 3)
+cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen,
+                        int32_t rows_per_block, int32_t n_heads, const SchedView& sched, uint16_t* bounds,
+                        cudaStream_t stream);
 
 cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                             int head_dim, bool causal, int n_ctas, cudaStream_t stream);

@@ -9,20 +9,89 @@ namespace dcp {
 
 constexpr int kPrepThreads = 1024;
 
+// Merging of short sequences into virtual sequences of at most 128 tokens.  One CTA.
+//
+// A sequence is "short" if length <= max_short (empty ones included).  Consecutive short sequences whose first
+// tokens fall into the same window of `window` = 129 - max_short packed positions form one virtual
+// sequence: it spans at most (window - 1) + max_short = 128 tokens.  The rule is local (a sequence
+// starts a virtual sequence iff it is not short, or its predecessor is not short, or the predecessor
+// starts in another window), so heads are found in parallel and compacted with a scan.
+// Outputs: vcu[0..n_v] = boundaries of the virtual sequences, vcu[n_v+1..n_seqs] = total_tokens
+// (empty padding, so that vcu is a valid boundary array of n_seqs sequences); hdr->n_vseq = n_v;
+// bounds[t] for every token t of an input sequence of at most 128 tokens = (first, end) position of
+// that sequence relative to its virtual sequence, one byte each.
+__global__ void __launch_bounds__(kPrepThreads) merge_kernel(const int32_t* __restrict__ cu, int32_t n_seqs,
+                                                             int32_t total_tokens, int32_t max_short,
+                                                             WorkspaceHeader* hdr, int32_t* vcu, uint16_t* bounds) {
+    __shared__ uint32_t chunk_sum[kPrepThreads];
+    __shared__ uint32_t n_v_sh;
+    const int tid = threadIdx.x;
+    const int window = kTile + 1 - max_short;
+    auto is_short = [&](int i) { return cu[i + 1] - cu[i] <= max_short; };
+    auto is_head = [&](int i) {
+        return i == 0 || !is_short(i) || !is_short(i - 1) || cu[i - 1] / window != cu[i] / window;
+    };
+    const int per = (n_seqs + kPrepThreads - 1) / kPrepThreads;
+    const int begin = min(tid * per, n_seqs), end = min(begin + per, n_seqs);
+    uint32_t local = 0;
+    for (int i = begin; i < end; ++i) local += is_head(i) ? 1u : 0u;
+    chunk_sum[tid] = local;
+    __syncthreads();
+    if (tid == 0) {
+        uint32_t run = 0;
+        for (int i = 0; i < kPrepThreads; ++i) {
+            const uint32_t c = chunk_sum[i];
+            chunk_sum[i] = run;
+            run += c;
+        }
+        n_v_sh = run;
+        hdr->n_vseq = run;
+    }
+    __syncthreads();
+    uint32_t run = chunk_sum[tid];
+    int32_t vstart = 0;
+    if (begin < end && !is_head(begin)) {            // the virtual sequence began in an earlier chunk
+        int j = begin - 1;
+        while (!is_head(j)) --j;                     // at most 127 non-empty members: a virtual sequence has <= 128 tokens
+        vstart = cu[j];
+    }
+    for (int i = begin; i < end; ++i) {
+        const int32_t a = cu[i], b = cu[i + 1];
+        if (is_head(i)) {
+            vcu[run++] = a;
+            vstart = a;
+        }
+        if (b - a <= kTile) {
+            const uint16_t packed = (uint16_t)((a - vstart) | ((b - vstart) << 8));
+            for (int32_t t = a; t < b; ++t) bounds[t] = packed;
+        }
+    }
+    const uint32_t n_v = n_v_sh;
+    for (uint32_t i = n_v + tid; i <= (uint32_t)n_seqs; i += kPrepThreads) vcu[i] = total_tokens;
+}
+
 // Rank sort, one thread per sequence over as many CTAs as needed: order[] = sequence ids sorted by
 // (length descending, id ascending).  Used on its own for batches of more than kPrepThreads
-// sequences; small batches do the same loop inside prep_kernel and save the launch.
-__global__ void __launch_bounds__(256) rank_kernel(const int32_t* __restrict__ cu, int32_t n_seqs, int32_t* order) {
+// sequences; small batches do the same loop inside prep_kernel and save the launch.  Sequences
+// from *n_live on (if given) are empty padding: they keep their own index as rank and are not
+// compared against.
+__global__ void __launch_bounds__(256) rank_kernel(const int32_t* __restrict__ cu, int32_t n_seqs,
+                                                   const uint32_t* __restrict__ n_live_ptr, int32_t* order) {
     __shared__ int32_t len_tile[256];
+    const int n_live = n_live_ptr ? min((int)*n_live_ptr, n_seqs) : n_seqs;
     const int i = blockIdx.x * 256 + threadIdx.x;
+    if ((int)blockIdx.x * 256 >= n_live) {             // a whole block of padding
+        if (i < n_seqs) order[i] = i;
+        return;
+    }
     const int32_t len_i = i < n_seqs ? cu[i + 1] - cu[i] : 0;
-    int rank = 0;
-    for (int j0 = 0; j0 < n_seqs; j0 += 256) {
+    int rank = i > n_live ? i - n_live : 0;             // padding before i, all of length 0 like i itself
+    for (int j0 = 0; j0 < n_live; j0 += 256) {
         const int j = j0 + threadIdx.x;
         __syncthreads();
-        len_tile[threadIdx.x] = j < n_seqs ? cu[j + 1] - cu[j] : -1;     // -1 never outranks anything
+        len_tile[threadIdx.x] = j < n_live ? cu[j + 1] - cu[j] : -1;     // -1 never outranks anything
         __syncthreads();
-        const int cnt = min(256, n_seqs - j0);
+        const int cnt = min(256, n_live - j0);
         for (int t = 0; t < cnt; ++t) {
             const int32_t len_j = len_tile[t];
             rank += (len_j > len_i) || (len_j == len_i && j0 + t < i);
@@ -106,16 +175,27 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __res
     }
 }
 
-int prep_launches(int32_t n_seqs) { return n_seqs > kPrepThreads ? 2 : 1; }
+int prep_launches(int32_t n_seqs, bool merge) { return (n_seqs > kPrepThreads ? 2 : 1) + (merge ? 1 : 0); }
 
-cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t rows_per_block, int32_t n_heads,
-                        const SchedView& sched, cudaStream_t stream) {
+cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen,
+                        int32_t rows_per_block, int32_t n_heads, const SchedView& sched, uint16_t* bounds,
+                        cudaStream_t stream) {
+    const int32_t* cu = cu_seqlens;
+    const uint32_t* n_live = nullptr;
+    if (bounds) {                                       // merge short sequences; everything below sees vcu
+        const int32_t max_short = max_seqlen < kMergeMaxLen ? (max_seqlen > 0 ? max_seqlen : 1) : kMergeMaxLen;
+        merge_kernel<<<1, kPrepThreads, 0, stream>>>(cu_seqlens, n_seqs, total_tokens, max_short, sched.hdr,
+                                                     const_cast<int32_t*>(sched.vcu), bounds);
+        if (cudaError_t e = cudaGetLastError()) return e;
+        cu = sched.vcu;
+        n_live = &sched.hdr->n_vseq;
+    }
     const int ranked = n_seqs > kPrepThreads;
     if (ranked) {
-        rank_kernel<<<(n_seqs + 255) / 256, 256, 0, stream>>>(cu_seqlens, n_seqs, const_cast<int32_t*>(sched.order));
+        rank_kernel<<<(n_seqs + 255) / 256, 256, 0, stream>>>(cu, n_seqs, n_live, const_cast<int32_t*>(sched.order));
         if (cudaError_t e = cudaGetLastError()) return e;
     }
-    prep_kernel<<<1, kPrepThreads, 0, stream>>>(cu_seqlens, n_seqs, rows_per_block, n_heads, sched.hdr,
+    prep_kernel<<<1, kPrepThreads, 0, stream>>>(cu, n_seqs, rows_per_block, n_heads, sched.hdr,
                                                 const_cast<int32_t*>(sched.order), const_cast<uint32_t*>(sched.prefix),
                                                 const_cast<uint32_t*>(sched.tile_prefix), ranked);
     return cudaGetLastError();
@@ -209,6 +289,9 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
         }
         }
     }
+    // only the tiles in use: the workspace is sized for an upper bound on the tile count
+    const size_t used_vec4 = (size_t)n_blocks * (size_t)(kTile * D / 4);
+    if (used_vec4 < dq_acc_vec4) dq_acc_vec4 = used_vec4;
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < dq_acc_vec4; i += stride)
         reinterpret_cast<float4*>(dq_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);

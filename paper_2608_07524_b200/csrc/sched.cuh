@@ -4,6 +4,13 @@
 // on one GPU the same problem shows up as SMs idling while one long sequence finishes.  The work
 // list therefore orders sequences longest first, and persistent CTAs pull items from it through a
 // global atomic counter, so the cheap items of short sequences fill the tail.
+//
+// Very short sequences (a 2-D model's temporal axis has 1-13 tokens per sequence) would each
+// occupy a whole 128-row tile.  Runs of consecutive short sequences are therefore merged into
+// "virtual sequences" of at most 128 tokens that the kernels treat as one tile with a
+// block-diagonal mask: the work list is built over the virtual boundaries `vcu` (a subsequence of
+// cu_seqlens, padded with empty sequences), and a per-token table gives, for tokens of virtual
+// sequences of at most 128 tokens, the range of positions the token's own sequence covers.
 #pragma once
 #include <cstdint>
 
@@ -11,35 +18,51 @@ namespace dcp {
 
 constexpr int kTile = 128;            // rows of a Q tile / keys of a K,V tile
 constexpr int kFwdRowsPerItem = 256;  // a forward work item is two Q tiles of one (sequence, head)
+constexpr int kMergeMaxLen = 64;      // sequences longer than this are never merged with their neighbours
 
 // First bytes of every workspace.  `status` must stay at offset 0 (dcp_query_status reads it).
 struct WorkspaceHeader {
     uint32_t status;        // 0 = ok, else a kStatus* code left by a kernel
     uint32_t work_counter;  // next unclaimed work item
     uint32_t n_items;       // items in the list
-    uint32_t pad[61];
+    uint32_t n_vseq;        // virtual sequences that are not padding
+    uint32_t pad[60];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
 
 // After the header: int32 order[n_seqs] (sequence ids, longest first, ties by id),
-// uint32 prefix[n_seqs + 1] (items before the i-th sequence of `order`) and
-// uint32 tile_prefix[n_seqs + 1] (128-row tiles before sequence b, in input order).
+// uint32 prefix[n_seqs + 1] (items before the i-th sequence of `order`),
+// uint32 tile_prefix[n_seqs + 1] (128-row tiles before sequence b, in input order) and
+// int32 vcu[n_seqs + 1] (virtual sequence boundaries; unused when sequences are not merged).
+// All of these are indexed by VIRTUAL sequence; `cu` is the boundary array the kernels read
+// (vcu, or the caller's cu_seqlens when merging is off).
 struct SchedView {
     WorkspaceHeader* hdr;
     const int32_t* order;
     const uint32_t* prefix;
     const uint32_t* tile_prefix;
+    const int32_t* vcu;
     int32_t n_seqs;
 };
 
-__host__ __device__ inline size_t sched_bytes(int32_t n_seqs) {
-    size_t b = sizeof(WorkspaceHeader) + sizeof(int32_t) * (size_t)n_seqs + 2 * sizeof(uint32_t) * ((size_t)n_seqs + 1);
-    return (b + 255) & ~(size_t)255;
+__host__ __device__ constexpr size_t sched_bytes(int32_t n_seqs) {
+    return (sizeof(WorkspaceHeader) + sizeof(int32_t) * (size_t)n_seqs + 2 * sizeof(uint32_t) * ((size_t)n_seqs + 1) +
+            sizeof(int32_t) * ((size_t)n_seqs + 1) + 255) & ~(size_t)255;
 }
 
-// Upper bound on the number of 128-row tiles of a packed batch (every sequence may end in a partial tile).
+// Per-token table of the merged path: low byte = first position, high byte = one past the last
+// position of the token's own sequence, both relative to the start of its virtual sequence.
+__host__ __device__ constexpr size_t bounds_bytes(int32_t total_tokens) {
+    return (sizeof(uint16_t) * (size_t)total_tokens + 255) & ~(size_t)255;
+}
+
+// Upper bound on the number of 128-row tiles of a packed batch: every (virtual) sequence may end in
+// a partial tile.  After merging there are at most n_seqs virtual sequences and also at most
+// 3 T / 65 + 2: one starts at sequence 0, at a sequence longer than kMergeMaxLen (at most T / 65 of
+// those), right after such a sequence, or where the window changes (a window has >= 65 positions).
 __host__ __device__ inline size_t max_tiles(int32_t total_tokens, int32_t n_seqs) {
-    return (size_t)total_tokens / kTile + (size_t)n_seqs;
+    const size_t by_windows = 3 * ((size_t)total_tokens / (kTile + 1 - kMergeMaxLen)) + 3;
+    return (size_t)total_tokens / kTile + ((size_t)n_seqs < by_windows ? (size_t)n_seqs : by_windows);
 }
 
 // A decoded work item.  len < 0 marks the end of the list.

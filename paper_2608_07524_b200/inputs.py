@@ -14,6 +14,9 @@ length distribution of Section 2.1 and the three synthetic mixes of Appendix A):
   config 4  "extreme"  one 131072-token sequence plus 64 lengths uniform in [128, 2048];
                        8 heads, head_dim 128; causal
   config 5  "stream"   256 batches, each 24 draws of the config-3 rule from one generator
+  "short2d"            the config-3 clips seen by a model that attends along one axis at a time
+                       (the paper's second architecture): per latent frame over its 256-3600
+                       tokens, then per spatial position over its 1-13 latent frames
 
 Uniform variates come from SplitMix64 so the draws are reproducible in any language.  The
 lists for configs 2-4 are also stored as text under tests/golden/ and a test checks that this
@@ -55,16 +58,36 @@ _RES = ((0.5, 256, 256), (0.8, 480, 640), (1.01, 720, 1280))
 _FRAMES = ((0.4, 1), (0.7, 16), (0.9, 32), (1.01, 51))
 
 
-def _video_draw(g: SplitMix64) -> int:
+def _video_sample(g: SplitMix64):
+    """(latent frames, tokens per latent frame) of one clip."""
     u1, u2 = g.uniform(), g.uniform()
     h, w = next((hh, ww) for t, hh, ww in _RES if u1 < t)
     frames = next(f for t, f in _FRAMES if u2 < t)
-    return -(-frames // 4) * (h // 16) * (w // 16)
+    return -(-frames // 4), (h // 16) * (w // 16)
+
+
+def _video_draw(g: SplitMix64) -> int:
+    f, s = _video_sample(g)
+    return f * s
 
 
 def video_lengths(n: int = 24, seed: int = 3) -> List[int]:
     g = SplitMix64(seed)
     return [_video_draw(g) for _ in range(n)]
+
+
+def short2d_lengths(axis: str, n: int = 24, seed: int = 3) -> List[int]:
+    """The config-3 clips as a 2-D model sees them (attention along one axis at a time): `spatial`
+    gives one sequence per latent frame (its tokens attend to each other), `temporal` one sequence
+    per spatial position (its frames attend to each other).  Both hold the same tokens in total."""
+    g = SplitMix64(seed)
+    out: List[int] = []
+    for _ in range(n):
+        f, s = _video_sample(g)
+        out += [s] * f if axis == "spatial" else [f] * s
+    if axis not in ("spatial", "temporal"):
+        raise ValueError("axis must be 'spatial' or 'temporal'")
+    return out
 
 
 def extreme_lengths(n_short: int = 64, seed: int = 4, long_len: int = 131072) -> List[int]:

@@ -94,6 +94,53 @@ def test_many_short_sequences(causal):
     check_full([int(x) for x in rng.integers(1, 200, size=300)], 2, 64, causal, seed=5)
 
 
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("d", [64, 128])
+def test_merged_tiny_sequences(causal, d):
+    # a 2-D model's temporal axis: thousands of sequences of 1-13 tokens, several of which share one tile
+    rng = np.random.default_rng(11)
+    check_full([int(x) for x in rng.choice([1, 4, 8, 13], size=700)], 2, d, causal, seed=11)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_merged_mixed_with_long_and_empty(causal):
+    # merged runs are broken by long, empty and medium sequences; lengths around the merge limit (64)
+    # and the tile size; a run that fills a tile exactly
+    lengths = [3, 5, 0, 7, 300, 1, 1, 1, 64, 64, 65, 63, 2, 128, 9, 0, 0, 4, 127, 13, 13, 13, 13, 13, 13, 13, 13, 13,
+               11, 129, 6, 6, 6, 6, 100, 2, 2, 60, 60, 8, 32, 32, 32, 32, 1]
+    check_full(lengths, 3, 128, causal, seed=12)
+
+
+def test_merged_all_single_tokens():
+    # every sequence has one token: O = V, dV = dO, dQ = dK = 0 whatever the packing
+    n = 1000
+    cu = np.arange(n + 1, dtype=np.int32)
+    q, k, v, g = inputs.make_qkvg(n, 2, 64, 13)
+    o, lse, dq, dk, dv = run_gpu(q, k, v, g, cu, False)
+    assert torch.equal(o.cpu(), v) and torch.equal(dv.cpu(), g)
+    # dS = P (dP - D) with dP = D up to fp32 rounding of two different summation orders
+    assert float(dq.float().abs().max()) <= 1e-4 and float(dk.float().abs().max()) <= 1e-4
+    ref_lse = (q.double() * k.double()).sum(-1).T.numpy() / 8.0
+    assert float(np.max(np.abs(to64(lse) - ref_lse))) <= LSE_ABS
+
+
+def test_merged_packing_independence():
+    # neighbours inside the same merged tile must not leak into each other
+    lengths = [10, 13, 7, 20, 13]
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    q, k, v, g = inputs.make_qkvg(int(cu[-1]), 2, 128, 14)
+    a = run_gpu(q, k, v, g, cu, False)
+    q2, k2, v2, g2 = (x.clone() for x in (q, k, v, g))
+    for x in (q2, k2, v2, g2):
+        x[:23] = torch.randn_like(x[:23].float()).to(torch.bfloat16) * 3
+        x[30:] = torch.randn_like(x[30:].float()).to(torch.bfloat16) * 3
+    b = run_gpu(q2, k2, v2, g2, cu, False)
+    for i in (0, 3, 4):
+        assert torch.equal(a[i][23:30], b[i][23:30])
+    assert torch.equal(a[1][:, 23:30], b[1][:, 23:30])
+    assert float((a[2][23:30].float() - b[2][23:30].float()).abs().max()) <= 2e-2
+
+
 def test_more_sequences_than_one_sorting_block():
     # above 1024 sequences the work list is ranked by a separate multi-CTA kernel
     rng = np.random.default_rng(6)
@@ -163,7 +210,7 @@ def test_launch_counter_and_profile():
     B.dcp_profile_read()
     before = B.dcp_launch_count()
     run_gpu(q, k, v, g, w.cu_seqlens, False)
-    assert B.dcp_launch_count() - before == 2 + 4          # forward: prep + main; backward: prep + 3
+    assert B.dcp_launch_count() - before == 3 + 5          # forward: merge + prep + main; backward: merge + prep + 3
     prof = B.dcp_profile_read()
     B.dcp_profile_enable(False)
     assert prof["fwd"][1] == 1 and prof["bwd_main"][1] == 1 and prof["prep"][1] == 2
