@@ -115,11 +115,80 @@ __device__ __forceinline__ void bwd_load_tile(uint8_t* dst, const CUtensorMap* m
         tma_load_3d(dst + b * BwdCfg<D>::kBoxBytes, map, bar, b * 64, head, row);
 }
 
+// Compute-warp work of an item that is a single tile pair (a virtual sequence of at most 128 tokens,
+// in which short sequences may have been merged): P^T and dS^T with a key seen only by the queries at
+// the positions of its own sequence, which the per-token table gives.  Kept out of line so that the
+// loop of the common case is compiled exactly as it would be without this path.  `g` is the running
+// tile-pair count of the calling thread (it selects the barrier phases).
+template <bool CAUSAL>
+__device__ __noinline__ void compute_single_tile_item(BwdControl& sh, const BwdParams& p, const WorkItem w, uint32_t st_tmem,
+                                                      uint32_t dp_tmem, uint8_t* ds_row, int half, int key_in_tile,
+                                                      uint32_t g, const WaitGuard guard) {
+    const int lane = threadIdx.x & 31;
+    const bool key_valid = key_in_tile < w.len;
+    int q_lo = 0, q_hi = 0;
+    if (key_valid) {
+        const uint32_t b = p.bounds[(size_t)w.tok0 + key_in_tile];
+        q_lo = (int)(b & 0xffu);
+        q_hi = (int)(b >> 8);
+    }
+    if (CAUSAL && key_in_tile > q_lo) q_lo = key_in_tile;     // a key is seen from its own position on
+    float pf[64];
+    mbar_wait(&sh.s_full, g & 1u, guard);
+    tc_fence_after();
+    {
+        uint32_t sr[64];
+        tmem_ld_x32(st_tmem, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+        tmem_ld_x32(st_tmem + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            const int q_first = half * 64 + c * 32;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+                const int qi = q_first + e;
+                const float x = fast_exp2(__uint_as_float(sr[c * 32 + e]) * p.scale_log2);
+                pf[c * 32 + e] = (qi >= q_lo && qi < q_hi) ? x : 0.f;
+            }
+            uint32_t pk[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) pk[e] = pack_bf16x2(pf[c * 32 + 2 * e], pf[c * 32 + 2 * e + 1]);
+            tmem_st_x16(st_tmem + c * 16, pk);
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(c == 0 ? &sh.p_half : &sh.p_full);
+        }
+    }
+    mbar_wait(&sh.dp_full, g & 1u, guard);
+    if (g >= 1) mbar_wait(&sh.ds_free, (g - 1) & 1u, guard);
+    tc_fence_after();
+    {
+        uint32_t dr[64];
+        tmem_ld_x32(dp_tmem, *reinterpret_cast<uint32_t(*)[32]>(&dr[0]));
+        tmem_ld_x32(dp_tmem + 32, *reinterpret_cast<uint32_t(*)[32]>(&dr[32]));
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            uint32_t pk[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                pk[e] = pack_bf16x2(pf[c * 8 + 2 * e] * __uint_as_float(dr[c * 8 + 2 * e]),
+                                    pf[c * 8 + 2 * e + 1] * __uint_as_float(dr[c * 8 + 2 * e + 1]));
+            *reinterpret_cast<uint4*>(ds_row + sw128_offset(key_in_tile, c)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+    }
+    fence_async_smem();
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sh.ds_full);
+}
+
 template <int D, bool CAUSAL>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_do,
-                const BwdParams p) {
+                const __grid_constant__ BwdParams p) {
     using Cfg = BwdCfg<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
     BwdControl& sh = *reinterpret_cast<BwdControl*>(smem + Cfg::kOffCtl);
@@ -403,16 +472,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             const int key = w.blk * kTile + key_in_tile;
             const bool key_valid = key < w.len;
             const bool key_tail = (w.blk + 1) * kTile > w.len;
-            // in a virtual sequence of merged sequences a key is seen only by the queries at positions
-            // [q_lo, q_hi) of its own sequence
-            const bool merged = p.bounds != nullptr && w.len <= kTile;
-            int q_lo = 0, q_hi = 0x7fffffff;
-            if (merged && key_valid) {
-                const uint32_t b = p.bounds[(size_t)w.tok0 + key];
-                q_lo = (int)(b & 0xffu);
-                q_hi = (int)(b >> 8);
-            }
 
+            if (p.bounds != nullptr && w.len <= kTile) {     // one tile pair, possibly several merged sequences
+                compute_single_tile_item<CAUSAL>(sh, p, w, st_tmem, dp_tmem, ds_row, half, key_in_tile, g, guard);
+                ++g;
+                first_q = n_q;                                // nothing left for the loop below
+            }
             for (int i = first_q; i < n_q; ++i, ++g) {
                 const bool diag = CAUSAL && i == w.blk;
                 float pf[64];
@@ -436,13 +501,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         // second is still being exponentiated
 #pragma unroll
                         for (int e = 0; e < 32; ++e) pf[c * 32 + e] = fast_exp2(__uint_as_float(sr[c * 32 + e]) * p.scale_log2);
-                        if (key_tail || diag || merged) {
+                        if (key_tail || diag) {
                             const int q_first = i * kTile + half * 64 + c * 32;   // query index of element 0
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) {
-                                const int qi = q_first + e;
-                                if (!key_valid || (diag && key > qi) || qi < q_lo || qi >= q_hi) pf[c * 32 + e] = 0.f;
-                            }
+                            for (int e = 0; e < 32; ++e)
+                                if (!key_valid || (diag && key > q_first + e)) pf[c * 32 + e] = 0.f;
                         }
                         uint32_t pk[16];
 #pragma unroll

@@ -114,10 +114,87 @@ __device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint6
     }
 }
 
+// Softmax of a work item that is a single tile (a virtual sequence of at most 128 tokens, in which
+// short sequences may have been merged): the row of a token sees only the positions of its own
+// sequence, given by the per-token table.  Kept out of line so that the multi-tile loop of the common
+// case is compiled exactly as it would be without this path.  Called by the 128 threads of softmax
+// group 0 with the parities of their next s_full and o_full phases.
+template <int D, bool CAUSAL>
+__device__ __noinline__ void softmax_single_tile_item(FwdShared& sh, const FwdParams& p, const WorkItem w,
+                                                      uint32_t s_tmem, uint32_t o_tmem, uint32_t s_parity,
+                                                      uint32_t o_parity, const WaitGuard guard) {
+    const int lane = threadIdx.x & 31;
+    const int row = threadIdx.x & 127;
+    const bool valid = row < w.len;
+    int first_key = 0, end_key = w.len;
+    if (valid) {
+        const uint32_t b = p.bounds[(size_t)w.tok0 + row];
+        first_key = (int)(b & 0xffu);
+        end_key = (int)(b >> 8);
+    }
+    const int last_key = CAUSAL ? (row < end_key - 1 ? row : end_key - 1) : end_key - 1;
+    mbar_wait(&sh.s_full[0], s_parity, guard);
+    tc_fence_after();
+    uint32_t s[128];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) tmem_ld_x32(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+    tmem_wait_ld();
+    float m = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 128; ++c) {
+        if (c > last_key || c < first_key) s[c] = 0xff800000u;         // -inf
+        m = fmaxf(m, __uint_as_float(s[c]));
+    }
+    const float neg_m = -m * p.scale_log2;
+    float l = 0.f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const float p0 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + 2 * i]), p.scale_log2, neg_m));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + 2 * i + 1]), p.scale_log2, neg_m));
+            l += p0 + p1;
+            pk[i] = pack_bf16x2(p0, p1);
+        }
+        tmem_st_x16(s_tmem + c * 16, pk);
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.p_part[0][c]);
+    }
+    mbar_wait(&sh.o_full[0], o_parity, guard);
+    tc_fence_after();
+    const float inv_l = 1.0f / l;
+    const size_t tok = (size_t)w.tok0 + (size_t)row;
+    __nv_bfloat16* out = p.o + (tok * p.n_heads + w.head) * D;
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) {
+        uint32_t acc[32];
+        tmem_ld_x32(o_tmem + c * 32, acc);
+        tmem_wait_ld();
+        if (valid) {
+#pragma unroll
+            for (int v4 = 0; v4 < 4; ++v4) {
+                uint4 val;
+                val.x = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 0]) * inv_l, __uint_as_float(acc[v4 * 8 + 1]) * inv_l);
+                val.y = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 2]) * inv_l, __uint_as_float(acc[v4 * 8 + 3]) * inv_l);
+                val.z = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 4]) * inv_l, __uint_as_float(acc[v4 * 8 + 5]) * inv_l);
+                val.w = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 6]) * inv_l, __uint_as_float(acc[v4 * 8 + 7]) * inv_l);
+                *reinterpret_cast<uint4*>(out + c * 32 + v4 * 8) = val;
+            }
+        }
+    }
+    if (valid) p.lse[(size_t)w.head * p.total_tokens + tok] = m * p.scale + __logf(l);
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sh.o_free[0]);
+}
+
 template <int D, bool CAUSAL>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                const __grid_constant__ CUtensorMap tmap_v, const FwdParams p) {
+                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ FwdParams p) {
     using Cfg = FwdCfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -308,19 +385,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             if (lane == 0) mbar_arrive(&sh.work_empty[slot]);
             ++n_work;
             if (w.len < 0) break;
+            if (p.bounds != nullptr && w.len <= kTile) {      // one tile, possibly several merged sequences
+                if (t == 0) {
+                    softmax_single_tile_item<D, CAUSAL>(sh, p, w, s_tmem, o_tmem, n_s & 1u, use & 1u, guard);
+                    ++n_s;
+                    ++use;
+                }
+                continue;
+            }
             const int r_tile = w.blk * kFwdRowsPerItem + t * kTile;
             const int nkv = kv_tiles_for<CAUSAL>(r_tile, w.len);
             if (nkv == 0) continue;
             const int row = r_tile + row_in_tile;       // row inside the sequence (may be >= len)
-            // a virtual sequence of at most one tile may hold several merged sequences: the row then
-            // sees only the positions [lo_key, hi_key) of its own sequence
-            const bool merged = p.bounds != nullptr && w.len <= kTile;
-            int lo_key = 0, hi_key = w.len;
-            if (merged && row < w.len) {
-                const uint32_t b = p.bounds[(size_t)w.tok0 + row];
-                lo_key = (int)(b & 0xffu);
-                hi_key = (int)(b >> 8);
-            }
 
             float m = -INFINITY, l = 0.f;
             for (int j = 0; j < nkv; ++j) {
@@ -335,14 +411,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 for (int c = 0; c < 4; ++c) tmem_ld_x32(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
                 tmem_wait_ld();
 
-                const bool boundary = (j == nkv - 1) && (CAUSAL || merged || (w.len & (kTile - 1)) != 0);
+                const bool boundary = (j == nkv - 1) && (CAUSAL || (w.len & (kTile - 1)) != 0);
                 if (boundary) {
-                    const int last_key = CAUSAL ? (row < hi_key - 1 ? row : hi_key - 1) : hi_key - 1;
+                    const int last_key = CAUSAL ? (row < w.len - 1 ? row : w.len - 1) : w.len - 1;
                     const int n_valid = last_key - j * kTile + 1;     // >= 1
-                    const int n_before = lo_key - j * kTile;          // > 0 only in a merged tile
 #pragma unroll
                     for (int c = 0; c < 128; ++c)
-                        if (c >= n_valid || c < n_before) s[c] = 0xff800000u;         // -inf
+                        if (c >= n_valid) s[c] = 0xff800000u;         // -inf
                 }
                 float part[8];      // eight independent chains instead of one 128-long one
 #pragma unroll

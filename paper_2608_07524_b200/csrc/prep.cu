@@ -9,6 +9,8 @@ namespace dcp {
 
 constexpr int kPrepThreads = 1024;
 
+__device__ inline uint32_t block_exclusive_scan(uint32_t v, uint32_t* scratch, uint32_t* total);
+
 // Merging of short sequences into virtual sequences of at most 128 tokens.  One CTA.
 //
 // A sequence is "short" if length <= max_short (empty ones included).  Consecutive short sequences whose first
@@ -23,8 +25,7 @@ constexpr int kPrepThreads = 1024;
 __global__ void __launch_bounds__(kPrepThreads) merge_kernel(const int32_t* __restrict__ cu, int32_t n_seqs,
                                                              int32_t total_tokens, int32_t max_short,
                                                              WorkspaceHeader* hdr, int32_t* vcu, uint16_t* bounds) {
-    __shared__ uint32_t chunk_sum[kPrepThreads];
-    __shared__ uint32_t n_v_sh;
+    __shared__ uint32_t scratch[33];
     const int tid = threadIdx.x;
     const int window = kTile + 1 - max_short;
     auto is_short = [&](int i) { return cu[i + 1] - cu[i] <= max_short; };
@@ -33,22 +34,10 @@ __global__ void __launch_bounds__(kPrepThreads) merge_kernel(const int32_t* __re
     };
     const int per = (n_seqs + kPrepThreads - 1) / kPrepThreads;
     const int begin = min(tid * per, n_seqs), end = min(begin + per, n_seqs);
-    uint32_t local = 0;
+    uint32_t local = 0, n_v = 0;
     for (int i = begin; i < end; ++i) local += is_head(i) ? 1u : 0u;
-    chunk_sum[tid] = local;
-    __syncthreads();
-    if (tid == 0) {
-        uint32_t run = 0;
-        for (int i = 0; i < kPrepThreads; ++i) {
-            const uint32_t c = chunk_sum[i];
-            chunk_sum[i] = run;
-            run += c;
-        }
-        n_v_sh = run;
-        hdr->n_vseq = run;
-    }
-    __syncthreads();
-    uint32_t run = chunk_sum[tid];
+    uint32_t run = block_exclusive_scan(local, scratch, &n_v);
+    if (tid == 0) hdr->n_vseq = n_v;
     int32_t vstart = 0;
     if (begin < end && !is_head(begin)) {            // the virtual sequence began in an earlier chunk
         int j = begin - 1;
@@ -66,7 +55,6 @@ __global__ void __launch_bounds__(kPrepThreads) merge_kernel(const int32_t* __re
             for (int32_t t = a; t < b; ++t) bounds[t] = packed;
         }
     }
-    const uint32_t n_v = n_v_sh;
     for (uint32_t i = n_v + tid; i <= (uint32_t)n_seqs; i += kPrepThreads) vcu[i] = total_tokens;
 }
 
@@ -100,79 +88,94 @@ __global__ void __launch_bounds__(256) rank_kernel(const int32_t* __restrict__ c
     if (i < n_seqs) order[rank] = i;
 }
 
+// Exclusive prefix sum of one value per thread over a CTA of kPrepThreads threads; *total receives
+// the sum.  scratch holds 33 words.
+__device__ inline uint32_t block_exclusive_scan(uint32_t v, uint32_t* scratch, uint32_t* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t incl = v;
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, s);
+        if (lane >= s) incl += t;
+    }
+    __syncthreads();                       // scratch may still be read from an earlier call
+    if (lane == 31) scratch[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t w = scratch[lane];
+        uint32_t wi = w;
+#pragma unroll
+        for (int s = 1; s < 32; s <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, wi, s);
+            if (lane >= s) wi += t;
+        }
+        scratch[lane] = wi - w;
+        if (lane == 31) scratch[32] = wi;
+    }
+    __syncthreads();
+    *total = scratch[32];
+    return scratch[warp] + incl - v;
+}
+
 // One CTA.  order[] as above (computed here unless `ranked`); prefix[i] = number of work items of the
 // first i sequences in that order, where a sequence of length L contributes
 // ceil(L / rows_per_block) * n_heads items; tile_prefix[b] = 128-row tiles before sequence b.
+// Sequences from *n_live_ptr on (if given) are empty padding and sorted last: only the live ones
+// are scanned, the rest get the totals.
 __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __restrict__ cu, int32_t n_seqs,
+                                                            const uint32_t* __restrict__ n_live_ptr,
                                                             int32_t rows_per_block, int32_t n_heads,
                                                             WorkspaceHeader* hdr, int32_t* order, uint32_t* prefix,
                                                             uint32_t* tile_prefix, int ranked) {
-    __shared__ uint32_t chunk_sum[kPrepThreads];
+    __shared__ uint32_t scratch[33];
+    __shared__ int32_t len_sh[kPrepThreads];
     const int tid = threadIdx.x;
-    if (!ranked) {
-        for (int i = tid; i < n_seqs; i += kPrepThreads) {
-            const int32_t len_i = cu[i + 1] - cu[i];
+    const int n_live = n_live_ptr ? min((int)*n_live_ptr, n_seqs) : n_seqs;
+    if (!ranked) {                                    // n_seqs <= kPrepThreads: one sequence per thread
+        len_sh[tid] = tid < n_seqs ? cu[tid + 1] - cu[tid] : -1;
+        __syncthreads();
+        if (tid < n_seqs) {
+            const int32_t len_i = len_sh[tid];
             int rank = 0;
             for (int j = 0; j < n_seqs; ++j) {
-                const int32_t len_j = cu[j + 1] - cu[j];
-                rank += (len_j > len_i) || (len_j == len_i && j < i);
+                const int32_t len_j = len_sh[j];
+                rank += (len_j > len_i) || (len_j == len_i && j < tid);
             }
-            order[rank] = i;
+            order[rank] = tid;
         }
     }
     __syncthreads();
     // exclusive scan of item counts over the sorted order: contiguous chunk per thread
-    const int per = (n_seqs + kPrepThreads - 1) / kPrepThreads;
-    const int begin = tid * per, end = min(begin + per, n_seqs);
+    const int per = (n_live + kPrepThreads - 1) / kPrepThreads;
+    const int begin = min(tid * per, n_live), end = min(begin + per, n_live);
     auto items_of = [&](int pos) -> uint32_t {
         const int s = order[pos];
         const int32_t len = cu[s + 1] - cu[s];
         return (uint32_t)((len + rows_per_block - 1) / rows_per_block) * (uint32_t)n_heads;
     };
-    uint32_t local = 0;
+    uint32_t local = 0, total = 0;
     for (int i = begin; i < end; ++i) local += items_of(i);
-    chunk_sum[tid] = local;
-    __syncthreads();
-    if (tid == 0) {
-        uint32_t run = 0;
-        for (int i = 0; i < kPrepThreads; ++i) {
-            const uint32_t c = chunk_sum[i];
-            chunk_sum[i] = run;
-            run += c;
-        }
-        prefix[n_seqs] = run;
-        hdr->n_items = run;
-        hdr->work_counter = 0;
-        hdr->status = 0;
-    }
-    __syncthreads();
-    uint32_t run = chunk_sum[tid];
+    uint32_t run = block_exclusive_scan(local, scratch, &total);
     for (int i = begin; i < end; ++i) {
         prefix[i] = run;
         run += items_of(i);
     }
-    __syncthreads();
+    for (int i = n_live + tid; i <= n_seqs; i += kPrepThreads) prefix[i] = total;
+    if (tid == 0) {
+        hdr->n_items = total;
+        hdr->work_counter = 0;
+        hdr->status = 0;
+    }
     // tile_prefix[b] = number of 128-row tiles of sequences 0..b-1 (input order): same two-level scan
     auto tiles_of = [&](int b) -> uint32_t { return (uint32_t)((cu[b + 1] - cu[b] + kTile - 1) / kTile); };
     local = 0;
     for (int i = begin; i < end; ++i) local += tiles_of(i);
-    chunk_sum[tid] = local;
-    __syncthreads();
-    if (tid == 0) {
-        uint32_t acc = 0;
-        for (int i = 0; i < kPrepThreads; ++i) {
-            const uint32_t c = chunk_sum[i];
-            chunk_sum[i] = acc;
-            acc += c;
-        }
-        tile_prefix[n_seqs] = acc;
-    }
-    __syncthreads();
-    run = chunk_sum[tid];
+    run = block_exclusive_scan(local, scratch, &total);
     for (int i = begin; i < end; ++i) {
         tile_prefix[i] = run;
         run += tiles_of(i);
     }
+    for (int i = n_live + tid; i <= n_seqs; i += kPrepThreads) tile_prefix[i] = total;
 }
 
 int prep_launches(int32_t n_seqs, bool merge) { return (n_seqs > kPrepThreads ? 2 : 1) + (merge ? 1 : 0); }
@@ -195,7 +198,7 @@ cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total
         rank_kernel<<<(n_seqs + 255) / 256, 256, 0, stream>>>(cu, n_seqs, n_live, const_cast<int32_t*>(sched.order));
         if (cudaError_t e = cudaGetLastError()) return e;
     }
-    prep_kernel<<<1, kPrepThreads, 0, stream>>>(cu, n_seqs, rows_per_block, n_heads, sched.hdr,
+    prep_kernel<<<1, kPrepThreads, 0, stream>>>(cu, n_seqs, n_live, rows_per_block, n_heads, sched.hdr,
                                                 const_cast<int32_t*>(sched.order), const_cast<uint32_t*>(sched.prefix),
                                                 const_cast<uint32_t*>(sched.tile_prefix), ranked);
     return cudaGetLastError();
