@@ -1,7 +1,8 @@
 #!/usr/bin/env python
 """Benchmark of the packed variable-length attention hot path (plan -> forward -> backward).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload video|text|extreme|stream]
+    python bench.py [--gpus N] [--steps K] [--warmup W]
+                    [--workload video|text|extreme|stream|spatial2d|temporal2d]
     python bench.py --impl reference ...        # the fp64 CPU oracle on a bounded sample
 
 One step = one pass of the whole path over one synthetic batch: dcp_plan on the batch's lengths,
@@ -151,7 +152,7 @@ def run_ours(args):
     import torch.distributed as dist
     from paper_2608_07524_b200 import binding as B
     from paper_2608_07524_b200 import inputs
-    from paper_2608_07524_b200.stream import StreamRunner, plan_batch
+    from paper_2608_07524_b200.stream import MicroBatch, StreamRunner, plan_batch
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -164,10 +165,20 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
     B.lib()      # fail loudly here if libdcp.so is missing
 
+    axis = None
     if args.workload == "stream":
         batches = inputs.stream_batches()[: args.stream_batches]
         H, d, causal = 16, 128, False
         name = f"stream: {len(batches)} batches of the video length mix, Lambda={args.layers}, budget {args.budget_gb} GB"
+    elif args.workload in ("spatial2d", "temporal2d"):
+        # the paper's second architecture attends along one axis of a clip at a time: the planner sees the
+        # clips, the kernels see one sequence per latent frame (spatial) or per spatial position (temporal)
+        axis = args.workload[:-2]
+        clips = inputs.video_clips()
+        batches, H, d, causal = [[f * s for f, s in clips]], 16, 128, False
+        seqs = inputs.axis_lengths(clips, axis)
+        name = (f"config-3 clips, {axis} axis of a 2-D model: {len(seqs)} sequences of {min(seqs)}-{max(seqs)} tokens, "
+                f"{sum(seqs)} tokens, 16 heads, head_dim 128, bidirectional")
     else:
         w = workload(args.workload)
         lengths = [L for L in w.lengths if not args.drop_longer_than or L <= args.drop_longer_than]
@@ -179,12 +190,17 @@ def run_ours(args):
             name += f" (profiling subset: sequences longer than {args.drop_longer_than} dropped)"
     budget = int(args.budget_gb * 10 ** 9)
     max_tokens = max(sum(b) for b in batches)
-    max_seqs = max(len(b) for b in batches)
+    max_seqs = max(len(b) for b in batches) if axis is None else len(seqs)
     runner = StreamRunner(max_tokens, max_seqs, H, d, causal, dev, value_seed=12 + 100 * rank)
 
     def flops_of(lengths):
         f = 14.0 * sum(float(L) * L for L in lengths) * d * H
         return 0.5 * f if causal else f
+
+    def along_axis(mb):
+        if axis is None:
+            return mb
+        return MicroBatch(inputs.axis_lengths([inputs.clip_shape(L) for L in mb.lengths], axis), mb.recompute)
 
     profile, plan_kw = None, {}
     if args.plan == "profiled":
@@ -202,6 +218,7 @@ def run_ours(args):
         tokens, flops = 0, 0.0
         for lengths in batches:
             for mb in plan_batch(lengths, budget, H, d, n_layers=args.layers, **plan_kw):
+                mb = along_axis(mb)
                 tokens += runner.run_micro_batch(mb)
                 flops += flops_of(mb.lengths)
         return tokens, flops
@@ -301,6 +318,16 @@ def run_ours(args):
                 "traffic": (BWD_MAIN_DRAM_BYTES_PER_LAUNCH.get(args.workload)
                             if not args.drop_longer_than and args.layers == 1 else None),
                 "launches": bwd_n, "avg_launch_ms": bwd_ms / max(bwd_n, 1)}
+    if axis == "temporal" and bwd_n:
+        # sequences of 1-13 tokens: a tile pair does ~1 % useful arithmetic, the kernel is bound by HBM.
+        # Algorithmic bytes of the backward main kernel per (token, head): q, k, v, dO read and dk, dv
+        # written (6 d bf16), lse and D read (8), one fp32 dQ partial accumulated (4 d).
+        tok_per_launch = tokens_all / world / max(bwd_n, 1)
+        gbs = tok_per_launch * H * (6 * d * 2 + 8 + 4 * d) / (bwd_ms / bwd_n * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "attn_bwd_kernel (backward main)", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                    "peak_source": f"hbm_gbs of {peaks['source']} MEASURED_PEAKS.json", "traffic": None,
+                    "launches": bwd_n, "avg_launch_ms": bwd_ms / bwd_n}
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
@@ -333,7 +360,8 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="video", choices=["video", "text", "extreme", "stream"])
+    ap.add_argument("--workload", default="video",
+                    choices=["video", "text", "extreme", "stream", "spatial2d", "temporal2d"])
     ap.add_argument("--stream-batches", type=int, default=256)
     ap.add_argument("--layers", type=int, default=1, help="planner's layer count Lambda")
     ap.add_argument("--plan", default="model", choices=["model", "profiled"],

@@ -40,7 +40,7 @@ struct BwdParams {
 // With `bounds` non-null, short sequences are first merged into virtual sequences: sched.vcu and
 // `bounds` are written and the list is built over sched.vcu, which the later kernels must then be
 // given as their boundary array; with `bounds` null the list is built over cu_seqlens itself.
-int prep_launches(int32_t n_seqs, bool merge);   // kernels launch_prep enqueues (1 to 3)
+int prep_launches(int32_t n_seqs, bool merge);   // kernels launch_prep enqueues (1 to 4)
 cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen,
                         int32_t rows_per_block, int32_t n_heads, const SchedView& sched, uint16_t* bounds,
                         cudaStream_t stream);

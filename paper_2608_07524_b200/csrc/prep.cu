@@ -19,43 +19,44 @@ __device__ inline uint32_t block_exclusive_scan(uint32_t v, uint32_t* scratch, u
 // starts a virtual sequence iff it is not short, or its predecessor is not short, or the predecessor
 // starts in another window), so heads are found in parallel and compacted with a scan.
 // Outputs: vcu[0..n_v] = boundaries of the virtual sequences, vcu[n_v+1..n_seqs] = total_tokens
-// (empty padding, so that vcu is a valid boundary array of n_seqs sequences); hdr->n_vseq = n_v;
-// bounds[t] for every token t of an input sequence of at most 128 tokens = (first, end) position of
-// that sequence relative to its virtual sequence, one byte each.
+// (empty padding, so that vcu is a valid boundary array of n_seqs sequences); hdr->n_vseq = n_v.
+__device__ __forceinline__ bool merge_is_head(const int32_t* __restrict__ cu, int i, int32_t max_short) {
+    const int window = kTile + 1 - max_short;
+    return i == 0 || cu[i + 1] - cu[i] > max_short || cu[i] - cu[i - 1] > max_short || cu[i - 1] / window != cu[i] / window;
+}
+
 __global__ void __launch_bounds__(kPrepThreads) merge_kernel(const int32_t* __restrict__ cu, int32_t n_seqs,
                                                              int32_t total_tokens, int32_t max_short,
-                                                             WorkspaceHeader* hdr, int32_t* vcu, uint16_t* bounds) {
+                                                             WorkspaceHeader* hdr, int32_t* vcu) {
     __shared__ uint32_t scratch[33];
     const int tid = threadIdx.x;
-    const int window = kTile + 1 - max_short;
-    auto is_short = [&](int i) { return cu[i + 1] - cu[i] <= max_short; };
-    auto is_head = [&](int i) {
-        return i == 0 || !is_short(i) || !is_short(i - 1) || cu[i - 1] / window != cu[i] / window;
-    };
+    auto is_head = [&](int i) { return merge_is_head(cu, i, max_short); };
     const int per = (n_seqs + kPrepThreads - 1) / kPrepThreads;
     const int begin = min(tid * per, n_seqs), end = min(begin + per, n_seqs);
     uint32_t local = 0, n_v = 0;
     for (int i = begin; i < end; ++i) local += is_head(i) ? 1u : 0u;
     uint32_t run = block_exclusive_scan(local, scratch, &n_v);
     if (tid == 0) hdr->n_vseq = n_v;
-    int32_t vstart = 0;
-    if (begin < end && !is_head(begin)) {            // the virtual sequence began in an earlier chunk
-        int j = begin - 1;
-        while (!is_head(j)) --j;                     // at most 127 non-empty members: a virtual sequence has <= 128 tokens
-        vstart = cu[j];
-    }
-    for (int i = begin; i < end; ++i) {
-        const int32_t a = cu[i], b = cu[i + 1];
-        if (is_head(i)) {
-            vcu[run++] = a;
-            vstart = a;
-        }
-        if (b - a <= kTile) {
-            const uint16_t packed = (uint16_t)((a - vstart) | ((b - vstart) << 8));
-            for (int32_t t = a; t < b; ++t) bounds[t] = packed;
-        }
-    }
+    for (int i = begin; i < end; ++i)
+        if (is_head(i)) vcu[run++] = cu[i];
     for (uint32_t i = n_v + tid; i <= (uint32_t)n_seqs; i += kPrepThreads) vcu[i] = total_tokens;
+}
+
+// One thread per input sequence of at most 128 tokens, over as many CTAs as needed: bounds[t] for
+// each of its tokens t = (first, end) position of the sequence relative to the start of its virtual
+// sequence, one byte each.  The start is found by walking back to the head of the run (the head rule
+// is local, so this does not wait for merge_kernel's scan).
+__global__ void __launch_bounds__(256) bounds_kernel(const int32_t* __restrict__ cu, int32_t n_seqs, int32_t max_short,
+                                                     uint16_t* __restrict__ bounds) {
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= n_seqs) return;
+    const int32_t a = cu[i], b = cu[i + 1];
+    if (b == a || b - a > kTile) return;
+    int j = i;
+    while (!merge_is_head(cu, j, max_short)) --j;     // at most 127 non-empty members before i
+    const int32_t vstart = cu[j];
+    const uint16_t packed = (uint16_t)((a - vstart) | ((b - vstart) << 8));
+    for (int32_t t = a; t < b; ++t) bounds[t] = packed;
 }
 
 // Rank sort, one thread per sequence over as many CTAs as needed: order[] = sequence ids sorted by
@@ -178,7 +179,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __res
     for (int i = n_live + tid; i <= n_seqs; i += kPrepThreads) tile_prefix[i] = total;
 }
 
-int prep_launches(int32_t n_seqs, bool merge) { return (n_seqs > kPrepThreads ? 2 : 1) + (merge ? 1 : 0); }
+int prep_launches(int32_t n_seqs, bool merge) { return (n_seqs > kPrepThreads ? 2 : 1) + (merge ? 2 : 0); }
 
 cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen,
                         int32_t rows_per_block, int32_t n_heads, const SchedView& sched, uint16_t* bounds,
@@ -188,7 +189,9 @@ cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total
     if (bounds) {                                       // merge short sequences; everything below sees vcu
         const int32_t max_short = max_seqlen < kMergeMaxLen ? (max_seqlen > 0 ? max_seqlen : 1) : kMergeMaxLen;
         merge_kernel<<<1, kPrepThreads, 0, stream>>>(cu_seqlens, n_seqs, total_tokens, max_short, sched.hdr,
-                                                     const_cast<int32_t*>(sched.vcu), bounds);
+                                                     const_cast<int32_t*>(sched.vcu));
+        if (cudaError_t e = cudaGetLastError()) return e;
+        if (n_seqs > 0) bounds_kernel<<<(n_seqs + 255) / 256, 256, 0, stream>>>(cu_seqlens, n_seqs, max_short, bounds);
         if (cudaError_t e = cudaGetLastError()) return e;
         cu = sched.vcu;
         n_live = &sched.hdr->n_vseq;

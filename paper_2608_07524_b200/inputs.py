@@ -76,18 +76,37 @@ def video_lengths(n: int = 24, seed: int = 3) -> List[int]:
     return [_video_draw(g) for _ in range(n)]
 
 
-def short2d_lengths(axis: str, n: int = 24, seed: int = 3) -> List[int]:
-    """The config-3 clips as a 2-D model sees them (attention along one axis at a time): `spatial`
-    gives one sequence per latent frame (its tokens attend to each other), `temporal` one sequence
-    per spatial position (its frames attend to each other).  Both hold the same tokens in total."""
+def video_clips(n: int = 24, seed: int = 3):
+    """The config-3 draws as (latent frames, tokens per latent frame) pairs."""
     g = SplitMix64(seed)
-    out: List[int] = []
-    for _ in range(n):
-        f, s = _video_sample(g)
-        out += [s] * f if axis == "spatial" else [f] * s
+    return [_video_sample(g) for _ in range(n)]
+
+
+def clip_shape(length: int):
+    """(latent frames, tokens per frame) of a clip given its token count (the products are distinct)."""
+    for _, h, w in _RES:
+        for _, frames in _FRAMES:
+            f, s = -(-frames // 4), (h // 16) * (w // 16)
+            if f * s == length:
+                return f, s
+    raise ValueError(f"{length} is not a clip length of the video mix")
+
+
+def axis_lengths(clips, axis: str) -> List[int]:
+    """Sequences a 2-D model attends over (one axis at a time): `spatial` gives one sequence per
+    latent frame (its tokens attend to each other), `temporal` one sequence per spatial position
+    (its frames attend to each other).  Both hold the same tokens in total."""
     if axis not in ("spatial", "temporal"):
         raise ValueError("axis must be 'spatial' or 'temporal'")
+    out: List[int] = []
+    for f, s in clips:
+        out += [s] * f if axis == "spatial" else [f] * s
     return out
+
+
+def short2d_lengths(axis: str, n: int = 24, seed: int = 3) -> List[int]:
+    """axis_lengths of the config-3 clips."""
+    return axis_lengths(video_clips(n, seed), axis)
 
 
 def extreme_lengths(n_short: int = 64, seed: int = 4, long_len: int = 131072) -> List[int]:

@@ -210,7 +210,7 @@ def test_launch_counter_and_profile():
     B.dcp_profile_read()
     before = B.dcp_launch_count()
     run_gpu(q, k, v, g, w.cu_seqlens, False)
-    assert B.dcp_launch_count() - before == 3 + 5          # forward: merge + prep + main; backward: merge + prep + 3
+    assert B.dcp_launch_count() - before == 4 + 6          # forward: merge + bounds + prep + main; backward: those + 3
     prof = B.dcp_profile_read()
     B.dcp_profile_enable(False)
     assert prof["fwd"][1] == 1 and prof["bwd_main"][1] == 1 and prof["prep"][1] == 2

@@ -1,5 +1,6 @@
-"""Full-size benchmark configurations (2 text, 3 video, 4 extreme imbalance) in the launch
-configuration the benchmark times.  A full fp64 evaluation of these is 10^13-10^14 flop, so the
+"""Full-size benchmark configurations (2 text, 3 video, 4 extreme imbalance, and the video clips
+seen along the spatial axis of a 2-D model) in the launch configuration the benchmark times; the
+temporal axis (20384 sequences of 1-13 tokens) is small enough for the oracle to check in full.  A full fp64 evaluation of these is 10^13-10^14 flop, so the
 oracle checks (a) sampled query rows (O, lse, dQ) and key columns (dK, dV), which the definition
 lets it compute one by one, (b) the shortest sequences completely, on every head, and (c) two
 whole-tensor identities that hold at any size:
@@ -39,9 +40,15 @@ def sample_positions(L, rng, n_random=24):
     return np.array(sorted(pos), np.int32)
 
 
-@pytest.fixture(scope="module", params=[2, 3, 4])
+def workload_of(param):
+    if isinstance(param, int):
+        return inputs.config(param)
+    return inputs.Workload(param, inputs.short2d_lengths(param[:-2]), 16, 128, False, 12)
+
+
+@pytest.fixture(scope="module", params=[2, 3, 4, "spatial2d"])
 def full_run(request):
-    w = inputs.config(request.param)
+    w = workload_of(request.param)
     dev = "cuda"
     q, k, v, g = inputs.make_qkvg_device(w.total_tokens, w.n_heads, w.head_dim, w.value_seed, dev)
     cud = torch.tensor(w.cu_seqlens, dtype=torch.int32, device=dev)
@@ -115,3 +122,23 @@ def test_whole_tensor_identities(full_run):
         bound = 8 * EPS_BF16 * torch.sqrt((dvs * dvs).sum(dim=0)) + ACC_BIAS * dvs.abs().sum(dim=0) + 1e-6
         assert bool(((lhs - rhs).abs() <= bound).all()), f"sum dV vs sum dO on sequence {seq}"
     assert bool(torch.isfinite(o.float()).all()) and bool(torch.isfinite(lse).all())
+
+
+def test_temporal_axis_in_full():
+    """Thousands of 1-13 token sequences, merged by the work-list kernels into tiles of up to 128
+    tokens: every output element against the oracle."""
+    w = workload_of("temporal2d")
+    q, k, v, g = inputs.make_qkvg_device(w.total_tokens, w.n_heads, w.head_dim, w.value_seed, "cuda")
+    cud = torch.tensor(w.cu_seqlens, dtype=torch.int32, device="cuda")
+    ws = B.alloc_workspace(w.total_tokens, len(w.lengths), w.n_heads, w.head_dim, True, "cuda")
+    o, lse = B.dcp_varlen_attn_fwd(q, k, v, cud, w.max_seqlen, w.causal, workspace=ws)
+    dq, dk, dv = B.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cud, w.max_seqlen, w.causal, workspace=ws)
+    B.dcp_query_status(ws)
+    qc, kc, vc, gc = (x.cpu() for x in (q, k, v, g))
+    O, Lse = oracle.attn_fwd(qc, kc, vc, w.cu_seqlens, w.causal)
+    rdq, rdk, rdv = oracle.attn_bwd(qc, kc, vc, gc, w.cu_seqlens, w.causal)
+    close("o", o, O)
+    close("dq", dq, rdq)
+    close("dk", dk, rdk)
+    close("dv", dv, rdv)
+    assert float(np.max(np.abs(lse.double().cpu().numpy() - Lse))) <= LSE_ABS

@@ -46,3 +46,19 @@ def test_flop_convention():
     assert abs(w.fwd_flops() / 1e12 - 22.785) < 0.01 and abs(w.fwd_bwd_flops() / 1e12 - 79.748) < 0.03
     w = inputs.config(2)
     assert abs(w.fwd_bwd_flops() / 1e12 - 4.086) < 0.01
+
+
+def test_two_dimensional_views_of_the_video_clips():
+    clips = inputs.video_clips()
+    assert [f * s for f, s in clips] == inputs.video_lengths()
+    assert all(inputs.clip_shape(f * s) == (f, s) for f, s in clips)
+    spatial, temporal = inputs.short2d_lengths("spatial"), inputs.short2d_lengths("temporal")
+    assert sum(spatial) == sum(temporal) == sum(inputs.video_lengths()) == 124992
+    assert len(spatial) == sum(f for f, _ in clips) == 121 and set(spatial) == {256, 1200, 3600}
+    assert len(temporal) == sum(s for _, s in clips) == 20384 and set(temporal) == {1, 4, 8, 13}
+    assert inputs.axis_lengths([(2, 3)], "spatial") == [3, 3] and inputs.axis_lengths([(2, 3)], "temporal") == [2, 2, 2]
+    import pytest
+    with pytest.raises(ValueError):
+        inputs.clip_shape(777)
+    with pytest.raises(ValueError):
+        inputs.axis_lengths(clips, "diagonal")
