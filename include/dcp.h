@@ -80,6 +80,33 @@ int dcp_plan_profiled(const int32_t* lengths, const int64_t* fwd_time, int32_t n
                       const dcp_plan_params* params, int32_t* mb_id, int32_t* n_mb, int32_t* recompute,
                       int64_t* cost);
 
+/* DCP-intra: batch size, sequence-parallel size and recompute count for one sequence length.
+ *
+ * Paper: Section 3.4, Eq. 4-6 and Algorithm 1.  Each candidate (b, p) carries what the dual-layer
+ * profile (Section 3.5) gives with EVERY layer recomputed: the forward time t_f of one layer, the
+ * activation bytes m one layer keeps when it is not recomputed, the iteration time T_(b,p) and the
+ * memory M_(b,p).  Letting `keep` layers keep their activations costs keep*m bytes and saves
+ * keep*t_f, so per candidate keep = min(Lambda, floor((capacity - M_(b,p)) / m)), the recompute count
+ * is r = Lambda - keep (the smallest that fits) and the time T_(b,p) - keep*t_f.  The listing's loop
+ * stops at the first count that fits; it is read as "the largest count that still fits", which is
+ * what its comment and the text say.  Among candidates the one with the highest throughput
+ * b / (p * time) wins (Eq. 1; the text says throughput, the listing compares times, which is the
+ * same when b and p are equal).  Ties: smaller p, then larger b, then the earlier candidate.
+ * Candidates with M_(b,p) > capacity are skipped; none left => DCP_ERR_INFEASIBLE.
+ * Host pointers; outputs *best (index), *recompute (r), time (nullable).  On one GPU every p is 1;
+ * the function itself does not touch a device. */
+typedef struct {
+    int32_t batch_size; /* b >= 1 */
+    int32_t sp_size;    /* p >= 1 */
+    int64_t t_f;        /* >= 0, any integer time unit */
+    int64_t m;          /* >= 0, bytes */
+    int64_t time_full;  /* T_(b,p) >= 1, same unit as t_f */
+    int64_t mem_full;   /* M_(b,p) >= 0, bytes */
+} dcp_intra_candidate;
+
+int dcp_intra_select(const dcp_intra_candidate* cands, int32_t n, int64_t mem_capacity, int32_t n_layers,
+                     int32_t* best, int32_t* recompute, int64_t* time);
+
 /* DCP-inter: accumulation-step counts that balance n batches running side by side.
  *
  * Paper: Section 3.3, Eq. 3, and Appendix C (G_min, G_max).  Batch i takes times[i] (any positive

@@ -220,3 +220,6 @@ def inter_bruteforce(times, g_min: int = 1, g_max: int = 4):
     if rc:
         raise ValueError(f"oracle_inter_bruteforce rejected its arguments or the space is too large ({rc})")
     return g[:n].tolist(), (hi.value << 64) | lo.value
+
+
+from .intra_oracle import intra_select  # noqa: E402,F401  (Algorithm 1, plain Python)

@@ -31,6 +31,11 @@ class PlanParams(ctypes.Structure):
                 ("const_bytes", ctypes.c_int64), ("fixed_cost", ctypes.c_int64)]
 
 
+class IntraCandidate(ctypes.Structure):
+    _fields_ = [("batch_size", ctypes.c_int32), ("sp_size", ctypes.c_int32), ("t_f", ctypes.c_int64),
+                ("m", ctypes.c_int64), ("time_full", ctypes.c_int64), ("mem_full", ctypes.c_int64)]
+
+
 def lib():
     """The loaded library.  Raises if libdcp.so has not been built (python -m paper_2608_07524_b200.build)."""
     global _lib
@@ -52,6 +57,8 @@ def lib():
                                             ctypes.POINTER(ctypes.c_int64)]
             L.dcp_plan_profiled.restype = ctypes.c_int
             L.dcp_inter_plan.argtypes = [i64p, i32, i32, i32, i32p, i64p, i64p]
+            L.dcp_intra_select.argtypes = [ctypes.POINTER(IntraCandidate), i32, i64, i32, i32p, i32p, i64p]
+            L.dcp_intra_select.restype = ctypes.c_int
             L.dcp_inter_plan.restype = ctypes.c_int
             L.dcp_varlen_attn_workspace.argtypes = [i32, i32, i32, i32, szp, szp]
             L.dcp_varlen_attn_workspace.restype = ctypes.c_int
@@ -145,6 +152,17 @@ def dcp_inter_plan(times, g_min: int = 1, g_max: int = 4) -> Tuple[List[int], in
     idle, it = ctypes.c_int64(0), ctypes.c_int64(0)
     _check(lib().dcp_inter_plan(arr, n, int(g_min), int(g_max), g, ctypes.byref(idle), ctypes.byref(it)))
     return list(g[:n]), int(idle.value), int(it.value)
+
+
+def dcp_intra_select(candidates, mem_capacity: int, n_layers: int) -> Tuple[int, int, int]:
+    """(index, recompute, time) of the throughput-optimal candidate (Algorithm 1).  Each candidate is
+    (batch_size, sp_size, t_f, m, time_full, mem_full), profiled with every layer recomputed."""
+    n = len(candidates)
+    arr = (IntraCandidate * max(n, 1))(*[IntraCandidate(*[int(x) for x in c]) for c in candidates])
+    best, rec, t = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int64(0)
+    _check(lib().dcp_intra_select(arr, n, int(mem_capacity), int(n_layers), ctypes.byref(best), ctypes.byref(rec),
+                                  ctypes.byref(t)))
+    return int(best.value), int(rec.value), int(t.value)
 
 
 def dcp_varlen_attn_workspace(total_tokens: int, n_seqs: int, n_heads: int, head_dim: int) -> Tuple[int, int]:
