@@ -326,7 +326,8 @@ def run_ours(args):
         gbs = tok_per_launch * H * (6 * d * 2 + 8 + 4 * d) / (bwd_ms / bwd_n * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": "attn_bwd_kernel (backward main)", "achieved": gbs, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
-                    "peak_source": f"hbm_gbs of {peaks['source']} MEASURED_PEAKS.json", "traffic": None,
+                    "peak_source": f"hbm_gbs of {peaks['source']} MEASURED_PEAKS.json",
+                    "traffic": 5.293e9,        # ncu, one launch of this workload (profiles/attn_fwd_bwd_temporal2d.md)
                     "launches": bwd_n, "avg_launch_ms": bwd_ms / bwd_n}
 
     cpu_baseline = None
