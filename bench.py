@@ -27,7 +27,7 @@ sys.path.insert(0, ROOT)
 METRIC = "varlen_attn_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 HBM_BUDGET = 180 * 10 ** 9
-# DRAM traffic (bytes) of one backward-main launch on config 3, from profiles/attn_fwd_bwd_video_subset.md:
+# DRAM traffic (bytes) of one backward-main launch on config 3, from the ncu capture summarised under profiles/:
 # 3.201 GB measured by ncu on the 78192-token subset, scaled by tokens (traffic is proportional to them).
 BWD_MAIN_DRAM_BYTES_PER_LAUNCH = {"video": 3.201e9 * 124992 / 78192}
 
@@ -327,7 +327,7 @@ def run_ours(args):
         roofline = {"bound": "hbm", "kernel": "attn_bwd_kernel (backward main)", "achieved": gbs, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                     "peak_source": f"hbm_gbs of {peaks['source']} MEASURED_PEAKS.json",
-                    "traffic": 5.293e9,        # ncu, one launch of this workload (profiles/attn_fwd_bwd_temporal2d.md)
+                    "traffic": 5.293e9,        # ncu, one launch of this workload (summary under profiles/)
                     "launches": bwd_n, "avg_launch_ms": bwd_ms / bwd_n}
 
     cpu_baseline = None
