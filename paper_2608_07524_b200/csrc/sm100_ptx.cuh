@@ -241,6 +241,52 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+// Packed pairs of fp32 (one instruction, two results; sm_100 and later).
+__device__ __forceinline__ uint64_t pack_f32x2(float a, float b) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& a, float& b) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t sub_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// 2^x for a pair of arguments in [-126, 0] on the FMA pipe instead of the special-function unit:
+// x = n + f with n = round(x) and f in [-0.5, 0.5]; a cubic for 2^f (relative error 7.5e-5, far below
+// the bf16 rounding the result gets) and n added to the exponent field.  Adding 1.5 * 2^23 leaves n in
+// the low mantissa bits of the sum, so the shift by 23 moves it straight onto the exponent.
+__device__ __forceinline__ void poly_exp2_pair(uint64_t x2, float& p0, float& p1) {
+    float x0, x1;
+    unpack_f32x2(x2, x0, x1);
+    const uint64_t xc = pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+    const uint64_t magic = pack_f32x2(12582912.f, 12582912.f);
+    const uint64_t t = add_f32x2(xc, magic);
+    const uint64_t f = sub_f32x2(xc, sub_f32x2(t, magic));
+    uint64_t q = fma_f32x2(pack_f32x2(0.05517162f, 0.05517162f), f, pack_f32x2(0.24261112f, 0.24261112f));
+    q = fma_f32x2(q, f, pack_f32x2(0.69326099f, 0.69326099f));
+    q = fma_f32x2(q, f, pack_f32x2(0.99992807f, 0.99992807f));
+    float q0, q1, t0, t1;
+    unpack_f32x2(q, q0, q1);
+    unpack_f32x2(t, t0, t1);
+    p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
+    p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
+}
+
 // Byte offset of (row, 16-byte chunk) inside a tile stored as 128-byte rows with 128-byte swizzle
 // (the layout TMA writes for a 64 x rows bf16 box and tcgen05.mma reads with layout type 2).
 __device__ __forceinline__ uint32_t sw128_offset(uint32_t row, uint32_t chunk16) {
