@@ -424,13 +424,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     for (int c = 0; c < 128; ++c)
                         if (c >= n_valid) s[c] = 0xff800000u;         // -inf
                 }
-                float part[8];      // eight independent chains instead of one 128-long one
+                float part[8];      // eight independent chains instead of one 128-long one, three-input maxima
 #pragma unroll
-                for (int c = 0; c < 8; ++c) part[c] = __uint_as_float(s[c]);
+                for (int c = 0; c < 8; ++c) part[c] = fmax3(__uint_as_float(s[c]), __uint_as_float(s[8 + c]), __uint_as_float(s[16 + c]));
 #pragma unroll
-                for (int c = 8; c < 128; ++c) part[c & 7] = fmaxf(part[c & 7], __uint_as_float(s[c]));
-                const float mx = fmaxf(fmaxf(fmaxf(part[0], part[1]), fmaxf(part[2], part[3])),
-                                       fmaxf(fmaxf(part[4], part[5]), fmaxf(part[6], part[7])));
+                for (int c = 24; c < 120; c += 16) {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        part[u] = fmax3(part[u], __uint_as_float(s[c + u]), __uint_as_float(s[c + 8 + u]));
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) part[u] = fmaxf(part[u], __uint_as_float(s[120 + u]));
+                const float mx = fmaxf(fmax3(part[0], part[1], part[2]), fmax3(fmax3(part[3], part[4], part[5]), part[6], part[7]));
 
                 const bool need = (mx - m) * p.scale_log2 > kRescaleThreshold;
                 if (__any_sync(0xffffffffu, need)) {

@@ -241,6 +241,13 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+// Maximum of three (one instruction on sm_100 and later).
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 // Packed pairs of fp32 (one instruction, two results; sm_100 and later).
 __device__ __forceinline__ uint64_t pack_f32x2(float a, float b) {
     uint64_t r;
