@@ -25,9 +25,11 @@
 // These 64 KB per (Q tile, K tile) pair are what bounds the kernel: the SM's path to L2 moves about
 // 15-25 bytes per clock for reductions, per-thread atomics and shared-memory bulk reductions alike,
 // and the atomics share the load/store unit with the compute warps' dS^T stores; with the atomics
-// compiled out the same kernel runs a third faster.  Measured and rejected: pacing the atomics,
-// bulk reductions from a 16 KB staging buffer, atomics into an L2-hot block (same time, so the
-// limit is on the SM's side), dK before dQ, and staggering the Q walk of neighbouring key blocks.
+// compiled out the same kernel runs a third faster.  What helps is pausing the drain warps briefly
+// between groups of atomics (see kRedGroup).  Measured and rejected: pacing by spinning on the clock
+// (the spin takes issue slots from the compute warps), bulk reductions from a 16 KB staging buffer,
+// atomics into an L2-hot block (same time, so the limit is on the SM's side), dK before dQ, and
+// staggering the Q walk of neighbouring key blocks.
 // dK and dV stay in tensor memory for the whole item and are written once (dK scaled by the
 // softmax scale).
 //
@@ -67,6 +69,13 @@ extern "C" int dcp_debug_read_timing(long long* out) {
 
 namespace dcp {
 
+// The drain warps pause after every kRedGroup vector atomics.  Issued back to back, a tile's 64 KB
+// of atomics fill the SM's queue towards L2, and the TMA requests and shared-memory stores of the
+// other warps wait behind them; a short sleep (which, unlike a spin on the clock, takes no issue
+// slots) lets those through.  Backward main kernel on config 3: 60.2 ms without, 58.3 with 4 / 200 ns
+// (150-250 ns alike; 100 ns no effect; 400 ns 75.6 ms); config 4: 100.0 -> 93.7 ms.
+constexpr int kRedGroup = 4;
+constexpr unsigned kRedSleepNs = 200;
 constexpr int kBwdThreads = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -631,11 +640,14 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.dq_free);
-                if (qrow < w.len) {
+                {
+                    const bool live = qrow < w.len;
 #pragma unroll
-                    for (int c = 0; c < D / 4; ++c)
-                        red_add_v4(dst + c * (kTile * 4), __uint_as_float(acc[c * 4]), __uint_as_float(acc[c * 4 + 1]),
+                    for (int c = 0; c < D / 4; ++c) {
+                        if (live) red_add_v4(dst + c * (kTile * 4), __uint_as_float(acc[c * 4]), __uint_as_float(acc[c * 4 + 1]),
                                    __uint_as_float(acc[c * 4 + 2]), __uint_as_float(acc[c * 4 + 3]));
+                        if ((c % kRedGroup) == kRedGroup - 1) __nanosleep(kRedSleepNs);
+                    }
                 }
             }
         }
