@@ -69,13 +69,17 @@ extern "C" int dcp_debug_read_timing(long long* out) {
 
 namespace dcp {
 
-// The drain warps pause after every kRedGroup vector atomics.  Issued back to back, a tile's 64 KB
-// of atomics fill the SM's queue towards L2, and the TMA requests and shared-memory stores of the
-// other warps wait behind them; a short sleep (which, unlike a spin on the clock, takes no issue
-// slots) lets those through.  Backward main kernel on config 3: 60.2 ms without, 58.3 with 4 / 200 ns
-// (150-250 ns alike; 100 ns no effect; 400 ns 75.6 ms); config 4: 100.0 -> 93.7 ms.
+// The drain warps pause after every kRedGroup vector atomics, and warp k of the four starts k pauses
+// late.  Issued back to back, a tile's 64 KB of atomics fill the SM's queue towards L2, and the TMA
+// requests and shared-memory stores of the other warps wait behind them; short sleeps (which, unlike
+// a spin on the clock, take no issue slots) let those through.  __nanosleep rounds down to steps of
+// about 128 ns here (100 ns had no effect, 150-250 ns the same effect), so the values sit in the
+// middle of a step.  Backward main kernel alone on config 3: 60.2 ms without any pause, 58.3 with the
+// pauses, 55.8 with the stagger as well; two steps per pause or per stagger, or a pause after every
+// second atomic, cost 57-85 ms.  In the power-capped bench loop: 61.7 -> 58.1 ms.
 constexpr int kRedGroup = 4;
-constexpr unsigned kRedSleepNs = 200;
+constexpr unsigned kRedSleepNs = 192;        // one step
+constexpr unsigned kRedStaggerNs = 128;      // per drain warp, plus half a step
 constexpr int kBwdThreads = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -642,6 +646,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 if (lane == 0) mbar_arrive(&sh.dq_free);
                 {
                     const bool live = qrow < w.len;
+                    if ((warp & 3) > 0) __nanosleep((warp & 3) * kRedStaggerNs + 64);
 #pragma unroll
                     for (int c = 0; c < D / 4; ++c) {
                         if (live) red_add_v4(dst + c * (kTile * 4), __uint_as_float(acc[c * 4]), __uint_as_float(acc[c * 4 + 1]),
