@@ -135,7 +135,9 @@ int dcp_inter_plan(const int64_t* times, int32_t n, int32_t g_min, int32_t g_max
  * 1/sqrt(head_dim).  Zero-length sequences are legal.  max_seqlen must be >= every length.
  */
 
-/* Bytes of caller-provided device workspace needed by the forward and the backward call. */
+/* Bytes of caller-provided device workspace needed by the forward and the backward call: the work
+ * list (per sequence), a 2-byte-per-token table used when runs of short sequences share a tile, and for
+ * the backward the per-row statistics and the fp32 dQ accumulator (per 128-row tile and head). */
 int dcp_varlen_attn_workspace(int32_t total_tokens, int32_t n_seqs, int32_t n_heads, int32_t head_dim,
                               size_t* fwd_bytes, size_t* bwd_bytes);
 
@@ -161,8 +163,11 @@ int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, const void*
  * real-time loop, a plug-in handed fixed buffers by its host program, a process whose allocator is
  * locked down after start-up).  Same operation, arguments, layouts and error codes as
  * dcp_varlen_attn_fwd, but the work-list scratch is a fixed array inside the library's device
- * image (about 50 KB, held by every GPU that loads the library until the process exits) instead of
+ * image (about 66 KB, held by every GPU that loads the library until the process exits) instead of
  * a caller buffer.  Limits and rules:
+ *   - runs of very short sequences are not merged into shared tiles here (the table that needs grows
+ *     with the token count), so such batches run slower than through dcp_varlen_attn_fwd; results
+ *     are the same;
  *   - n_seqs <= DCP_NOALLOC_MAX_SEQS, else DCP_ERR_UNSUPPORTED and nothing is enqueued;
  *   - the call allocates nothing on the device and frees nothing;
  *   - the first call on each device looks up the array's device address (a synchronous runtime
