@@ -152,7 +152,7 @@ def run_ours(args):
     import torch.distributed as dist
     from paper_2608_07524_b200 import binding as B
     from paper_2608_07524_b200 import inputs
-    from paper_2608_07524_b200.stream import MicroBatch, StreamRunner, plan_batch
+    from paper_2608_07524_b200.stream import HostPipeline, MicroBatch, StreamRunner, plan_batch
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -299,41 +299,11 @@ def run_ours(args):
         # same way).  Every step's inputs still cross PCIe and every step's results are read back; the
         # timed region includes filling and draining the pipeline.
         runners = [runner, StreamRunner(max_tokens, max_seqs, H, d, causal, dev, value_seed=13 + 100 * rank)]
-        host_out2 = [torch.empty((T, H, d), dtype=torch.bfloat16).pin_memory() for _ in range(4)]
-        host_lse2 = torch.empty((H * T,), dtype=torch.float32).pin_memory()
-        outs = [(host_out, host_lse), (host_out2, host_lse2)]
-        s_comp, s_in, s_out = torch.cuda.current_stream(), torch.cuda.Stream(), torch.cuda.Stream()
+        pipe = HostPipeline(runners, T)
         n_pipe = 2 * n_e2e
 
         def pipeline(n):
-            ev_comp, ev_out = [], []
-            for i in range(n):
-                r = runners[i & 1]
-                with torch.cuda.stream(s_in):
-                    if i >= 2:
-                        s_in.wait_event(ev_comp[i - 2])          # that set's inputs are no longer being read
-                    for hbuf, dbuf in zip(host_in, (r.q, r.k, r.v, r.g)):
-                        dbuf[:T].copy_(hbuf, non_blocking=True)
-                    ev_in = torch.cuda.Event()
-                    ev_in.record(s_in)
-                s_comp.wait_event(ev_in)
-                if i >= 2:
-                    s_comp.wait_event(ev_out[i - 2])             # that set's results have left
-                step(r)
-                ev = torch.cuda.Event()
-                ev.record(s_comp)
-                ev_comp.append(ev)
-                with torch.cuda.stream(s_out):
-                    s_out.wait_event(ev)
-                    ho, hl = outs[i & 1]
-                    for hbuf, dbuf in zip(ho, (r.o, r.dq, r.dk, r.dv)):
-                        hbuf.copy_(dbuf[:T], non_blocking=True)
-                    hl.copy_(r.lse[: H * T], non_blocking=True)
-                    ev = torch.cuda.Event()
-                    ev.record(s_out)
-                    ev_out.append(ev)
-            for ev in ev_out[-2:]:
-                s_comp.wait_event(ev)
+            pipe.run(host_in, step, n)
 
         pipeline(2)
         barrier()
@@ -355,7 +325,7 @@ def run_ours(args):
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_pipe,
                "how": "two sets of device buffers, copies and compute on three streams",
                "one_stream_value": per_step_flops * n_e2e / (float(serial_ms.item()) * 1e-3) / 1e12}
-        del runners, host_out2, host_lse2
+        del runners, pipe
         del host_in, host_out, host_lse
 
     if rank != 0:

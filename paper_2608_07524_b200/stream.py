@@ -98,3 +98,62 @@ class StreamRunner:
 
     def check(self):
         binding.dcp_query_status(self.ws)
+
+
+class HostPipeline:
+    """Steps whose inputs live in pinned host memory and whose results go back to it.
+
+    Two StreamRunners (two sets of device buffers) and three streams: while step i computes, the
+    inputs of step i+1 cross to the device and the results of step i-1 cross back, the way a
+    training loop prefetches its next batch.  Every step's q, k, v, dO are copied in and its o, lse,
+    dq, dk, dv are copied out; only the overlap is added.
+    """
+
+    def __init__(self, runners: Sequence[StreamRunner], tokens: int):
+        import torch
+        self.torch = torch
+        self.runners = list(runners)
+        if len(self.runners) != 2:
+            raise ValueError("the pipeline alternates between exactly two runners")
+        r = self.runners[0]
+        self.T, self.H = tokens, r.H
+        shape = (tokens, r.H, r.d)
+        self.host_out = [[torch.empty(shape, dtype=torch.bfloat16).pin_memory() for _ in range(4)] for _ in range(2)]
+        self.host_lse = [torch.empty((r.H * tokens,), dtype=torch.float32).pin_memory() for _ in range(2)]
+        self.s_in, self.s_out = torch.cuda.Stream(), torch.cuda.Stream()
+
+    def run(self, host_in, step_fn, n_steps: int):
+        """host_in: pinned q, k, v, dO.  step_fn(runner) enqueues one step's kernels on the current
+        stream.  Returns when everything is enqueued; the current stream ends up waiting for the
+        last results to reach the host buffers."""
+        torch = self.torch
+        T, H = self.T, self.H
+        s_comp = torch.cuda.current_stream()
+        ev_comp, ev_out = [], []
+        for i in range(n_steps):
+            r = self.runners[i & 1]
+            with torch.cuda.stream(self.s_in):
+                if i >= 2:
+                    self.s_in.wait_event(ev_comp[i - 2])         # that set's inputs are no longer being read
+                for hbuf, dbuf in zip(host_in, (r.q, r.k, r.v, r.g)):
+                    dbuf[:T].copy_(hbuf, non_blocking=True)
+                ev_in = torch.cuda.Event()
+                ev_in.record(self.s_in)
+            s_comp.wait_event(ev_in)
+            if i >= 2:
+                s_comp.wait_event(ev_out[i - 2])                 # that set's results have left
+            step_fn(r)
+            ev = torch.cuda.Event()
+            ev.record(s_comp)
+            ev_comp.append(ev)
+            with torch.cuda.stream(self.s_out):
+                self.s_out.wait_event(ev)
+                for hbuf, dbuf in zip(self.host_out[i & 1], (r.o, r.dq, r.dk, r.dv)):
+                    hbuf.copy_(dbuf[:T], non_blocking=True)
+                self.host_lse[i & 1].copy_(r.lse[: H * T], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(self.s_out)
+                ev_out.append(ev)
+        for ev in ev_out[-2:]:
+            s_comp.wait_event(ev)
+
