@@ -293,6 +293,7 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
     p.bounds = bounds;
     p.stats = stats;
     p.dq_acc = dq_acc;
+    p.dq = static_cast<__nv_bfloat16*>(dq);
     p.dk = static_cast<__nv_bfloat16*>(dk);
     p.dv = static_cast<__nv_bfloat16*>(dv);
     p.sched = sched;

@@ -644,7 +644,21 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.dq_free);
-                {
+                if (w.len <= kTile) {
+                    // the sequence's only tile pair: this is the whole dQ, no accumulation needed
+                    if (qrow < w.len) {
+                        __nv_bfloat16* out = p.dq + (((size_t)w.tok0 + qrow) * p.n_heads + w.head) * D;
+#pragma unroll
+                        for (int c = 0; c < D / 8; ++c) {
+                            uint4 val;
+                            val.x = pack_bf16x2(__uint_as_float(acc[c * 8 + 0]) * p.scale, __uint_as_float(acc[c * 8 + 1]) * p.scale);
+                            val.y = pack_bf16x2(__uint_as_float(acc[c * 8 + 2]) * p.scale, __uint_as_float(acc[c * 8 + 3]) * p.scale);
+                            val.z = pack_bf16x2(__uint_as_float(acc[c * 8 + 4]) * p.scale, __uint_as_float(acc[c * 8 + 5]) * p.scale);
+                            val.w = pack_bf16x2(__uint_as_float(acc[c * 8 + 6]) * p.scale, __uint_as_float(acc[c * 8 + 7]) * p.scale);
+                            *reinterpret_cast<uint4*>(out + c * 8) = val;
+                        }
+                    }
+                } else {
                     const bool live = qrow < w.len;
                     if ((warp & 3) > 0) __nanosleep((warp & 3) * kRedStaggerNs + 64);
 #pragma unroll

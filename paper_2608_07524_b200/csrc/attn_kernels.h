@@ -27,6 +27,7 @@ struct BwdParams {
                                   // columns 0-2 = -lse/scale split in three bf16 parts, 8-10 = -D likewise
                                   // (D_i = sum_c dO_ic O_ic); rows past the sequence end hold -1e30 and 0
     float* dq_acc;        // fp32, tile-blocked: [tile][head][d/4][128 rows][4]; zeroed before the main kernel
+    __nv_bfloat16* dq;    // final dQ: written directly for sequences of a single tile, by the post kernel otherwise
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
     SchedView sched;

@@ -234,6 +234,13 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
         while (lo + 1 < n_seqs && tile_prefix[lo + 1] <= t) ++lo;   // skip empty sequences
         const int row0 = (int)(t - tile_prefix[lo]) * kTile;
         const int len = cu[lo + 1] - cu[lo];
+        if (len > kTile) {
+            // this (tile, head) block of the dQ accumulator; a sequence of a single tile needs none (its
+            // one tile pair yields the whole dQ, which the main kernel writes directly)
+            float4* acc_blk = reinterpret_cast<float4*>(dq_acc) + (size_t)blk * (kTile * D / 4);
+            if ((size_t)(blk + 1) * (kTile * D / 4) <= dq_acc_vec4)
+                for (int e = threadIdx.x; e < kTile * D / 4; e += blockDim.x) acc_blk[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         {
         uint8_t* out = reinterpret_cast<uint8_t*>(stats) + ((size_t)t * n_heads + h) * (kTile * 16 * 2);
         // a warp takes rows warp, warp+8, ...; four rows per pass so that eight loads are in flight per lane
@@ -295,12 +302,6 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
         }
         }
     }
-    // only the tiles in use: the workspace is sized for an upper bound on the tile count
-    const size_t used_vec4 = (size_t)n_blocks * (size_t)(kTile * D / 4);
-    if (used_vec4 < dq_acc_vec4) dq_acc_vec4 = used_vec4;
-    const size_t stride = (size_t)gridDim.x * blockDim.x;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < dq_acc_vec4; i += stride)
-        reinterpret_cast<float4*>(dq_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
 cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, const float* lse, const int32_t* cu_seqlens,
@@ -338,6 +339,7 @@ __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__
         const int row0 = (int)(t - tile_prefix[lo]) * kTile;
         const int len = cu[lo + 1] - cu[lo];
         const int rows = min(kTile, len - row0);
+        if (len <= kTile) continue;       // a single tile pair: the main kernel has written dq itself
         {
         const float4* src = reinterpret_cast<const float4*>(dq_acc + ((size_t)t * n_heads + h) * (kTile * D));
         for (int e = threadIdx.x; e < kTile * D / 4; e += blockDim.x) {
