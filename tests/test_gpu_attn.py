@@ -239,3 +239,19 @@ def test_host_pipeline_matches_direct_run():
         assert torch.equal(ho, o) and torch.equal(hdk, dk) and torch.equal(hdv, dv)
         assert float((hdq.float() - dq.float()).abs().max()) <= 2e-2
         assert torch.equal(pipe.host_lse[s].view(H, T), lse)
+
+
+@pytest.mark.parametrize("seed", list(range(12)))
+def test_random_length_mixes(seed):
+    """Random mixes of empty, tiny, sub-tile, tile-edge and multi-tile sequences: exercises every way
+    short runs can be merged and broken up next to sequences that are not merged."""
+    rng = np.random.default_rng(1000 + seed)
+    pools = [[0], [1, 2, 3, 5, 8, 13], list(range(14, 65)), [63, 64, 65, 66], list(range(67, 128)), [127, 128, 129, 130],
+             [200, 256, 257, 300, 511, 640]]
+    weights = np.array([1, 6, 3, 2, 2, 2, 1.5])
+    n = int(rng.integers(3, 60))
+    lengths = [int(rng.choice(pools[int(rng.choice(len(pools), p=weights / weights.sum()))])) for _ in range(n)]
+    if sum(lengths) == 0:
+        lengths.append(7)
+    causal = bool(seed & 1)
+    check_full(lengths, int(rng.choice([1, 2, 3])), int(rng.choice([64, 128])), causal, seed=2000 + seed)
