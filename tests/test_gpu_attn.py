@@ -255,3 +255,13 @@ def test_random_length_mixes(seed):
         lengths.append(7)
     causal = bool(seed & 1)
     check_full(lengths, int(rng.choice([1, 2, 3])), int(rng.choice([64, 128])), causal, seed=2000 + seed)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_many_sequences_mixed_with_long_ones(causal):
+    # more than 1024 sequences (multi-CTA ranking over the merged list) with a few multi-tile ones in between
+    rng = np.random.default_rng(77)
+    lengths = [int(x) for x in rng.choice([0, 1, 2, 4, 8, 13, 30, 64, 65, 100], size=1300)]
+    for pos, L in ((5, 700), (400, 129), (401, 1000), (1299, 300)):
+        lengths[pos] = L
+    check_full(lengths, 1, 64, causal, seed=78)
