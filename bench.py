@@ -175,10 +175,10 @@ def run_ours(args):
         # clips, the kernels see one sequence per latent frame (spatial) or per spatial position (temporal)
         axis = args.workload[:-2]
         clips = inputs.video_clips()
-        batches, H, d, causal = [[f * s for f, s in clips]], 16, 128, False
+        batches, H, d, causal = [[f * s for f, s in clips]], 16, args.head_dim, False
         seqs = inputs.axis_lengths(clips, axis)
         name = (f"config-3 clips, {axis} axis of a 2-D model: {len(seqs)} sequences of {min(seqs)}-{max(seqs)} tokens, "
-                f"{sum(seqs)} tokens, 16 heads, head_dim 128, bidirectional")
+                f"{sum(seqs)} tokens, 16 heads, head_dim {d}, bidirectional")
     else:
         w = workload(args.workload)
         lengths = [L for L in w.lengths if not args.drop_longer_than or L <= args.drop_longer_than]
@@ -389,6 +389,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="video",
                     choices=["video", "text", "extreme", "stream", "spatial2d", "temporal2d"])
+    ap.add_argument("--head-dim", type=int, default=128,
+                    help="head dimension of the 2-D workloads (the paper's second model has 72)")
     ap.add_argument("--stream-batches", type=int, default=256)
     ap.add_argument("--layers", type=int, default=1, help="planner's layer count Lambda")
     ap.add_argument("--plan", default="model", choices=["model", "profiled"],

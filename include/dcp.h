@@ -9,7 +9,8 @@
  * Tensor layout: q, k, v, o, d_o, dq, dk, dv are bf16, shape [total_tokens, n_heads, head_dim],
  * contiguous, sequences packed back to back; sequence b owns tokens cu_seqlens[b] ..
  * cu_seqlens[b+1]-1.  lse is fp32, shape [n_heads, total_tokens].  Device pointers must be
- * 16-byte aligned.  Supported head_dim: 64 and 128.  n_heads is the same for q, k and v.
+ * 16-byte aligned.  Supported head_dim: multiples of 8 up to 128 (64 and 128 are native; the
+ * others run zero-padded to the next of the two).  n_heads is the same for q, k and v.
  */
 #ifndef DCP_H_
 #define DCP_H_
@@ -25,7 +26,7 @@ enum {
     DCP_OK = 0,
     DCP_ERR_INVALID_ARG = 1, /* null pointer, negative size, misaligned pointer, ...            */
     DCP_ERR_INFEASIBLE = 2,  /* planner: one sequence exceeds the budget even at full recompute */
-    DCP_ERR_UNSUPPORTED = 3, /* head_dim not 64/128, device is not sm_100                       */
+    DCP_ERR_UNSUPPORTED = 3, /* head_dim not a multiple of 8 up to 128, device is not sm_100    */
     DCP_ERR_WORKSPACE = 4,   /* workspace missing or smaller than dcp_varlen_attn_workspace     */
     DCP_ERR_CUDA = 5,        /* a CUDA runtime/driver call or a launch failed                   */
     DCP_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired (see dcp_query_status)       */

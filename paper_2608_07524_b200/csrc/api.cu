@@ -121,8 +121,8 @@ int check_shape(const char* fn, int32_t n_seqs, int32_t total_tokens, int32_t ma
         return fail(DCP_ERR_INVALID_ARG, "%s: negative size or n_heads < 1", fn);
     if (n_seqs > 65535) return fail(DCP_ERR_UNSUPPORTED, "%s: at most 65535 sequences per call", fn);
     if (n_heads > 65535) return fail(DCP_ERR_UNSUPPORTED, "%s: at most 65535 heads", fn);
-    if (head_dim != 64 && head_dim != 128)
-        return fail(DCP_ERR_UNSUPPORTED, "%s: head_dim %d is not supported (64 or 128)", fn, head_dim);
+    if (head_dim < 8 || head_dim > 128 || head_dim % 8 != 0)
+        return fail(DCP_ERR_UNSUPPORTED, "%s: head_dim %d is not supported (a multiple of 8 up to 128)", fn, head_dim);
     if (max_seqlen > total_tokens) return fail(DCP_ERR_INVALID_ARG, "%s: max_seqlen exceeds total_tokens", fn);
     if (!(softmax_scale >= 0.f) || std::isinf(softmax_scale))
         return fail(DCP_ERR_INVALID_ARG, "%s: softmax_scale must be finite and >= 0 (0 selects 1/sqrt(d))", fn);
@@ -145,6 +145,9 @@ SchedView carve_sched(void* workspace, int32_t n_seqs) {
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// The kernels work on 64 or 128 columns per head; other head dimensions run zero-padded to the next of the two.
+size_t padded_dim(int32_t head_dim) { return head_dim <= 64 ? 64 : 128; }
+
 }  // namespace
 }  // namespace dcp
 
@@ -162,7 +165,7 @@ extern "C" int dcp_varlen_attn_workspace(int32_t total_tokens, int32_t n_seqs, i
     if (fwd_bytes) *fwd_bytes = sched;
     if (bwd_bytes)
         *bwd_bytes = sched + align256(max_tiles(total_tokens, n_seqs) * n_heads * (size_t)(kTile * 16 * 2)) +
-                     align256(sizeof(float) * max_tiles(total_tokens, n_seqs) * kTile * n_heads * head_dim);
+                     align256(sizeof(float) * max_tiles(total_tokens, n_seqs) * kTile * n_heads * padded_dim(head_dim));
     return DCP_OK;
 }
 
@@ -212,6 +215,7 @@ static int attn_fwd_impl(const char* fn, bool merge, const void* q, const void* 
     p.lse = lse;
     p.sched = sched;
     p.n_heads = n_heads;
+    p.head_dim = head_dim;
     p.total_tokens = total_tokens;
     p.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
     p.scale_log2 = p.scale * 1.4426950408889634f;
@@ -281,7 +285,7 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
     {
         ScopedTimer t(DCP_KERNEL_BWD_PRE, stream);
         e = launch_bwd_pre(static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, vcu,
-                           sched, stats, dq_acc, max_tiles(total_tokens, n_seqs) * kTile * n_heads * head_dim,
+                           sched, stats, dq_acc, max_tiles(total_tokens, n_seqs) * kTile * n_heads * padded_dim(head_dim),
                            total_tokens, n_heads, head_dim,
                            softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim), dev.sm_count, stream);
     }
@@ -298,6 +302,7 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
     p.dv = static_cast<__nv_bfloat16*>(dv);
     p.sched = sched;
     p.n_heads = n_heads;
+    p.head_dim = head_dim;
     p.total_tokens = total_tokens;
     p.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
     p.scale_log2 = p.scale * 1.4426950408889634f;

@@ -581,7 +581,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             mbar_wait(&sh.dkv_full, n_work & 1u, guard);
             tc_fence_after();
             const size_t tok = (size_t)w.tok0 + (size_t)key;
-            const size_t out_off = (tok * p.n_heads + w.head) * D + half * (D / 2);
+            const size_t out_off = (tok * p.n_heads + w.head) * p.head_dim + half * (D / 2);
 #pragma unroll
             for (int which = 0; which < 2; ++which) {
                 const uint32_t src = tmem + lane_base + (which == 0 ? Cfg::kDv : Cfg::kDk) + half * (D / 2);
@@ -600,7 +600,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                             val.y = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 2]) * mul, __uint_as_float(acc[v4 * 8 + 3]) * mul);
                             val.z = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 4]) * mul, __uint_as_float(acc[v4 * 8 + 5]) * mul);
                             val.w = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 6]) * mul, __uint_as_float(acc[v4 * 8 + 7]) * mul);
-                            *reinterpret_cast<uint4*>(dst + c * 32 + v4 * 8) = val;
+                            if (half * (D / 2) + c * 32 + v4 * 8 < p.head_dim) *reinterpret_cast<uint4*>(dst + c * 32 + v4 * 8) = val;
                         }
                     }
                 }
@@ -647,7 +647,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 if (w.len <= kTile) {
                     // the sequence's only tile pair: this is the whole dQ, no accumulation needed
                     if (qrow < w.len) {
-                        __nv_bfloat16* out = p.dq + (((size_t)w.tok0 + qrow) * p.n_heads + w.head) * D;
+                        __nv_bfloat16* out = p.dq + (((size_t)w.tok0 + qrow) * p.n_heads + w.head) * p.head_dim;
 #pragma unroll
                         for (int c = 0; c < D / 8; ++c) {
                             uint4 val;
@@ -655,7 +655,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                             val.y = pack_bf16x2(__uint_as_float(acc[c * 8 + 2]) * p.scale, __uint_as_float(acc[c * 8 + 3]) * p.scale);
                             val.z = pack_bf16x2(__uint_as_float(acc[c * 8 + 4]) * p.scale, __uint_as_float(acc[c * 8 + 5]) * p.scale);
                             val.w = pack_bf16x2(__uint_as_float(acc[c * 8 + 6]) * p.scale, __uint_as_float(acc[c * 8 + 7]) * p.scale);
-                            *reinterpret_cast<uint4*>(out + c * 8) = val;
+                            if (c * 8 < p.head_dim) *reinterpret_cast<uint4*>(out + c * 8) = val;
                         }
                     }
                 } else {
@@ -689,7 +689,7 @@ static cudaError_t launch_one(const CUtensorMap& tq, const CUtensorMap& tk, cons
 
 cudaError_t launch_attn_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
                             const BwdParams& p, int head_dim, bool causal, int n_ctas, cudaStream_t stream) {
-    if (head_dim == 128)
+    if (head_dim > 64)
         return causal ? launch_one<128, true>(tq, tk, tv, tdo, p, n_ctas, stream)
                       : launch_one<128, false>(tq, tk, tv, tdo, p, n_ctas, stream);
     return causal ? launch_one<64, true>(tq, tk, tv, tdo, p, n_ctas, stream)

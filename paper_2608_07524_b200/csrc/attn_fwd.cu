@@ -172,7 +172,7 @@ __device__ __noinline__ void softmax_single_tile_item(FwdShared& sh, const FwdPa
     tc_fence_after();
     const float inv_l = 1.0f / l;
     const size_t tok = (size_t)w.tok0 + (size_t)row;
-    __nv_bfloat16* out = p.o + (tok * p.n_heads + w.head) * D;
+    __nv_bfloat16* out = p.o + (tok * p.n_heads + w.head) * p.head_dim;
 #pragma unroll
     for (int c = 0; c < D / 32; ++c) {
         uint32_t acc[32];
@@ -186,7 +186,7 @@ __device__ __noinline__ void softmax_single_tile_item(FwdShared& sh, const FwdPa
                 val.y = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 2]) * inv_l, __uint_as_float(acc[v4 * 8 + 3]) * inv_l);
                 val.z = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 4]) * inv_l, __uint_as_float(acc[v4 * 8 + 5]) * inv_l);
                 val.w = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 6]) * inv_l, __uint_as_float(acc[v4 * 8 + 7]) * inv_l);
-                *reinterpret_cast<uint4*>(out + c * 32 + v4 * 8) = val;
+                if (c * 32 + v4 * 8 < p.head_dim) *reinterpret_cast<uint4*>(out + c * 32 + v4 * 8) = val;
             }
         }
     }
@@ -506,7 +506,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             const float inv_l = 1.0f / l;
             const bool valid = row < w.len;
             const size_t tok = (size_t)w.tok0 + (size_t)row;
-            __nv_bfloat16* out = p.o + (tok * p.n_heads + w.head) * D;
+            __nv_bfloat16* out = p.o + (tok * p.n_heads + w.head) * p.head_dim;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t acc[32];
@@ -520,7 +520,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         val.y = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 2]) * inv_l, __uint_as_float(acc[v4 * 8 + 3]) * inv_l);
                         val.z = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 4]) * inv_l, __uint_as_float(acc[v4 * 8 + 5]) * inv_l);
                         val.w = pack_bf16x2(__uint_as_float(acc[v4 * 8 + 6]) * inv_l, __uint_as_float(acc[v4 * 8 + 7]) * inv_l);
-                        *reinterpret_cast<uint4*>(out + c * 32 + v4 * 8) = val;
+                        if (c * 32 + v4 * 8 < p.head_dim) *reinterpret_cast<uint4*>(out + c * 32 + v4 * 8) = val;
                     }
                 }
             }
@@ -549,7 +549,7 @@ static cudaError_t launch_one(const CUtensorMap& tq, const CUtensorMap& tk, cons
 
 cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                             int head_dim, bool causal, int n_ctas, cudaStream_t stream) {
-    if (head_dim == 128)
+    if (head_dim > 64)
         return causal ? launch_one<128, true>(tq, tk, tv, p, n_ctas, stream) : launch_one<128, false>(tq, tk, tv, p, n_ctas, stream);
     return causal ? launch_one<64, true>(tq, tk, tv, p, n_ctas, stream) : launch_one<64, false>(tq, tk, tv, p, n_ctas, stream);
 }

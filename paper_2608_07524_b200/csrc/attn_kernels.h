@@ -15,6 +15,8 @@ struct FwdParams {
     float* lse;
     SchedView sched;
     int32_t n_heads;
+    int32_t head_dim;     // columns of a row in global memory (a multiple of 8); the kernels work on 64 or 128
+                          // columns, those past head_dim read as zeros (TMA fills them) and are never stored
     int32_t total_tokens;
     float scale;        // softmax scale
     float scale_log2;   // scale * log2(e)
@@ -32,6 +34,7 @@ struct BwdParams {
     __nv_bfloat16* dv;
     SchedView sched;
     int32_t n_heads;
+    int32_t head_dim;     // as in FwdParams
     int32_t total_tokens;
     float scale;
     float scale_log2;

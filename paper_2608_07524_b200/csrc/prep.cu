@@ -221,7 +221,8 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
                                                       const int32_t* __restrict__ cu, const uint32_t* __restrict__ tile_prefix,
                                                       int32_t n_seqs, __nv_bfloat16* __restrict__ stats,
                                                       float* __restrict__ dq_acc, size_t dq_acc_vec4,
-                                                      int32_t total_tokens, int32_t n_heads, float inv_scale) {
+                                                      int32_t total_tokens, int32_t n_heads, int32_t head_dim,
+                                                      float inv_scale) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t n_blocks = tile_prefix[n_seqs] * (uint32_t)n_heads;
     for (uint32_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
@@ -256,13 +257,15 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
                 nl[u] = -1e30f;
                 if (row0 + r < len) {
                     const size_t tok = (size_t)cu[lo] + row0 + r;
-                    const size_t row = tok * n_heads + h;
+                    const size_t row = (tok * n_heads + h) * (size_t)head_dim;     // rows hold head_dim <= D columns
                     if (kPer == 4) {
-                        a[u] = *reinterpret_cast<const uint2*>(o + row * D + lane * 4);
-                        b[u] = *reinterpret_cast<const uint2*>(d_o + row * D + lane * 4);
-                    } else {
-                        a[u].x = *reinterpret_cast<const uint32_t*>(o + row * D + lane * 2);
-                        b[u].x = *reinterpret_cast<const uint32_t*>(d_o + row * D + lane * 2);
+                        if (lane * 4 < head_dim) {
+                            a[u] = *reinterpret_cast<const uint2*>(o + row + lane * 4);
+                            b[u] = *reinterpret_cast<const uint2*>(d_o + row + lane * 4);
+                        }
+                    } else if (lane * 2 < head_dim) {
+                        a[u].x = *reinterpret_cast<const uint32_t*>(o + row + lane * 2);
+                        b[u].x = *reinterpret_cast<const uint32_t*>(d_o + row + lane * 2);
                     }
                     if (lane == 0) nl[u] = -lse[(size_t)h * total_tokens + tok] * inv_scale;
                 }
@@ -309,12 +312,14 @@ cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, con
                            int32_t total_tokens, int32_t n_heads, int32_t head_dim, float scale, int n_sms,
                            cudaStream_t stream) {
     const int blocks = n_sms * 8;
-    if (head_dim == 128)
+    if (head_dim > 64)
         bwd_pre_kernel<128><<<blocks, 256, 0, stream>>>(o, d_o, lse, cu_seqlens, sched.tile_prefix, sched.n_seqs, stats,
-                                                        dq_acc, dq_acc_elems / 4, total_tokens, n_heads, 1.0f / scale);
+                                                        dq_acc, dq_acc_elems / 4, total_tokens, n_heads, head_dim,
+                                                        1.0f / scale);
     else
         bwd_pre_kernel<64><<<blocks, 256, 0, stream>>>(o, d_o, lse, cu_seqlens, sched.tile_prefix, sched.n_seqs, stats,
-                                                       dq_acc, dq_acc_elems / 4, total_tokens, n_heads, 1.0f / scale);
+                                                       dq_acc, dq_acc_elems / 4, total_tokens, n_heads, head_dim,
+                                                       1.0f / scale);
     return cudaGetLastError();
 }
 
@@ -324,7 +329,7 @@ cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, con
 template <int D>
 __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict__ dq,
                                                        const int32_t* __restrict__ cu, const uint32_t* __restrict__ tile_prefix,
-                                                       int32_t n_seqs, int32_t n_heads, float scale) {
+                                                       int32_t n_seqs, int32_t n_heads, int32_t head_dim, float scale) {
     constexpr int kRowBytes = D * 2 + 16;                    // padded row of bf16
     __shared__ __align__(16) uint8_t tile[kTile * kRowBytes];
     const uint32_t n_blocks = tile_prefix[n_seqs] * (uint32_t)n_heads;
@@ -353,11 +358,11 @@ __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__
             *reinterpret_cast<uint2*>(tile + r * kRowBytes + c4 * 8) = pk;
         }
         __syncthreads();
-        constexpr int kChunks = D * 2 / 16;                  // 16-byte chunks per row
+        const int kChunks = head_dim * 2 / 16;               // 16-byte chunks per stored row (head_dim <= D columns)
         for (int e = threadIdx.x; e < rows * kChunks; e += blockDim.x) {
             const int r = e / kChunks, c = e % kChunks;
             const uint4 v = *reinterpret_cast<const uint4*>(tile + r * kRowBytes + c * 16);
-            __nv_bfloat16* out = dq + (((size_t)cu[lo] + row0 + r) * n_heads + h) * D;
+            __nv_bfloat16* out = dq + (((size_t)cu[lo] + row0 + r) * n_heads + h) * (size_t)head_dim;
             reinterpret_cast<uint4*>(out)[c] = v;
         }
         __syncthreads();
@@ -368,10 +373,12 @@ __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__
 cudaError_t launch_bwd_post(const float* dq_acc, __nv_bfloat16* dq, const int32_t* cu_seqlens, const SchedView& sched,
                             int32_t n_heads, int32_t head_dim, float scale, int n_sms, cudaStream_t stream) {
     const int blocks = n_sms * 4;
-    if (head_dim == 128)
-        bwd_post_kernel<128><<<blocks, 256, 0, stream>>>(dq_acc, dq, cu_seqlens, sched.tile_prefix, sched.n_seqs, n_heads, scale);
+    if (head_dim > 64)
+        bwd_post_kernel<128><<<blocks, 256, 0, stream>>>(dq_acc, dq, cu_seqlens, sched.tile_prefix, sched.n_seqs, n_heads,
+                                                         head_dim, scale);
     else
-        bwd_post_kernel<64><<<blocks, 256, 0, stream>>>(dq_acc, dq, cu_seqlens, sched.tile_prefix, sched.n_seqs, n_heads, scale);
+        bwd_post_kernel<64><<<blocks, 256, 0, stream>>>(dq_acc, dq, cu_seqlens, sched.tile_prefix, sched.n_seqs, n_heads,
+                                                        head_dim, scale);
     return cudaGetLastError();
 }
 

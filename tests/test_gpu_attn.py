@@ -185,7 +185,7 @@ def test_packing_independence_on_gpu():
 
 def test_library_rejects_bad_arguments():
     dev = "cuda"
-    q = torch.zeros((10, 2, 96), dtype=torch.bfloat16, device=dev)
+    q = torch.zeros((10, 2, 100), dtype=torch.bfloat16, device=dev)       # not a multiple of 8
     cu = torch.tensor([0, 10], dtype=torch.int32, device=dev)
     with pytest.raises(B.DcpError) as e:
         B.dcp_varlen_attn_fwd(q, q, q, cu, 10, False)
@@ -265,3 +265,12 @@ def test_many_sequences_mixed_with_long_ones(causal):
     for pos, L in ((5, 700), (400, 129), (401, 1000), (1299, 300)):
         lengths[pos] = L
     check_full(lengths, 1, 64, causal, seed=78)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("d", [8, 40, 72, 96, 120])
+def test_head_dims_between_the_native_ones(causal, d):
+    # head dimensions other than 64 and 128 run zero-padded to the next of the two (72 is the head
+    # dimension of the paper's second model: hidden size 1152 over 16 heads)
+    check_full([300, 5, 13, 8, 129, 64, 1, 250], 3, d, causal, seed=90 + d)
+

@@ -40,10 +40,10 @@ def sample_positions(L, rng, n_random=24):
     return np.array(sorted(pos), np.int32)
 
 
-def workload_of(param):
+def workload_of(param, head_dim=128):
     if isinstance(param, int):
         return inputs.config(param)
-    return inputs.Workload(param, inputs.short2d_lengths(param[:-2]), 16, 128, False, 12)
+    return inputs.Workload(param, inputs.short2d_lengths(param[:-2]), 16, head_dim, False, 12)
 
 
 @pytest.fixture(scope="module", params=[2, 3, 4, "spatial2d"])
@@ -124,10 +124,12 @@ def test_whole_tensor_identities(full_run):
     assert bool(torch.isfinite(o.float()).all()) and bool(torch.isfinite(lse).all())
 
 
-def test_temporal_axis_in_full():
+@pytest.mark.parametrize("head_dim", [128, 72])
+def test_temporal_axis_in_full(head_dim):
     """Thousands of 1-13 token sequences, merged by the work-list kernels into tiles of up to 128
-    tokens: every output element against the oracle."""
-    w = workload_of("temporal2d")
+    tokens: every output element against the oracle.  72 is the head dimension of the paper's
+    second model (it runs zero-padded to 128 columns)."""
+    w = workload_of("temporal2d", head_dim)
     q, k, v, g = inputs.make_qkvg_device(w.total_tokens, w.n_heads, w.head_dim, w.value_seed, "cuda")
     cud = torch.tensor(w.cu_seqlens, dtype=torch.int32, device="cuda")
     ws = B.alloc_workspace(w.total_tokens, len(w.lengths), w.n_heads, w.head_dim, True, "cuda")
