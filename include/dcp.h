@@ -134,6 +134,9 @@ int dcp_inter_plan(const int64_t* times, int32_t n, int32_t g_min, int32_t g_max
  * Both calls only enqueue work on `cuda_stream` (a cudaStream_t; NULL = the default stream);
  * they neither synchronise nor read cu_seqlens on the host.  softmax_scale = 0 selects
  * 1/sqrt(head_dim).  Zero-length sequences are legal.  max_seqlen must be >= every length.
+ * cu_seqlens is checked on the device (it must start at 0, never decrease, end at total_tokens, and
+ * fit the workspace that max_seqlen promised): if it does not hold, the call computes nothing,
+ * leaves the outputs as they were and dcp_query_status returns DCP_ERR_INVALID_ARG.
  */
 
 /* Bytes of caller-provided device workspace needed by the forward and the backward call: the work
@@ -184,8 +187,8 @@ int dcp_varlen_attn_fwd_noalloc(const void* q, const void* k, const void* v, con
                                 int32_t causal, float softmax_scale, void* o, float* lse, void* cuda_stream);
 
 /* Synchronises `cuda_stream`, then reads the status word at the start of `workspace`.
- * Returns DCP_OK, DCP_ERR_TIMEOUT (a kernel abandoned a bounded wait; results are invalid) or
- * DCP_ERR_CUDA. */
+ * Returns DCP_OK, DCP_ERR_TIMEOUT (a kernel abandoned a bounded wait; results are invalid),
+ * DCP_ERR_INVALID_ARG (cu_seqlens was inconsistent; nothing was computed) or DCP_ERR_CUDA. */
 int dcp_query_status(const void* workspace, void* cuda_stream);
 
 /* Measurement aid (no counterpart in the paper).  While enabled, every attention call records a

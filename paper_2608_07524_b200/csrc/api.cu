@@ -197,7 +197,8 @@ static int attn_fwd_impl(const char* fn, bool merge, const void* q, const void* 
     cudaError_t e;
     {
         ScopedTimer t(DCP_KERNEL_PREP, stream);
-        e = launch_prep(cu_seqlens, n_seqs, total_tokens, max_seqlen, kFwdRowsPerItem, n_heads, sched, bounds, stream);
+        e = launch_prep(cu_seqlens, n_seqs, total_tokens, max_seqlen, kFwdRowsPerItem, n_heads, sched, bounds, UINT32_MAX,
+                        stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: work-list kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(prep_launches(n_seqs, merge));
@@ -269,7 +270,8 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
     cudaError_t e;
     {
         ScopedTimer t(DCP_KERNEL_PREP, stream);
-        e = launch_prep(cu_seqlens, n_seqs, total_tokens, max_seqlen, kTile, n_heads, sched, bounds, stream);
+        e = launch_prep(cu_seqlens, n_seqs, total_tokens, max_seqlen, kTile, n_heads, sched, bounds,
+                        (uint32_t)max_tiles(total_tokens, n_seqs), stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: work-list kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(prep_launches(n_seqs, true));
@@ -377,6 +379,10 @@ extern "C" int dcp_query_status(const void* workspace, void* cuda_stream) {
     cudaError_t e = cudaMemcpyAsync(&status, workspace, sizeof status, cudaMemcpyDeviceToHost, stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "dcp_query_status: %s", cudaGetErrorString(e));
+    if (status == kStatusBadLengths)
+        return fail(DCP_ERR_INVALID_ARG,
+                    "cu_seqlens disagrees with n_seqs, total_tokens or max_seqlen (it must start at 0, never decrease, end "
+                    "at total_tokens, and no sequence may exceed max_seqlen); nothing was computed");
     if (status != 0) return fail(DCP_ERR_TIMEOUT, "a kernel abandoned a bounded wait (device status %u); results are invalid", status);
     return DCP_OK;
 }

@@ -45,9 +45,12 @@ struct BwdParams {
 // `bounds` are written and the list is built over sched.vcu, which the later kernels must then be
 // given as their boundary array; with `bounds` null the list is built over cu_seqlens itself.
 int prep_launches(int32_t n_seqs, bool merge);   // kernels launch_prep enqueues (1 to 4)
+// tile_capacity = number of 128-row tiles the per-tile storage of the workspace holds (UINT32_MAX if the
+// call uses none).  Inconsistent boundaries or more tiles than that leave an empty work list and
+// kStatusBadLengths in the status word.
 cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen,
                         int32_t rows_per_block, int32_t n_heads, const SchedView& sched, uint16_t* bounds,
-                        cudaStream_t stream);
+                        uint32_t tile_capacity, cudaStream_t stream);
 
 cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                             int head_dim, bool causal, int n_ctas, cudaStream_t stream);

@@ -33,6 +33,19 @@ __global__ void __launch_bounds__(kPrepThreads) merge_kernel(const int32_t* __re
     auto is_head = [&](int i) { return merge_is_head(cu, i, max_short); };
     const int per = (n_seqs + kPrepThreads - 1) / kPrepThreads;
     const int begin = min(tid * per, n_seqs), end = min(begin + per, n_seqs);
+    // The boundaries come from the caller and index everything that follows: they must start at 0, never
+    // decrease and end at total_tokens.  If not, the status word says so and every sequence is made empty,
+    // which turns the rest of the call into no-ops.  This kernel is the first of a call, so it also resets
+    // the status word.
+    int bad = (tid == 0 && (cu[0] != 0 || cu[n_seqs] != total_tokens)) ? 1 : 0;
+    for (int i = begin; i < end; ++i) bad |= cu[i + 1] < cu[i] ? 1 : 0;
+    bad = __syncthreads_or(bad);
+    if (tid == 0) hdr->status = bad ? (uint32_t)kStatusBadLengths : (uint32_t)kStatusOk;
+    if (bad) {
+        for (int i = tid; i <= n_seqs; i += kPrepThreads) vcu[i] = 0;
+        if (tid == 0) hdr->n_vseq = 0;
+        return;
+    }
     uint32_t local = 0, n_v = 0;
     for (int i = begin; i < end; ++i) local += is_head(i) ? 1u : 0u;
     uint32_t run = block_exclusive_scan(local, scratch, &n_v);
@@ -47,9 +60,9 @@ __global__ void __launch_bounds__(kPrepThreads) merge_kernel(const int32_t* __re
 // sequence, one byte each.  The start is found by walking back to the head of the run (the head rule
 // is local, so this does not wait for merge_kernel's scan).
 __global__ void __launch_bounds__(256) bounds_kernel(const int32_t* __restrict__ cu, int32_t n_seqs, int32_t max_short,
-                                                     uint16_t* __restrict__ bounds) {
+                                                     const WorkspaceHeader* __restrict__ hdr, uint16_t* __restrict__ bounds) {
     const int i = blockIdx.x * 256 + threadIdx.x;
-    if (i >= n_seqs) return;
+    if (i >= n_seqs || hdr->status != kStatusOk) return;      // merge_kernel found the boundaries inconsistent
     const int32_t a = cu[i], b = cu[i + 1];
     if (b == a || b - a > kTile) return;
     int j = i;
@@ -127,11 +140,25 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __res
                                                             const uint32_t* __restrict__ n_live_ptr,
                                                             int32_t rows_per_block, int32_t n_heads,
                                                             WorkspaceHeader* hdr, int32_t* order, uint32_t* prefix,
-                                                            uint32_t* tile_prefix, int ranked) {
+                                                            uint32_t* tile_prefix, int ranked, int32_t total_tokens,
+                                                            uint32_t tile_capacity) {
     __shared__ uint32_t scratch[33];
     __shared__ int32_t len_sh[kPrepThreads];
     const int tid = threadIdx.x;
     const int n_live = n_live_ptr ? min((int)*n_live_ptr, n_seqs) : n_seqs;
+    if (!n_live_ptr) {
+        // no merge_kernel ran before: check the caller's boundaries here (see merge_kernel)
+        int bad = (tid == 0 && (cu[0] != 0 || cu[n_seqs] != total_tokens)) ? 1 : 0;
+        for (int i = tid; i < n_seqs; i += kPrepThreads) bad |= cu[i + 1] < cu[i] ? 1 : 0;
+        bad = __syncthreads_or(bad);
+        if (tid == 0) hdr->status = bad ? (uint32_t)kStatusBadLengths : (uint32_t)kStatusOk;
+        if (bad) {
+            for (int i = tid; i <= n_seqs; i += kPrepThreads) { prefix[i] = 0; tile_prefix[i] = 0; }
+            for (int i = tid; i < n_seqs; i += kPrepThreads) order[i] = i;
+            if (tid == 0) { hdr->n_items = 0; hdr->work_counter = 0; }
+            return;
+        }
+    }
     if (!ranked) {                                    // n_seqs <= kPrepThreads: one sequence per thread
         len_sh[tid] = tid < n_seqs ? cu[tid + 1] - cu[tid] : -1;
         __syncthreads();
@@ -165,13 +192,19 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __res
     if (tid == 0) {
         hdr->n_items = total;
         hdr->work_counter = 0;
-        hdr->status = 0;
     }
     // tile_prefix[b] = number of 128-row tiles of sequences 0..b-1 (input order): same two-level scan
     auto tiles_of = [&](int b) -> uint32_t { return (uint32_t)((cu[b + 1] - cu[b] + kTile - 1) / kTile); };
     local = 0;
     for (int i = begin; i < end; ++i) local += tiles_of(i);
     run = block_exclusive_scan(local, scratch, &total);
+    if (total > tile_capacity) {
+        // more tiles than the workspace was sized for: max_seqlen was understated (the bound on merged runs
+        // relies on it).  Nothing may index the per-tile storage: no items, no tiles.
+        for (int i = tid; i <= n_seqs; i += kPrepThreads) tile_prefix[i] = 0;
+        if (tid == 0) { hdr->n_items = 0; hdr->status = kStatusBadLengths; }
+        return;
+    }
     for (int i = begin; i < end; ++i) {
         tile_prefix[i] = run;
         run += tiles_of(i);
@@ -183,7 +216,7 @@ int prep_launches(int32_t n_seqs, bool merge) { return (n_seqs > kPrepThreads ? 
 
 cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen,
                         int32_t rows_per_block, int32_t n_heads, const SchedView& sched, uint16_t* bounds,
-                        cudaStream_t stream) {
+                        uint32_t tile_capacity, cudaStream_t stream) {
     const int32_t* cu = cu_seqlens;
     const uint32_t* n_live = nullptr;
     if (bounds) {                                       // merge short sequences; everything below sees vcu
@@ -191,7 +224,8 @@ cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total
         merge_kernel<<<1, kPrepThreads, 0, stream>>>(cu_seqlens, n_seqs, total_tokens, max_short, sched.hdr,
                                                      const_cast<int32_t*>(sched.vcu));
         if (cudaError_t e = cudaGetLastError()) return e;
-        if (n_seqs > 0) bounds_kernel<<<(n_seqs + 255) / 256, 256, 0, stream>>>(cu_seqlens, n_seqs, max_short, bounds);
+        if (n_seqs > 0)
+            bounds_kernel<<<(n_seqs + 255) / 256, 256, 0, stream>>>(cu_seqlens, n_seqs, max_short, sched.hdr, bounds);
         if (cudaError_t e = cudaGetLastError()) return e;
         cu = sched.vcu;
         n_live = &sched.hdr->n_vseq;
@@ -203,7 +237,7 @@ cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total
     }
     prep_kernel<<<1, kPrepThreads, 0, stream>>>(cu, n_seqs, n_live, rows_per_block, n_heads, sched.hdr,
                                                 const_cast<int32_t*>(sched.order), const_cast<uint32_t*>(sched.prefix),
-                                                const_cast<uint32_t*>(sched.tile_prefix), ranked);
+                                                const_cast<uint32_t*>(sched.tile_prefix), ranked, total_tokens, tile_capacity);
     return cudaGetLastError();
 }
 

@@ -20,6 +20,14 @@ constexpr int kTile = 128;            // rows of a Q tile / keys of a K,V tile
 constexpr int kFwdRowsPerItem = 256;  // a forward work item is two Q tiles of one (sequence, head)
 constexpr int kMergeMaxLen = 64;      // sequences longer than this are never merged with their neighbours
 
+// Status codes a kernel may leave in the workspace's status word (0 = no error).
+enum : uint32_t {
+    kStatusOk = 0,
+    kStatusWaitTimeout = 1,
+    kStatusBadSmemAlign = 2,
+    kStatusBadLengths = 3     // cu_seqlens disagrees with the sizes the caller declared; nothing was computed
+};
+
 // First bytes of every workspace.  `status` must stay at offset 0 (dcp_query_status reads it).
 struct WorkspaceHeader {
     uint32_t status;        // 0 = ok, else a kStatus* code left by a kernel

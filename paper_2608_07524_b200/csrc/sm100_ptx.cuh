@@ -5,11 +5,10 @@
 #include <cstdint>
 #include <cuda_bf16.h>
 
+#include "sched.cuh"     // status codes
+
 namespace dcp {
 
-// ------------------------------------------------------------------------------------------
-// Status codes a kernel may leave in the caller's status word (0 = no error).
-enum : uint32_t { kStatusOk = 0, kStatusWaitTimeout = 1, kStatusBadSmemAlign = 2 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));

@@ -274,3 +274,55 @@ def test_head_dims_between_the_native_ones(causal, d):
     # dimension of the paper's second model: hidden size 1152 over 16 heads)
     check_full([300, 5, 13, 8, 129, 64, 1, 250], 3, d, causal, seed=90 + d)
 
+
+
+def test_inconsistent_boundaries_are_reported_not_used():
+    """cu_seqlens is device data the host never reads; the work-list kernels check it (starts at 0,
+    never decreases, ends at total_tokens, fits the per-tile storage that max_seqlen promised) and, if
+    it does not hold, leave an empty work list and a status the host can query.  Outputs stay as
+    they were; nothing is read or written out of bounds."""
+    dev = "cuda"
+    T, H, d = 600, 2, 64
+    q, k, v, g = (x.to(dev) for x in inputs.make_qkvg(T, H, d, 60))
+    for bad_cu in ([0, 200, 100, 600], [0, 200, 400, 590], [5, 200, 400, 600], [0, 200, 400, 700]):
+        cud = torch.tensor(bad_cu, dtype=torch.int32, device=dev)
+        ws = B.alloc_workspace(T, 3, H, d, True, dev)
+        o = torch.full_like(q, 7.0)
+        lse = torch.zeros((H, T), dtype=torch.float32, device=dev)
+        B.dcp_varlen_attn_fwd(q, k, v, cud, 300, False, out=o, lse=lse, workspace=ws)
+        with pytest.raises(B.DcpError) as e:
+            B.dcp_query_status(ws)
+        assert e.value.code == B.DCP_ERR_INVALID_ARG
+        assert bool((o == 7.0).all())
+        dq = torch.full_like(q, 3.0)
+        B.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cud, 300, False, dq=dq, dk=torch.empty_like(q), dv=torch.empty_like(q),
+                              workspace=ws)
+        with pytest.raises(B.DcpError) as e:
+            B.dcp_query_status(ws)
+        assert e.value.code == B.DCP_ERR_INVALID_ARG and bool((dq == 3.0).all())
+        # the same workspace works again with consistent boundaries
+        good = torch.tensor([0, 200, 400, 600], dtype=torch.int32, device=dev)
+        B.dcp_varlen_attn_fwd(q, k, v, good, 200, False, out=o, lse=lse, workspace=ws)
+        B.dcp_query_status(ws)
+        assert bool(torch.isfinite(o.float()).all()) and not bool((o == 7.0).all())
+
+
+def test_understated_max_seqlen_cannot_overrun_the_workspace():
+    # 2000 sequences of 14 tokens declared as "at most 13": none is merged, so the batch has more tiles than
+    # the workspace (sized on the promise) holds; the backward must refuse instead of indexing past its storage
+    dev = "cuda"
+    n, L, H, d = 2000, 14, 1, 64
+    T = n * L
+    q, k, v, g = (x.to(dev) for x in inputs.make_qkvg(T, H, d, 61))
+    cud = torch.arange(0, T + 1, L, dtype=torch.int32, device=dev)
+    ws = B.alloc_workspace(T, n, H, d, True, dev)
+    o, lse = B.dcp_varlen_attn_fwd(q, k, v, cud, 13, False, workspace=ws)      # forward has no per-tile storage
+    B.dcp_query_status(ws)
+    dq = torch.full_like(q, 3.0)
+    B.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cud, 13, False, dq=dq, dk=torch.empty_like(q), dv=torch.empty_like(q), workspace=ws)
+    with pytest.raises(B.DcpError) as e:
+        B.dcp_query_status(ws)
+    assert e.value.code == B.DCP_ERR_INVALID_ARG and bool((dq == 3.0).all())
+    dq, dk, dv = B.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cud, L, False, workspace=ws)      # the truth: fine
+    B.dcp_query_status(ws)
+    assert bool(torch.isfinite(dq.float()).all())
