@@ -280,6 +280,8 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
         uint8_t* out = reinterpret_cast<uint8_t*>(stats) + ((size_t)t * n_heads + h) * (kTile * 16 * 2);
         // a warp takes rows warp, warp+8, ...; four rows per pass so that eight loads are in flight per lane
         constexpr int kPer = D / 32;           // elements per lane: 2 or 4
+        const bool lane_live = lane * kPer < head_dim;
+        const int lane_col = lane_live ? lane * kPer : 0;
         for (int r0 = warp; r0 < kTile; r0 += 32) {
             float acc[4], nl[4];
             uint2 a[4], b[4];
@@ -291,16 +293,17 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
                 nl[u] = -1e30f;
                 if (row0 + r < len) {
                     const size_t tok = (size_t)cu[lo] + row0 + r;
-                    const size_t row = (tok * n_heads + h) * (size_t)head_dim;     // rows hold head_dim <= D columns
+                    // rows hold head_dim <= D columns; lanes past them re-read column 0 and drop it, so that the
+                    // loads stay unconditional and eight of them are in flight per lane
+                    const size_t row = (tok * n_heads + h) * (size_t)head_dim + lane_col;
                     if (kPer == 4) {
-                        if (lane * 4 < head_dim) {
-                            a[u] = *reinterpret_cast<const uint2*>(o + row + lane * 4);
-                            b[u] = *reinterpret_cast<const uint2*>(d_o + row + lane * 4);
-                        }
-                    } else if (lane * 2 < head_dim) {
-                        a[u].x = *reinterpret_cast<const uint32_t*>(o + row + lane * 2);
-                        b[u].x = *reinterpret_cast<const uint32_t*>(d_o + row + lane * 2);
+                        a[u] = *reinterpret_cast<const uint2*>(o + row);
+                        b[u] = *reinterpret_cast<const uint2*>(d_o + row);
+                    } else {
+                        a[u].x = *reinterpret_cast<const uint32_t*>(o + row);
+                        b[u].x = *reinterpret_cast<const uint32_t*>(d_o + row);
                     }
+                    if (!lane_live) a[u] = make_uint2(0u, 0u);
                     if (lane == 0) nl[u] = -lse[(size_t)h * total_tokens + tok] * inv_scale;
                 }
             }
