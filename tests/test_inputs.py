@@ -62,3 +62,24 @@ def test_two_dimensional_views_of_the_video_clips():
         inputs.clip_shape(777)
     with pytest.raises(ValueError):
         inputs.axis_lengths(clips, "diagonal")
+
+
+def test_cubic_for_exp2_on_the_fma_pipe_is_accurate_enough():
+    """The forward kernel evaluates a share of its exponentials as 2^n * p(f), n = round(x), f = x - n in
+    [-0.5, 0.5], p a cubic (coefficients as in the kernel), with n added into the exponent field after
+    the add-a-magic-number rounding.  Emulated here in fp32: the result must stay well inside the bf16
+    rounding (2^-9) that P gets anyway."""
+    import numpy as np
+    c0, c1, c2, c3 = (np.float32(v) for v in (0.99992807, 0.69326099, 0.24261112, 0.05517162))
+    magic = np.float32(12582912.0)
+    x = np.concatenate([np.linspace(-126.0, 0.0, 200001), -np.logspace(-6, 2, 2000)]).astype(np.float32)
+    xc = np.maximum(x, np.float32(-126.0))
+    t = (xc + magic).astype(np.float32)
+    f = (xc - (t - magic).astype(np.float32)).astype(np.float32)
+    assert float(np.abs(f).max()) <= 0.5
+    q = ((c3 * f + c2) * f + c1) * f + c0
+    bits = q.astype(np.float32).view(np.uint32) + (t.view(np.uint32) << np.uint32(23))
+    got = bits.view(np.float32).astype(np.float64)
+    want = np.exp2(xc.astype(np.float64))
+    rel = np.abs(got / want - 1.0)
+    assert float(rel.max()) < 1.5e-4 < 2.0 ** -9 / 10
