@@ -439,8 +439,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 
                 const bool need = (mx - m) * p.scale_log2 > kRescaleThreshold;
                 if (__any_sync(0xffffffffu, need)) {
-                    const float m_new = fmaxf(m, mx);
-                    const float factor = fast_exp2((m - m_new) * p.scale_log2);
+                    // the branch is warp-wide (the accumulator rescale below is a warp-collective tensor-memory
+                    // access), but each row raises its own maximum only if it needs to itself: what a row
+                    // computes must not depend on the other rows of its warp, some of which may belong to the
+                    // next sequence of the packed batch
+                    const float m_new = need ? fmaxf(m, mx) : m;
+                    const float factor = need ? fast_exp2((m - m_new) * p.scale_log2) : 1.0f;
                     m = m_new;
                     l *= factor;
                     if (j > 0) {

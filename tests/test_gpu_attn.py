@@ -130,15 +130,16 @@ def test_merged_packing_independence():
     cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
     q, k, v, g = inputs.make_qkvg(int(cu[-1]), 2, 128, 14)
     a = run_gpu(q, k, v, g, cu, False)
-    q2, k2, v2, g2 = (x.clone() for x in (q, k, v, g))
-    for x in (q2, k2, v2, g2):
-        x[:23] = torch.randn_like(x[:23].float()).to(torch.bfloat16) * 3
-        x[30:] = torch.randn_like(x[30:].float()).to(torch.bfloat16) * 3
-    b = run_gpu(q2, k2, v2, g2, cu, False)
-    for i in (0, 3, 4):
-        assert torch.equal(a[i][23:30], b[i][23:30])
-    assert torch.equal(a[1][:, 23:30], b[1][:, 23:30])
-    assert float((a[2][23:30].float() - b[2][23:30].float()).abs().max()) <= 2e-2
+    gen = torch.Generator().manual_seed(4321)
+    for _ in range(20):
+        q2, k2, v2, g2 = (x.clone() for x in (q, k, v, g))
+        for x in (q2, k2, v2, g2):
+            x[:23] = (torch.randn(x[:23].shape, generator=gen) * 3).to(torch.bfloat16)
+            x[30:] = (torch.randn(x[30:].shape, generator=gen) * 3).to(torch.bfloat16)
+        b = run_gpu(q2, k2, v2, g2, cu, False)
+        for i in (0, 2, 3, 4):      # a single tile pair: no atomics, dq is bit-exact too
+            assert torch.equal(a[i][23:30], b[i][23:30])
+        assert torch.equal(a[1][:, 23:30], b[1][:, 23:30])
 
 
 def test_more_sequences_than_one_sorting_block():
@@ -166,21 +167,23 @@ def test_backward_in_isolation(causal):
 
 def test_packing_independence_on_gpu():
     """A sequence's outputs do not change when its neighbours' data change (tail tiles read the
-    next sequence's rows through TMA, so the masks must hide them completely)."""
+    next sequence's rows through TMA, so the masks must hide them completely, and no decision a row
+    takes may depend on the other rows of its warp).  Many neighbour draws: a dependence through the
+    lazy rescale of the running maximum only shows for a few per cent of them."""
     lengths = [100, 200, 150]
     cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
     q, k, v, g = inputs.make_qkvg(int(cu[-1]), 2, 128, 9)
     a = run_gpu(q, k, v, g, cu, False)
-    q2, k2, v2, g2 = (x.clone() for x in (q, k, v, g))
-    for x in (q2, k2, v2, g2):
-        x[:100] = torch.randn_like(x[:100].float()).to(torch.bfloat16) * 3
-        x[300:] = torch.randn_like(x[300:].float()).to(torch.bfloat16) * 3
-    b = run_gpu(q2, k2, v2, g2, cu, False)
-    for i in (0, 3, 4):        # o, dk, dv: no atomics involved, bit-exact
-        assert torch.equal(a[i][100:300], b[i][100:300])
-    assert torch.equal(a[1][:, 100:300], b[1][:, 100:300])
-    # dq is summed with atomics in arbitrary order: compare within rounding
-    assert float((a[2][100:300].float() - b[2][100:300].float()).abs().max()) <= 2e-2
+    gen = torch.Generator().manual_seed(1234)
+    for _ in range(60):
+        q2, k2, v2, g2 = (x.clone() for x in (q, k, v, g))
+        for x in (q2, k2, v2, g2):
+            x[:100] = (torch.randn(x[:100].shape, generator=gen) * 3).to(torch.bfloat16)
+            x[300:] = (torch.randn(x[300:].shape, generator=gen) * 3).to(torch.bfloat16)
+        b = run_gpu(q2, k2, v2, g2, cu, False)
+        for i in (0, 2, 3, 4):     # o, dq, dk, dv: this sequence has two key blocks, and a + b = b + a in fp32
+            assert torch.equal(a[i][100:300], b[i][100:300])
+        assert torch.equal(a[1][:, 100:300], b[1][:, 100:300])
 
 
 def test_library_rejects_bad_arguments():
