@@ -171,7 +171,7 @@ int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, const void*
  * a caller buffer.  Limits and rules:
  *   - runs of very short sequences are not merged into shared tiles here (the table that needs grows
  *     with the token count), so such batches run slower than through dcp_varlen_attn_fwd; results
- *     are the same;
+ *     agree within rounding (sequences of at most 128 tokens take different code paths);
  *   - n_seqs <= DCP_NOALLOC_MAX_SEQS, else DCP_ERR_UNSUPPORTED and nothing is enqueued;
  *   - the call allocates nothing on the device and frees nothing;
  *   - the first call on each device looks up the array's device address (a synchronous runtime
