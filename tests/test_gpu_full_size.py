@@ -144,3 +144,36 @@ def test_temporal_axis_in_full(head_dim):
     close("dk", dk, rdk)
     close("dv", dv, rdv)
     assert float(np.max(np.abs(lse.double().cpu().numpy() - Lse))) <= LSE_ABS
+
+
+@pytest.mark.parametrize("cfg", [2, 3])
+def test_full_size_outputs_do_not_depend_on_neighbours(cfg):
+    """Replace one sequence's q, k, v, dO (the second longest) and run again: every other sequence's o,
+    lse, dk and dv must come out bit for bit the same (dq is summed by atomics in arbitrary order once
+    a sequence has more than two key blocks, so it is compared within rounding)."""
+    w = inputs.config(cfg)
+    dev = "cuda"
+    q, k, v, g = inputs.make_qkvg_device(w.total_tokens, w.n_heads, w.head_dim, w.value_seed, dev)
+    cud = torch.tensor(w.cu_seqlens, dtype=torch.int32, device=dev)
+    ws = B.alloc_workspace(w.total_tokens, len(w.lengths), w.n_heads, w.head_dim, True, dev)
+
+    def run():
+        o, lse = B.dcp_varlen_attn_fwd(q, k, v, cud, w.max_seqlen, w.causal, workspace=ws)
+        dq, dk, dv = B.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cud, w.max_seqlen, w.causal, workspace=ws)
+        B.dcp_query_status(ws)
+        return o, lse, dq, dk, dv
+
+    a = run()
+    victim = int(np.argsort(w.lengths)[-2])
+    lo, hi = w.cu_seqlens[victim], w.cu_seqlens[victim + 1]
+    gen = torch.Generator(device=dev).manual_seed(99)
+    for x in (q, k, v, g):
+        x[lo:hi] = (torch.randn(x[lo:hi].shape, generator=gen, device=dev) * 2).to(torch.bfloat16)
+    b = run()
+    keep = torch.ones(w.total_tokens, dtype=torch.bool, device=dev)
+    keep[lo:hi] = False
+    for i in (0, 3, 4):
+        assert torch.equal(a[i][keep], b[i][keep])
+    assert torch.equal(a[1][:, keep], b[1][:, keep])
+    assert float((a[2][keep].float() - b[2][keep].float()).abs().max()) <= 3e-2
+    assert not torch.equal(a[0][lo:hi], b[0][lo:hi])
