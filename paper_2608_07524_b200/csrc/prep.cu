@@ -13,16 +13,29 @@ __device__ inline uint32_t block_exclusive_scan(uint32_t v, uint32_t* scratch, u
 
 // Merging of short sequences into virtual sequences of at most 128 tokens.  One CTA.
 //
-// A sequence is "short" if length <= max_short (empty ones included).  Consecutive short sequences whose first
-// tokens fall into the same window of `window` = 129 - max_short packed positions form one virtual
-// sequence: it spans at most (window - 1) + max_short = 128 tokens.  The rule is local (a sequence
-// starts a virtual sequence iff it is not short, or its predecessor is not short, or the predecessor
-// starts in another window), so heads are found in parallel and compacted with a scan.
+// A sequence is "short" if length <= max_short (empty ones included).  Two local rules say when a short
+// sequence joins the virtual sequence of its short predecessor:
+//   rule 0: both START in the same window of `window` = 129 - max_short packed positions, so a virtual
+//           sequence spans at most (window - 1) + max_short = 128 tokens;
+//   rule 1: the predecessor's first and this sequence's last token lie in the same ALIGNED window of 128
+//           positions, so a virtual sequence lies inside one such window (sequences that cross a window
+//           boundary stay alone).
+// Rule 0 fills tiles well when sequences are much shorter than 64 tokens, rule 1 when they are close to
+// 64 and aligned (64-token sequences pair up exactly, which their start windows of 65 almost never allow).
+// Both are local (whether a sequence starts a virtual sequence depends on it and its predecessor only),
+// so heads are found in parallel and compacted with a scan; the kernel counts the heads under both rules
+// and keeps the rule that gives fewer (rule 1 only if the batch has no empty sequence, which keeps the
+// bound on the number of tiles that sizes the workspace: it is derived for rule 0).
 // Outputs: vcu[0..n_v] = boundaries of the virtual sequences, vcu[n_v+1..n_seqs] = total_tokens
-// (empty padding, so that vcu is a valid boundary array of n_seqs sequences); hdr->n_vseq = n_v.
-__device__ __forceinline__ bool merge_is_head(const int32_t* __restrict__ cu, int i, int32_t max_short) {
-    const int window = kTile + 1 - max_short;
-    return i == 0 || cu[i + 1] - cu[i] > max_short || cu[i] - cu[i - 1] > max_short || cu[i - 1] / window != cu[i] / window;
+// (empty padding, so that vcu is a valid boundary array of n_seqs sequences); hdr->n_vseq = n_v;
+// hdr->merge_rule = the rule used.
+__device__ __forceinline__ bool merge_is_head(const int32_t* __restrict__ cu, int i, int32_t max_short, uint32_t rule) {
+    if (i == 0 || cu[i + 1] - cu[i] > max_short || cu[i] - cu[i - 1] > max_short) return true;
+    if (rule == 0) {
+        const int window = kTile + 1 - max_short;
+        return cu[i - 1] / window != cu[i] / window;
+    }
+    return cu[i - 1] / kTile != (cu[i + 1] - 1) / kTile;
 }
 
 __global__ void __launch_bounds__(kPrepThreads) merge_kernel(const int32_t* __restrict__ cu, int32_t n_seqs,
@@ -30,7 +43,6 @@ __global__ void __launch_bounds__(kPrepThreads) merge_kernel(const int32_t* __re
                                                              WorkspaceHeader* hdr, int32_t* vcu) {
     __shared__ uint32_t scratch[33];
     const int tid = threadIdx.x;
-    auto is_head = [&](int i) { return merge_is_head(cu, i, max_short); };
     const int per = (n_seqs + kPrepThreads - 1) / kPrepThreads;
     const int begin = min(tid * per, n_seqs), end = min(begin + per, n_seqs);
     // The boundaries come from the caller and index everything that follows: they must start at 0, never
@@ -46,12 +58,25 @@ __global__ void __launch_bounds__(kPrepThreads) merge_kernel(const int32_t* __re
         if (tid == 0) hdr->n_vseq = 0;
         return;
     }
-    uint32_t local = 0, n_v = 0;
-    for (int i = begin; i < end; ++i) local += is_head(i) ? 1u : 0u;
-    uint32_t run = block_exclusive_scan(local, scratch, &n_v);
-    if (tid == 0) hdr->n_vseq = n_v;
+    uint32_t local0 = 0, local1 = 0, n_v0 = 0, n_v1 = 0;
+    int empty = 0;
+    for (int i = begin; i < end; ++i) {
+        local0 += merge_is_head(cu, i, max_short, 0) ? 1u : 0u;
+        local1 += merge_is_head(cu, i, max_short, 1) ? 1u : 0u;
+        empty |= cu[i + 1] == cu[i] ? 1 : 0;
+    }
+    empty = __syncthreads_or(empty);
+    const uint32_t run0 = block_exclusive_scan(local0, scratch, &n_v0);
+    const uint32_t run1 = block_exclusive_scan(local1, scratch, &n_v1);
+    const uint32_t rule = (!empty && n_v1 < n_v0) ? 1u : 0u;
+    const uint32_t n_v = rule ? n_v1 : n_v0;
+    uint32_t run = rule ? run1 : run0;
+    if (tid == 0) {
+        hdr->n_vseq = n_v;
+        hdr->merge_rule = rule;
+    }
     for (int i = begin; i < end; ++i)
-        if (is_head(i)) vcu[run++] = cu[i];
+        if (merge_is_head(cu, i, max_short, rule)) vcu[run++] = cu[i];
     for (uint32_t i = n_v + tid; i <= (uint32_t)n_seqs; i += kPrepThreads) vcu[i] = total_tokens;
 }
 
@@ -65,8 +90,9 @@ __global__ void __launch_bounds__(256) bounds_kernel(const int32_t* __restrict__
     if (i >= n_seqs || hdr->status != kStatusOk) return;      // merge_kernel found the boundaries inconsistent
     const int32_t a = cu[i], b = cu[i + 1];
     if (b == a || b - a > kTile) return;
+    const uint32_t rule = hdr->merge_rule;
     int j = i;
-    while (!merge_is_head(cu, j, max_short)) --j;     // at most 127 non-empty members before i
+    while (!merge_is_head(cu, j, max_short, rule)) --j;     // at most 127 non-empty members before i
     const int32_t vstart = cu[j];
     const uint16_t packed = (uint16_t)((a - vstart) | ((b - vstart) << 8));
     for (int32_t t = a; t < b; ++t) bounds[t] = packed;

@@ -34,7 +34,8 @@ struct WorkspaceHeader {
     uint32_t work_counter;  // next unclaimed work item
     uint32_t n_items;       // items in the list
     uint32_t n_vseq;        // virtual sequences that are not padding
-    uint32_t pad[60];
+    uint32_t merge_rule;    // which of the two merging rules built them (see merge_kernel)
+    uint32_t pad[59];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
 

@@ -329,3 +329,12 @@ def test_understated_max_seqlen_cannot_overrun_the_workspace():
     dq, dk, dv = B.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cud, L, False, workspace=ws)      # the truth: fine
     B.dcp_query_status(ws)
     assert bool(torch.isfinite(dq.float()).all())
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_merged_by_aligned_windows(causal):
+    # no empty sequence and lengths near 64: pairing inside aligned 128-token windows gives fewer tiles
+    # than start windows do, so the work-list kernels take their second merging rule
+    lengths = [64] * 9 + [60, 4, 64, 32, 32, 33, 31, 64, 200, 64, 64, 50, 14, 64, 1, 63]
+    check_full(lengths, 2, 128, causal, seed=95)
+    check_full([64] * 40, 1, 64, causal, seed=96)
