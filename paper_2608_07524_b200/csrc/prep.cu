@@ -274,7 +274,8 @@ cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total
 // accumulators with a K=16 MMA against a tile of ones.  Rows past the sequence end get -1e30 and 0,
 // which makes their probabilities vanish without masking.  The tile is stored in the MMA's shared-
 // memory layout (8x8 core matrices; column halves 2048 bytes apart) and is 4 KB-aligned, so one bulk
-// copy fetches it.  Also zeroes the fp32 dQ accumulator.  HBM-bound.
+// copy fetches it.  Also zeroes the fp32 dQ accumulator blocks of sequences longer than one tile (a
+// sequence of a single tile gets its dQ written directly by the main kernel).  HBM-bound.
 template <int D>
 __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __restrict__ o,
                                                       const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ lse,
@@ -388,7 +389,8 @@ cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, con
 
 // Backward helper 2: dq[T, H, d] = bf16(scale * dq_acc).  dq_acc holds, per (tile, head), a block
 // [d/4][128 rows][4 floats]; a CTA reads one block with coalesced 16-byte loads, transposes it in
-// shared memory as bf16 and writes whole rows.  Rows past the sequence end are skipped.
+// shared memory as bf16 and writes whole rows.  Rows past the sequence end are skipped, and so are
+// sequences of a single tile, whose dQ the main kernel has already written.
 template <int D>
 __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict__ dq,
                                                        const int32_t* __restrict__ cu, const uint32_t* __restrict__ tile_prefix,
