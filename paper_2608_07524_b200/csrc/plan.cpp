@@ -84,6 +84,15 @@ int plan_impl(const char* who, const int32_t* lengths, const int64_t* weight, in
     std::vector<int32_t> cut(n + 1, n), rec(n + 1, 0);
     best[n] = {0, 0};
     for (int32_t i = n - 1; i >= 0; --i) {
+        // If the whole suffix fits without recomputation, one block is optimal: it costs T_C, every other
+        // plan costs at least that, and ties go to fewer blocks.  This keeps batches that the budget does
+        // not bind (the usual case) linear instead of quadratic in n.
+        if (min_recompute(tok[n] - tok[i], p, budget) == 0) {
+            best[i] = {(u128)p.fixed_cost, 1};
+            cut[i] = n;
+            rec[i] = 0;
+            continue;
+        }
         bool have = false;
         for (int32_t j = i + 1; j <= n; ++j) {
             const int r = min_recompute(tok[j] - tok[i], p, budget);
