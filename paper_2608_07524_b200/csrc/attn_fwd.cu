@@ -144,22 +144,35 @@ __device__ __noinline__ void softmax_single_tile_item(FwdShared& sh, const FwdPa
 #pragma unroll
     for (int c = 0; c < 4; ++c) tmem_ld_x32(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
     tmem_wait_ld();
-    float m = -INFINITY;
 #pragma unroll
-    for (int c = 0; c < 128; ++c) {
+    for (int c = 0; c < 128; ++c)
         if (c > last_key || c < first_key) s[c] = 0xff800000u;         // -inf
-        m = fmaxf(m, __uint_as_float(s[c]));
+    // this item is one dependent chain S -> softmax -> PV per CTA: eight maxima and two packed sums run
+    // side by side instead of one 128-long chain each
+    float part[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) part[c] = fmax3(__uint_as_float(s[c]), __uint_as_float(s[8 + c]), __uint_as_float(s[16 + c]));
+#pragma unroll
+    for (int c = 24; c < 120; c += 16) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) part[u] = fmax3(part[u], __uint_as_float(s[c + u]), __uint_as_float(s[c + 8 + u]));
     }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) part[u] = fmaxf(part[u], __uint_as_float(s[120 + u]));
+    const float m = fmaxf(fmax3(part[0], part[1], part[2]), fmax3(fmax3(part[3], part[4], part[5]), part[6], part[7]));
     const float neg_m = -m * p.scale_log2;
-    float l = 0.f;
+    const uint64_t sc2 = pack_f32x2(p.scale_log2, p.scale_log2), nm2 = pack_f32x2(neg_m, neg_m);
+    uint64_t sum2[2] = {0ull, 0ull};
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
         uint32_t pk[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + 2 * i]), p.scale_log2, neg_m));
-            const float p1 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + 2 * i + 1]), p.scale_log2, neg_m));
-            l += p0 + p1;
+            float x0, x1;
+            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[c * 32 + 2 * i]), __uint_as_float(s[c * 32 + 2 * i + 1])), sc2, nm2),
+                         x0, x1);
+            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+            sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(p0, p1));
             pk[i] = pack_bf16x2(p0, p1);
         }
         tmem_st_x16(s_tmem + c * 16, pk);
@@ -167,6 +180,13 @@ __device__ __noinline__ void softmax_single_tile_item(FwdShared& sh, const FwdPa
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.p_part[0][c]);
+    }
+    float l;
+    {
+        float a0, a1, b0, b1;
+        unpack_f32x2(sum2[0], a0, a1);
+        unpack_f32x2(sum2[1], b0, b1);
+        l = (a0 + a1) + (b0 + b1);
     }
     mbar_wait(&sh.o_full[0], o_parity, guard);
     tc_fence_after();
