@@ -353,7 +353,7 @@ def run_ours(args):
         roofline = {"bound": "hbm", "kernel": "attn_bwd_kernel (backward main)", "achieved": gbs, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                     "peak_source": f"hbm_gbs of {peaks['source']} MEASURED_PEAKS.json",
-                    "traffic": 3.750e9,        # ncu, one launch of this workload (summary under profiles/)
+                    "traffic": 3.758e9,        # ncu, one launch of this workload (summary under profiles/)
                     "launches": bwd_n, "avg_launch_ms": bwd_ms / bwd_n}
 
     cpu_baseline = None
