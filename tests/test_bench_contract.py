@@ -35,3 +35,26 @@ def test_cuda_arm_fails_loudly_without_a_gpu():
     r = run_bench("--steps", "1", "--warmup", "0", "--no-cpu-baseline")
     assert r.returncode != 0
     assert "no CPU fallback" in (r.stderr + r.stdout)
+
+
+import pytest  # noqa: E402
+
+
+@pytest.mark.gpu
+def test_cuda_arm_prints_the_contract_line():
+    r = run_bench("--workload", "text", "--steps", "2", "--warmup", "3")
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+                "vs_baseline", "dtype", "data", "config", "clocks", "e2e", "gpu_launches", "roofline", "cpu_baseline"):
+        assert key in line, key
+    assert line["dtype"] == "bf16" and line["data"] == "synthetic" and line["scaling"] == "weak" and line["n_gpus"] == 1
+    assert line["value"] > 100 and line["gpu_launches"] == 2 * 10            # ten kernels per step
+    assert "workload" in line["config"]
+    roof = line["roofline"]
+    assert roof["bound"] in ("tensor", "hbm") and 0 < roof["frac"] < 1.2 and roof["achieved"] > 0 and roof["peak"] > 0
+    e2e = line["e2e"]
+    assert e2e["value"] > 0 and e2e["h2d_bytes_per_step"] > 0 and e2e["d2h_bytes_per_step"] > 0
+    assert line["clocks"]["sm_max_mhz"] >= line["clocks"]["sm_mhz"] > 0
+    base = line["cpu_baseline"]
+    assert base["kind"] == "oracle" and base["value"] > 0 and base["cores"] >= 1
