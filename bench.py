@@ -300,7 +300,7 @@ def run_ours(args):
         # timed region includes filling and draining the pipeline.
         runners = [runner, StreamRunner(max_tokens, max_seqs, H, d, causal, dev, value_seed=13 + 100 * rank)]
         pipe = HostPipeline(runners, T)
-        n_pipe = 2 * n_e2e
+        n_pipe = 4 * n_e2e       # long enough that filling and draining the pipeline is a small part
 
         def pipeline(n):
             pipe.run(host_in, step, n)
