@@ -289,6 +289,12 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
     for (uint32_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
         const uint32_t t = blk / n_heads, h = blk % n_heads;
         int lo = 0, hi = n_seqs;                              // sequence owning tile t
+        // when every sequence so far has exactly one tile (batches of merged short sequences), tile t belongs
+        // to sequence t: check that before paying for a binary search of dependent loads
+        if ((int)t < n_seqs && tile_prefix[t] <= t && tile_prefix[t + 1] > t) {
+            lo = (int)t;
+            hi = lo + 1;
+        }
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
             if (tile_prefix[mid] <= t) lo = mid; else hi = mid;
@@ -401,6 +407,12 @@ __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__
     for (uint32_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
         const uint32_t t = blk / n_heads, h = blk % n_heads;
         int lo = 0, hi = n_seqs;                              // sequence owning tile t
+        // when every sequence so far has exactly one tile (batches of merged short sequences), tile t belongs
+        // to sequence t: check that before paying for a binary search of dependent loads
+        if ((int)t < n_seqs && tile_prefix[t] <= t && tile_prefix[t + 1] > t) {
+            lo = (int)t;
+            hi = lo + 1;
+        }
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
             if (tile_prefix[mid] <= t) lo = mid; else hi = mid;
