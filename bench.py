@@ -194,13 +194,15 @@ def run_ours(args):
     runner = StreamRunner(max_tokens, max_seqs, H, d, causal, dev, value_seed=12 + 100 * rank)
 
     def flops_of(lengths):
-        f = 14.0 * sum(float(L) * L for L in lengths) * d * H
+        import numpy as np
+        ls = np.asarray(lengths, dtype=np.float64)
+        f = 14.0 * float((ls * ls).sum()) * d * H
         return 0.5 * f if causal else f
 
     def along_axis(mb):
         if axis is None:
             return mb
-        return MicroBatch(inputs.axis_lengths([inputs.clip_shape(L) for L in mb.lengths], axis), mb.recompute)
+        return MicroBatch(inputs.axis_lengths_array([inputs.clip_shape(L) for L in mb.lengths], axis), mb.recompute)
 
     profile, plan_kw = None, {}
     if args.plan == "profiled":

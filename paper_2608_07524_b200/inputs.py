@@ -104,6 +104,16 @@ def axis_lengths(clips, axis: str) -> List[int]:
     return out
 
 
+def axis_lengths_array(clips, axis: str):
+    """axis_lengths as an int32 numpy array, without a Python loop over the sequences."""
+    import numpy as np
+    if axis not in ("spatial", "temporal"):
+        raise ValueError("axis must be 'spatial' or 'temporal'")
+    f = np.fromiter((c[0] for c in clips), dtype=np.int32, count=len(clips))
+    s = np.fromiter((c[1] for c in clips), dtype=np.int32, count=len(clips))
+    return np.repeat(s, f) if axis == "spatial" else np.repeat(f, s)
+
+
 def short2d_lengths(axis: str, n: int = 24, seed: int = 3) -> List[int]:
     """axis_lengths of the config-3 clips."""
     return axis_lengths(video_clips(n, seed), axis)

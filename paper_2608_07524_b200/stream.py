@@ -12,17 +12,19 @@ from __future__ import annotations
 from dataclasses import dataclass
 from typing import List, Sequence
 
+import numpy as np
+
 from . import binding
 
 
 @dataclass
 class MicroBatch:
-    lengths: List[int]        # in planner order (longest first)
+    lengths: Sequence[int]    # in planner order (longest first); a list or an integer numpy array
     recompute: int            # layers whose forward is re-run before backward
 
     @property
     def total_tokens(self) -> int:
-        return sum(self.lengths)
+        return int(sum(self.lengths)) if isinstance(self.lengths, list) else int(self.lengths.sum())
 
 
 def plan_batch(lengths: Sequence[int], hbm_budget_bytes: int, n_heads: int, head_dim: int,
@@ -67,6 +69,7 @@ class StreamRunner:
         # only after the copy that read it has finished (tracked by an event per slot)
         self.n_slots = 16
         self.cu_host = torch.empty((self.n_slots, max_seqs + 1), dtype=torch.int32).pin_memory()
+        self.cu_host_np = self.cu_host.numpy()          # same memory: boundaries are written with numpy
         self.cu_dev = torch.empty((self.n_slots, max_seqs + 1), dtype=torch.int32, device=device)
         self.cu_events = [None] * self.n_slots
         self.calls = 0
@@ -74,14 +77,19 @@ class StreamRunner:
     def run_micro_batch(self, mb: MicroBatch) -> int:
         """Enqueue forward (+ recompute forward) + backward for one micro-batch; returns its tokens."""
         torch = self.torch
-        n, T = len(mb.lengths), mb.total_tokens
+        lens = np.asarray(mb.lengths, dtype=np.int32)
+        n = int(lens.size)
         slot = self.calls % self.n_slots
         self.calls += 1
         if self.cu_events[slot] is not None:
             self.cu_events[slot].synchronize()
+        # thousands of sequences per micro-batch are normal (a 2-D model's temporal axis): the host side of
+        # a step must stay well under the kernels' time, so no Python loop touches the lengths
+        cu_np = self.cu_host_np[slot, : n + 1]
+        cu_np[0] = 0
+        np.cumsum(lens, out=cu_np[1:])
+        T = int(cu_np[n])
         cu = self.cu_host[slot, : n + 1]
-        cu[0] = 0
-        cu[1:] = torch.tensor(mb.lengths, dtype=torch.int32).cumsum(0)
         cu_dev = self.cu_dev[slot, : n + 1]
         cu_dev.copy_(cu, non_blocking=True)
         ev = torch.cuda.Event()
@@ -89,7 +97,7 @@ class StreamRunner:
         self.cu_events[slot] = ev
         q, k, v, g, o = (x[:T] for x in (self.q, self.k, self.v, self.g, self.o))
         lse = self.lse[: self.H * T].view(self.H, T)
-        max_len = max(mb.lengths)
+        max_len = int(lens.max())
         for _ in range(1 + (1 if mb.recompute > 0 else 0)):
             binding.dcp_varlen_attn_fwd(q, k, v, cu_dev, max_len, self.causal, out=o, lse=lse, workspace=self.ws)
         binding.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cu_dev, max_len, self.causal, dq=self.dq[:T], dk=self.dk[:T],
