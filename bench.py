@@ -2,15 +2,17 @@
 """Benchmark of the packed variable-length attention hot path (plan -> forward -> backward).
 
     python bench.py [--gpus N] [--steps K] [--warmup W]
-                    [--workload video|text|extreme|stream|spatial2d|temporal2d]
+                    [--workload video|text|extreme|stream|spatial2d|temporal2d] [--order longest|input]
     python bench.py --impl reference ...        # the fp64 CPU oracle on a bounded sample
 
 One step = one pass of the whole path over one synthetic batch: dcp_plan on the batch's lengths,
-then for every micro-batch the work-list kernel, forward attention, and the three backward kernels
-(plus a second forward when the plan asks for recomputation).  Inputs are resident in HBM before
-the timed region; they are several times larger than L2, so no flush is needed between steps.
+then for every micro-batch the work-list kernels, forward attention, and the three backward kernels
+(plus a second forward when the plan asks for recomputation, and the gather / scatter copies when the
+plan splits the batch).  Inputs are resident in HBM before the timed region; they are several times
+larger than L2, so no flush is needed between steps.
 Prints one JSON line (rank 0).  Under torchrun every rank runs the same batch shape on its own GPU
-(weak scaling, no data-path collective); time is the max over ranks.
+(weak scaling, no data-path collective); time is the max over ranks.  At one GPU the line also
+carries, under "others", a few steps of every other workload, so that one run records them all.
 """
 from __future__ import annotations
 
@@ -26,10 +28,7 @@ sys.path.insert(0, ROOT)
 
 METRIC = "varlen_attn_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
-HBM_BUDGET = 180 * 10 ** 9
-# DRAM traffic (bytes) of one backward-main launch on config 3, from the ncu capture summarised under profiles/:
-# 3.201 GB measured by ncu on the 78192-token subset, scaled by tokens (traffic is proportional to them).
-BWD_MAIN_DRAM_BYTES_PER_LAUNCH = {"video": 3.201e9 * 124992 / 78192}
+WORKLOADS = ["video", "text", "extreme", "stream", "spatial2d", "temporal2d"]
 
 
 def load_peaks():
@@ -41,6 +40,18 @@ def load_peaks():
                 "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
     except Exception:
         return {"burst": 1590.0, "sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+def load_dram_traffic(workload: str):
+    """DRAM bytes one backward-main launch moves on this workload, as a profiler capture measured them
+    (a small case scaled by tokens where the full one is too large to capture), or None if no capture of
+    the current kernel is on record."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
+            entry = json.load(f)["bwd_main"].get(workload)
+        return float(entry["bytes_per_launch"]) if entry and not entry.get("stale") else None
+    except Exception:
+        return None
 
 
 class ClockSampler(threading.Thread):
@@ -147,12 +158,140 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------ CUDA arm
+class Job:
+    """One workload set up for timing: its batches, a runner holding them on the device, and `step`."""
+
+    def __init__(self, args, name: str, dev, rank: int, shuffle: bool = False):
+        import numpy as np
+        from paper_2608_07524_b200 import inputs
+        from paper_2608_07524_b200.stream import StreamRunner
+        self.args, self.workload = args, name
+        self.axis = None
+        if name == "stream":
+            self.batches = inputs.stream_batches()[: args.stream_batches]
+            self.H, self.d, self.causal = 16, 128, False
+            self.desc = (f"stream: {len(self.batches)} batches of the video length mix, Lambda={args.layers}, "
+                         f"budget {args.budget_gb} GB")
+        elif name in ("spatial2d", "temporal2d"):
+            # the paper's second architecture attends along one axis of a clip at a time: the planner sees the
+            # clips, the kernels see one sequence per latent frame (spatial) or per spatial position (temporal)
+            self.axis = name[:-2]
+            clips = inputs.video_clips()
+            self.batches, self.H, self.d, self.causal = [[f * s for f, s in clips]], 16, args.head_dim, False
+            seqs = inputs.axis_lengths(clips, self.axis)
+            self.n_axis_seqs = len(seqs)
+            self.desc = (f"config-3 clips, {self.axis} axis of a 2-D model: {len(seqs)} sequences of {min(seqs)}-{max(seqs)} "
+                         f"tokens, {sum(seqs)} tokens, 16 heads, head_dim {self.d}, bidirectional")
+        else:
+            w = workload(name)
+            lengths = [L for L in w.lengths if not args.drop_longer_than or L <= args.drop_longer_than]
+            if args.longest_last:
+                lengths = sorted(lengths)              # the hardest order for a scheduler that takes sequences as they come
+            self.batches, self.H, self.d, self.causal = [lengths], w.n_heads, w.head_dim, w.causal
+            self.desc = {"video": "config 3 video-DiT-like: 24 sequences, 124992 tokens, 16 heads, head_dim 128, bidirectional",
+                         "text": "config 2 text-like: 32 sequences, 79299 tokens, 16 heads, head_dim 128, causal",
+                         "extreme": "config 4 extreme imbalance: 131072 + 64 short, 206646 tokens, 8 heads, head_dim 128, causal"}[name]
+            if args.drop_longer_than:
+                self.desc += f" (profiling subset: sequences longer than {args.drop_longer_than} dropped)"
+            if args.longest_last:
+                self.desc += " (packed shortest first, the longest sequence last)"
+        self.budget = int(args.budget_gb * 10 ** 9)
+        self.max_tokens = max(sum(b) for b in self.batches)
+        self.max_seqs = max(len(b) for b in self.batches) if self.axis is None else self.n_axis_seqs
+        self.value_seed = 12 + 100 * rank
+        self.dev = dev
+        self.runner = StreamRunner(self.max_tokens, self.max_seqs, self.H, self.d, self.causal, dev, value_seed=self.value_seed)
+        self.profile, self.plan_kw = None, {}
+        self.np = np
+
+    def use_profile(self):
+        # Section 3.5: measure t_f, t_b per length bucket on this GPU (second of two runs) and let the
+        # planner use the table instead of its L^2 stand-in; T_C is then in nanoseconds
+        from paper_2608_07524_b200.profiler import dual_layer_profile
+        buckets = sorted(set(L for b in self.batches for L in b))
+        if len(buckets) > 16:
+            buckets = [buckets[i * (len(buckets) - 1) // 15] for i in range(16)]
+        self.profile = dual_layer_profile(buckets, self.H, self.d, self.causal, device=self.dev)
+        self.plan_kw = dict(profile=self.profile, fixed_cost=self.args.fixed_cost_ns)
+        self.desc += f", planner fed by a {len(buckets)}-bucket dual-layer profile (T_C = {self.args.fixed_cost_ns} ns)"
+
+    def flops_of(self, lengths):
+        ls = self.np.asarray(lengths, dtype=self.np.float64)
+        f = 14.0 * float((ls * ls).sum()) * self.d * self.H
+        return 0.5 * f if self.causal else f
+
+    def along_axis(self, mb):
+        if self.axis is None:
+            return mb
+        from paper_2608_07524_b200 import inputs
+        from paper_2608_07524_b200.stream import MicroBatch
+        return MicroBatch(inputs.axis_lengths_array([inputs.clip_shape(int(L)) for L in mb.lengths], self.axis), mb.recompute,
+                          mb.seq_index, mb.seg)
+
+    def step(self, r=None):
+        from paper_2608_07524_b200.stream import plan_batch
+        r = self.runner if r is None else r
+        tokens, flops = 0, 0.0
+        for lengths in self.batches:
+            plan = plan_batch(lengths, self.budget, self.H, self.d, n_layers=self.args.layers, **self.plan_kw)
+            batch_tokens = int(sum(lengths))
+            for mb in plan.micro_batches:
+                mb = self.along_axis(mb)
+                tokens += r.run_micro_batch(mb, batch_tokens)
+                flops += self.flops_of(mb.lengths)
+        return tokens, flops
+
+    def sm_busy(self):
+        """Per persistent CTA, how long it was busy in the last forward and backward main launch: the spread
+        is the single-GPU imbalance (max / mean = 1 means every SM worked until the end)."""
+        from paper_2608_07524_b200 import binding as B
+        out = {}
+        for which, key in ((0, "fwd"), (1, "bwd_main")):
+            begin, end = B.dcp_read_cta_spans(self.runner.ws, which)
+            if begin.size == 0:
+                continue
+            busy = self.np.sort((end - begin).astype(self.np.float64)) / 1e6
+            span = float(end.max() - begin.min()) / 1e6
+            out[key] = {"ctas": int(busy.size), "min_ms": float(busy[0]), "median_ms": float(busy[busy.size // 2]),
+                        "max_ms": float(busy[-1]), "max_over_mean": float(busy[-1] / max(busy.mean(), 1e-12)),
+                        "idle_frac": float(1.0 - busy.mean() / max(span, 1e-12))}
+        return out
+
+
+def timed_steps(job, steps, warmup, barrier):
+    """(ms over `steps` steps, tokens, flops, launches, per-kernel profile) after `warmup` untimed steps."""
+    import torch
+    from paper_2608_07524_b200 import binding as B
+    for _ in range(warmup):
+        job.step()
+    job.runner.check()
+    B.dcp_profile_enable(True)
+    B.dcp_profile_read()
+    barrier()
+    launches0 = B.dcp_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    tokens = flops = 0
+    for _ in range(steps):
+        t, f = job.step()
+        tokens += t
+        flops += f
+    e1.record()
+    torch.cuda.synchronize()
+    ms_total = e0.elapsed_time(e1)
+    launches = B.dcp_launch_count() - launches0
+    barrier()
+    prof = B.dcp_profile_read()
+    B.dcp_profile_enable(False)
+    job.runner.check()
+    return ms_total, tokens, flops, launches, prof
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2608_07524_b200 import binding as B
-    from paper_2608_07524_b200 import inputs
-    from paper_2608_07524_b200.stream import HostPipeline, MicroBatch, StreamRunner, plan_batch
+    from paper_2608_07524_b200.stream import HostPipeline, StreamRunner
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -164,99 +303,27 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     B.lib()      # fail loudly here if libdcp.so is missing
+    B.dcp_set_work_order(args.order == "input")
 
-    axis = None
-    if args.workload == "stream":
-        batches = inputs.stream_batches()[: args.stream_batches]
-        H, d, causal = 16, 128, False
-        name = f"stream: {len(batches)} batches of the video length mix, Lambda={args.layers}, budget {args.budget_gb} GB"
-    elif args.workload in ("spatial2d", "temporal2d"):
-        # the paper's second architecture attends along one axis of a clip at a time: the planner sees the
-        # clips, the kernels see one sequence per latent frame (spatial) or per spatial position (temporal)
-        axis = args.workload[:-2]
-        clips = inputs.video_clips()
-        batches, H, d, causal = [[f * s for f, s in clips]], 16, args.head_dim, False
-        seqs = inputs.axis_lengths(clips, axis)
-        name = (f"config-3 clips, {axis} axis of a 2-D model: {len(seqs)} sequences of {min(seqs)}-{max(seqs)} tokens, "
-                f"{sum(seqs)} tokens, 16 heads, head_dim {d}, bidirectional")
-    else:
-        w = workload(args.workload)
-        lengths = [L for L in w.lengths if not args.drop_longer_than or L <= args.drop_longer_than]
-        batches, H, d, causal = [lengths], w.n_heads, w.head_dim, w.causal
-        name = {"video": "config 3 video-DiT-like: 24 sequences, 124992 tokens, 16 heads, head_dim 128, bidirectional",
-                "text": "config 2 text-like: 32 sequences, 79299 tokens, 16 heads, head_dim 128, causal",
-                "extreme": "config 4 extreme imbalance: 131072 + 64 short, 206646 tokens, 8 heads, head_dim 128, causal"}[args.workload]
-        if args.drop_longer_than:
-            name += f" (profiling subset: sequences longer than {args.drop_longer_than} dropped)"
-    budget = int(args.budget_gb * 10 ** 9)
-    max_tokens = max(sum(b) for b in batches)
-    max_seqs = max(len(b) for b in batches) if axis is None else len(seqs)
-    runner = StreamRunner(max_tokens, max_seqs, H, d, causal, dev, value_seed=12 + 100 * rank)
-
-    def flops_of(lengths):
-        import numpy as np
-        ls = np.asarray(lengths, dtype=np.float64)
-        f = 14.0 * float((ls * ls).sum()) * d * H
-        return 0.5 * f if causal else f
-
-    def along_axis(mb):
-        if axis is None:
-            return mb
-        return MicroBatch(inputs.axis_lengths_array([inputs.clip_shape(L) for L in mb.lengths], axis), mb.recompute)
-
-    profile, plan_kw = None, {}
+    job = Job(args, args.workload, dev, rank)
     if args.plan == "profiled":
-        # Section 3.5: measure t_f, t_b per length bucket on this GPU (second of two runs) and let the
-        # planner use the table instead of its L^2 stand-in; T_C is then in nanoseconds
-        from paper_2608_07524_b200.profiler import dual_layer_profile
-        buckets = sorted(set(L for b in batches for L in b))
-        if len(buckets) > 16:
-            buckets = [buckets[i * (len(buckets) - 1) // 15] for i in range(16)]
-        profile = dual_layer_profile(buckets, H, d, causal, device=dev)
-        plan_kw = dict(profile=profile, fixed_cost=args.fixed_cost_ns)
-        name += f", planner fed by a {len(buckets)}-bucket dual-layer profile (T_C = {args.fixed_cost_ns} ns)"
-
-    def step(r=None):
-        r = runner if r is None else r
-        tokens, flops = 0, 0.0
-        for lengths in batches:
-            for mb in plan_batch(lengths, budget, H, d, n_layers=args.layers, **plan_kw):
-                mb = along_axis(mb)
-                tokens += r.run_micro_batch(mb)
-                flops += flops_of(mb.lengths)
-        return tokens, flops
+        job.use_profile()
+    H, d, causal, max_tokens, max_seqs = job.H, job.d, job.causal, job.max_tokens, job.max_seqs
+    runner, step, axis, desc = job.runner, job.step, job.axis, job.desc
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(physical_gpu_index(local))
     for _ in range(args.warmup):
         step()
     runner.check()
-
-    sampler = ClockSampler(physical_gpu_index(local))
-    B.dcp_profile_enable(True)
-    B.dcp_profile_read()
-    barrier()
     sampler.start()
-    launches0 = B.dcp_launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    tokens = flops = 0
-    for _ in range(args.steps):
-        t, f = step()
-        tokens += t
-        flops += f
-    e1.record()
-    torch.cuda.synchronize()
-    ms_total = e0.elapsed_time(e1)
-    launches = B.dcp_launch_count() - launches0
-    barrier()
+    ms_total, tokens, flops, launches, prof = timed_steps(job, args.steps, 0, barrier)
     clocks = sampler.stop()
-    prof = B.dcp_profile_read()
-    B.dcp_profile_enable(False)
-    runner.check()
+    sm_busy = job.sm_busy()
 
     t_ms = torch.tensor([ms_total], dtype=torch.float64, device=dev)
     totals = torch.tensor([flops, float(tokens)], dtype=torch.float64, device=dev)
@@ -348,14 +415,13 @@ def run_ours(args):
 
     peaks = load_peaks()
     bwd_ms, bwd_n = prof["bwd_main"]
-    fwd_ms, fwd_n = prof["fwd"]
     bwd_flops_per_launch = (flops / args.steps) * (2.5 / 3.5) / max(bwd_n / args.steps, 1)
     achieved = bwd_flops_per_launch / (bwd_ms / max(bwd_n, 1) * 1e-3) / 1e12 if bwd_n else None
+    plain = not args.drop_longer_than and args.layers == 1 and not args.longest_last and args.order == "longest"
     roofline = {"bound": "tensor", "kernel": "attn_bwd_kernel (backward main)", "achieved": achieved,
                 "peak": peaks["sustained"], "unit": UNIT, "frac": (achieved / peaks["sustained"]) if achieved else None,
                 "peak_source": f"bf16_tflops_sustained of {peaks['source']} MEASURED_PEAKS.json",
-                "traffic": (BWD_MAIN_DRAM_BYTES_PER_LAUNCH.get(args.workload)
-                            if not args.drop_longer_than and args.layers == 1 else None),
+                "traffic": load_dram_traffic(args.workload) if plain else None,
                 "launches": bwd_n, "avg_launch_ms": bwd_ms / max(bwd_n, 1)}
     if axis == "temporal" and bwd_n:
         # sequences of 1-13 tokens: a tile pair does ~1 % useful arithmetic, the kernel is bound by HBM.
@@ -366,8 +432,34 @@ def run_ours(args):
         roofline = {"bound": "hbm", "kernel": "attn_bwd_kernel (backward main)", "achieved": gbs, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                     "peak_source": f"hbm_gbs of {peaks['source']} MEASURED_PEAKS.json",
-                    "traffic": 3.758e9,        # ncu, one launch of this workload (summary under profiles/)
+                    "traffic": load_dram_traffic("temporal2d") if d == 128 else None,
                     "launches": bwd_n, "avg_launch_ms": bwd_ms / bwd_n}
+
+    # ---- a few steps of every other workload, so that one run records them all (single GPU only)
+    others = None
+    if world == 1 and not args.no_others:
+        others = {}
+        del job, runner, step
+        torch.cuda.empty_cache()
+        for name in WORKLOADS:
+            if name == args.workload:
+                continue
+            o_args = argparse.Namespace(**vars(args))
+            o_args.drop_longer_than, o_args.longest_last = 0, False
+            o_args.layers, o_args.budget_gb, o_args.stream_batches, o_args.head_dim = 1, 180.0, 32, 128
+            try:
+                oj = Job(o_args, name, dev, rank)
+                n_steps = 2 if name in ("stream", "extreme") else 5
+                ms, tok, fl, _, pr = timed_steps(oj, n_steps, 3 if name != "stream" else 1, barrier)
+                v = fl / (ms * 1e-3) / 1e12
+                others[name] = {"workload": oj.desc, "steps": n_steps, "ms_per_step": ms / n_steps, "value": v, "unit": UNIT,
+                                "tokens_per_s": tok / (ms * 1e-3), "frac_of_bf16_peak_burst": v / peaks["burst"],
+                                "kernel_ms_per_step": {k: x[0] / n_steps for k, x in pr.items()},
+                                "sm_busy": oj.sm_busy()}
+                del oj
+            except Exception as ex:
+                others[name] = {"error": str(ex)[:200]}
+            torch.cuda.empty_cache()
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
@@ -381,13 +473,15 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": name, "l2": "inputs (2 GB+) larger than L2, no flush", "hbm_budget_bytes": budget,
-                   "n_layers": args.layers},
+        "config": {"workload": desc, "l2": "inputs (2 GB+) larger than L2, no flush",
+                   "hbm_budget_bytes": int(args.budget_gb * 10 ** 9), "n_layers": args.layers, "work_order": args.order},
         "tokens_per_s": tokens_all / (ms_total * 1e-3),
         "frac_of_bf16_peak": {"burst": value / world / peaks["burst"], "sustained": value / world / peaks["sustained"],
                               "source": peaks["source"]},
         "kernel_ms_per_step": {k: v[0] / args.steps for k, v in prof.items()},
+        "sm_busy": sm_busy,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu_baseline,
+        "others": others,
     }
     print(json.dumps(line), flush=True)
     if world > 1:
@@ -400,8 +494,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="video",
-                    choices=["video", "text", "extreme", "stream", "spatial2d", "temporal2d"])
+    ap.add_argument("--workload", default="video", choices=WORKLOADS)
     ap.add_argument("--head-dim", type=int, default=128,
                     help="head dimension of the 2-D workloads (the paper's second model has 72)")
     ap.add_argument("--stream-batches", type=int, default=256)
@@ -410,7 +503,12 @@ def main():
                     help="planner's forward-time source: the L^2 model or a dual-layer profile measured first")
     ap.add_argument("--fixed-cost-ns", type=int, default=20000, help="T_C per micro-batch for --plan profiled")
     ap.add_argument("--budget-gb", type=float, default=180.0, help="planner's HBM budget in decimal GB")
+    ap.add_argument("--order", default="longest", choices=["longest", "input"],
+                    help="work order of the kernels: longest sequence first (the default) or as the sequences come")
+    ap.add_argument("--longest-last", action="store_true",
+                    help="pack the batch shortest first (with --order input: what the length-aware order is worth)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-others", action="store_true", help="skip the short runs of the other workloads")
     ap.add_argument("--drop-longer-than", type=int, default=0,
                     help="profiling aid: drop sequences longer than this from the workload (0 = keep all)")
     args = ap.parse_args()

@@ -81,6 +81,82 @@ int dcp_plan_profiled(const int32_t* lengths, const int64_t* fwd_time, int32_t n
                       const dcp_plan_params* params, int32_t* mb_id, int32_t* n_mb, int32_t* recompute,
                       int64_t* cost);
 
+/* A candidate of dcp_intra_select (described there). */
+typedef struct {
+    int32_t batch_size; /* b >= 1 */
+    int32_t sp_size;    /* p >= 1 */
+    int64_t t_f;        /* >= 0, any integer time unit */
+    int64_t m;          /* >= 0, bytes */
+    int64_t time_full;  /* T_(b,p) >= 1, same unit as t_f */
+    int64_t mem_full;   /* M_(b,p) >= 0, bytes */
+} dcp_intra_candidate;
+
+/* Data layout of a planned batch.
+ *
+ * Paper: Section 3.1 (the settings chosen for an incoming batch are applied to that batch's data:
+ * its sequences are regrouped into the micro-batches the plan names).  The batch's tensors hold the
+ * sequences packed in input order; micro-batch k gets its own packed tensors holding, in input
+ * order, the sequences i with mb_id[i] == k.  This call turns (lengths, mb_id) into what the copies
+ * and the attention calls need.  Host pointers; nothing touches a device.  Outputs:
+ *   mb_seq_offset [n_mb + 1]  micro-batch k owns entries mb_seq_offset[k] .. mb_seq_offset[k+1]-1 of seq_index
+ *   seq_index [n]             input index of every entry
+ *   mb_cu [n + n_mb]          micro-batch k's boundary array (its cu_seqlens, starting at 0) occupies
+ *                             mb_cu[mb_seq_offset[k] + k ...], one entry more than it has sequences
+ *   seg_offset [n_mb + 1], seg [3 * seg_capacity], *n_seg
+ *                             micro-batch k's copy list is seg[3*seg_offset[k] .. 3*seg_offset[k+1]): triples
+ *                             (first row in the batch, first row in the micro-batch, rows), each at most
+ *                             max_rows rows (long sequences are cut so that a copy kernel's CTAs get
+ *                             pieces of similar size) - the form dcp_copy_segments takes.
+ * lengths may contain zeros.  If seg_capacity is too small the call returns DCP_ERR_WORKSPACE with
+ * *n_seg set to the number needed (n + sum(lengths) / max_rows always suffices). */
+int dcp_plan_segments(const int32_t* lengths, const int32_t* mb_id, int32_t n, int32_t n_mb, int32_t max_rows,
+                      int32_t* mb_seq_offset, int32_t* seq_index, int32_t* mb_cu, int32_t* seg_offset, int32_t* seg,
+                      int32_t seg_capacity, int32_t* n_seg);
+
+/* Copies row ranges between two device tensors on `cuda_stream` (enqueue only): the gather of a
+ * micro-batch's sequences out of a batch and the scatter of its results back (Section 3.1, as above).
+ * seg: device int32 [n_seg][3] = (a, b, rows).  reverse == 0: rows b.. of dst = rows a.. of src;
+ * reverse != 0: rows a.. of dst = rows b.. of src.  A row is row_bytes bytes (a multiple of 4; 16-byte
+ * multiples with 16-byte aligned tensors take the fast path).  n_planes > 1 repeats the copy for planes
+ * src_plane_bytes / dst_plane_bytes apart: lse [n_heads, T] is n_heads planes of 4-byte rows.  Ranges
+ * must lie inside both tensors and must not overlap in dst; nothing checks that. */
+int dcp_copy_segments(const void* src, void* dst, const int32_t* seg, int32_t n_seg, int64_t row_bytes,
+                      int32_t n_planes, int64_t src_plane_bytes, int64_t dst_plane_bytes, int32_t reverse,
+                      void* cuda_stream);
+
+/* Profiled times between the profiled lengths.
+ *
+ * Paper: Section 3.5 measures t_f, t_b per candidate; it does not say how a length between two
+ * profiled ones is handled.  Here: bucket_len [n_buckets] strictly ascending, bucket_val the measured
+ * per-sequence value (any integer unit, >= 0).  For a length L: below the first bucket linear in L
+ * (val_0 * L / len_0: short sequences are bound by memory traffic); between two buckets linear; above
+ * the last quadratic (val_last * L^2 / len_last^2: attention time).  Floor division throughout.
+ * Host pointers; out [n]. */
+int dcp_profile_interp(const int32_t* bucket_len, const int64_t* bucket_val, int32_t n_buckets, const int32_t* lengths,
+                       int32_t n, int64_t* out);
+
+/* Modelled time of one micro-batch, Eq. 4-5: Lambda * (sum t_f + sum t_b) + r * sum t_f + T_C, from
+ * the per-sequence per-layer times fwd_time, bwd_time [n] (host). */
+int dcp_model_time(const int64_t* fwd_time, const int64_t* bwd_time, int32_t n, int32_t n_layers, int32_t recompute,
+                   int64_t fixed_cost, int64_t* time);
+
+/* One row of the candidate table Algorithm 1 takes, from a dual-layer measurement (Section 3.5: the
+ * profile runs with every layer recomputed and the model is extrapolated as
+ * T_(b,p) = Lambda * (2 t_f + t_b) + T_C; Eq. 6 at r = Lambda gives M_(b,p) = Lambda * m_inp + M_C).
+ * t_f, t_b: measured forward / backward time of one layer for the whole candidate batch; act_bytes = m,
+ * what one layer keeps when it is not recomputed; inp_bytes = m_inp. */
+int dcp_intra_candidate_from_profile(int32_t batch_size, int32_t sp_size, int64_t t_f, int64_t t_b, int64_t act_bytes,
+                                     int64_t inp_bytes, int32_t n_layers, int64_t const_bytes, int64_t fixed_cost,
+                                     dcp_intra_candidate* out);
+
+/* Which rank owns which sequence when a batch is sharded over world_size GPUs without any
+ * data-path collective (every (sequence, head) is independent).
+ *
+ * Paper: Section 2.3 (imbalance across devices comes from sequence length; attention cost grows with
+ * L^2).  Sequences are dealt longest first (ties by index) to the rank with the least accumulated
+ * L^2 (lowest rank on ties).  Host pointers; rank_of [n]; load [world_size] (nullable) = sum of L^2. */
+int dcp_shard_sequences(const int32_t* lengths, int32_t n, int32_t world_size, int32_t* rank_of, int64_t* load);
+
 /* DCP-intra: batch size, sequence-parallel size and recompute count for one sequence length.
  *
  * Paper: Section 3.4, Eq. 4-6 and Algorithm 1.  Each candidate (b, p) carries what the dual-layer
@@ -96,15 +172,6 @@ int dcp_plan_profiled(const int32_t* lengths, const int64_t* fwd_time, int32_t n
  * Candidates with M_(b,p) > capacity are skipped; none left => DCP_ERR_INFEASIBLE.
  * Host pointers; outputs *best (index), *recompute (r), time (nullable).  On one GPU every p is 1;
  * the function itself does not touch a device. */
-typedef struct {
-    int32_t batch_size; /* b >= 1 */
-    int32_t sp_size;    /* p >= 1 */
-    int64_t t_f;        /* >= 0, any integer time unit */
-    int64_t m;          /* >= 0, bytes */
-    int64_t time_full;  /* T_(b,p) >= 1, same unit as t_f */
-    int64_t mem_full;   /* M_(b,p) >= 0, bytes */
-} dcp_intra_candidate;
-
 int dcp_intra_select(const dcp_intra_candidate* cands, int32_t n, int64_t mem_capacity, int32_t n_layers,
                      int32_t* best, int32_t* recompute, int64_t* time);
 
@@ -137,6 +204,7 @@ int dcp_inter_plan(const int64_t* times, int32_t n, int32_t g_min, int32_t g_max
  * cu_seqlens is checked on the device (it must start at 0, never decrease, end at total_tokens, and
  * fit the workspace that max_seqlen promised): if it does not hold, the call computes nothing,
  * leaves the outputs as they were and dcp_query_status returns DCP_ERR_INVALID_ARG.
+ * The workspace needs no initialisation and may be reused by any number of calls on one stream.
  */
 
 /* Bytes of caller-provided device workspace needed by the forward and the backward call: the work
@@ -146,7 +214,7 @@ int dcp_varlen_attn_workspace(int32_t total_tokens, int32_t n_seqs, int32_t n_he
                               size_t* fwd_bytes, size_t* bwd_bytes);
 
 /* q, k, v (device, in) -> o, lse (device, out).  workspace: device, >= fwd_bytes, 256-byte
- * aligned; its first word is a status word that dcp_query_status reads. */
+ * aligned; its first word is a status word that dcp_query_status reads and clears. */
 int dcp_varlen_attn_fwd(const void* q, const void* k, const void* v, const int32_t* cu_seqlens, int32_t n_seqs,
                         int32_t total_tokens, int32_t max_seqlen, int32_t n_heads, int32_t head_dim,
                         int32_t causal, float softmax_scale, void* o, float* lse, void* workspace,
@@ -167,7 +235,7 @@ int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, const void*
  * real-time loop, a plug-in handed fixed buffers by its host program, a process whose allocator is
  * locked down after start-up).  Same operation, arguments, layouts and error codes as
  * dcp_varlen_attn_fwd, but the work-list scratch is a fixed array inside the library's device
- * image (about 66 KB, held by every GPU that loads the library until the process exits) instead of
+ * image (about 74 KB, held by every GPU that loads the library until the process exits) instead of
  * a caller buffer.  Limits and rules:
  *   - runs of very short sequences are not merged into shared tiles here (the table that needs grows
  *     with the token count), so such batches run slower than through dcp_varlen_attn_fwd; results
@@ -179,17 +247,41 @@ int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, const void*
  *   - all calls on a device share the one array, which keeps the previous call's contents; the
  *     library re-initialises what it needs at the start of every call, but two calls whose kernels
  *     may overlap on the GPU (different streams) race on it - serialise them;
- *   - the device status word of this variant lives in that array and is not readable through
- *     dcp_query_status; the kernels' waits are bounded all the same. */
+ *   - the device status word of this variant lives in that array: dcp_noalloc_status reads it. */
 #define DCP_NOALLOC_MAX_SEQS 4096
 int dcp_varlen_attn_fwd_noalloc(const void* q, const void* k, const void* v, const int32_t* cu_seqlens, int32_t n_seqs,
                                 int32_t total_tokens, int32_t max_seqlen, int32_t n_heads, int32_t head_dim,
                                 int32_t causal, float softmax_scale, void* o, float* lse, void* cuda_stream);
 
-/* Synchronises `cuda_stream`, then reads the status word at the start of `workspace`.
+/* dcp_query_status for the built-in array of dcp_varlen_attn_fwd_noalloc on the current device
+ * (synchronises `cuda_stream`, reports and clears).  It allocates nothing either. */
+int dcp_noalloc_status(void* cuda_stream);
+
+/* Synchronises `cuda_stream`, then reads the status word at the start of `workspace`.  The word is
+ * sticky on the device: it keeps the most severe failure of ANY call made on this workspace since the
+ * previous query, and this call clears it after reporting.
  * Returns DCP_OK, DCP_ERR_TIMEOUT (a kernel abandoned a bounded wait; results are invalid),
- * DCP_ERR_INVALID_ARG (cu_seqlens was inconsistent; nothing was computed) or DCP_ERR_CUDA. */
-int dcp_query_status(const void* workspace, void* cuda_stream);
+ * DCP_ERR_INVALID_ARG (cu_seqlens was inconsistent; that call computed nothing) or DCP_ERR_CUDA. */
+int dcp_query_status(void* workspace, void* cuda_stream);
+
+/* Self-test of the bounded-wait path (no counterpart in the paper).  Every device-side wait of this
+ * library gives up after a poll limit, raises the workspace's status word and lets its CTA run to the
+ * end instead of hanging the GPU.  This call enqueues one tiny CTA that waits, with that same helper and
+ * a limit of `spin_limit` polls (at most 2^20), on a barrier nothing ever arrives at, and then returns
+ * normally; dcp_query_status(workspace) must afterwards report DCP_ERR_TIMEOUT.  It never traps.
+ * workspace: device, at least 256 bytes, 256-byte aligned. */
+int dcp_selftest_wait_timeout(void* workspace, uint32_t spin_limit, void* cuda_stream);
+
+/* Measurement aids for the work order (no counterpart in the paper beyond the problem itself:
+ * Section 2.3's imbalance, which on one GPU shows as SMs idling while one long sequence finishes).
+ * dcp_set_work_order(1) makes later calls list sequences as they come instead of longest first;
+ * dcp_set_work_order(0) restores the default.  Process-wide.
+ * dcp_read_cta_spans synchronises `cuda_stream` and returns, for the last forward (which = 0) or
+ * backward main (which = 1) launch on `workspace`, when each persistent CTA started and when it ran
+ * out of work, in nanoseconds of the GPU's global timer: begin_ns, end_ns [256] (host), *n_ctas valid. */
+int dcp_set_work_order(int input_order);
+int dcp_read_cta_spans(const void* workspace, int32_t which, void* cuda_stream, int64_t* begin_ns, int64_t* end_ns,
+                       int32_t* n_ctas);
 
 /* Measurement aid (no counterpart in the paper).  While enabled, every attention call records a
  * pair of CUDA events around each kernel it launches, on the caller's stream.  dcp_profile_read

@@ -223,3 +223,4 @@ def inter_bruteforce(times, g_min: int = 1, g_max: int = 4):
 
 
 from .intra_oracle import intra_select  # noqa: E402,F401  (Algorithm 1, plain Python)
+from . import profile_oracle, shard_oracle  # noqa: E402,F401

@@ -1,21 +1,29 @@
-"""Oracle for the DCP-intra selection (Algorithm 1 of the paper, Section 3.4).
+"""Oracle for the DCP-intra selection (Section 3.4, Algorithm 1, Eq. 1 and Eq. 4-6 of the paper).
 
-TEST INFRASTRUCTURE ONLY: plain Python, exact rational arithmetic, the algorithm's steps in the
-paper's order and notation.
+TEST INFRASTRUCTURE ONLY: plain Python, exact rational arithmetic, exhaustive search.
 
-Input: memory capacity M, model layers L, candidates C = {(b, p): (t_f, m, T_(b,p), M_(b,p))} from a
-profile taken with every layer recomputed.  For each candidate the algorithm lets as many layers as
-the spare memory allows keep their activations (each costs m bytes more and saves t_f), takes the
-resulting time, and keeps the best candidate.
+What is selected.  Every candidate setting (batch size b, sequence-parallel size p) comes with four
+profiled numbers taken with ALL layers recomputed: the forward time of one layer, the bytes one
+layer keeps when it is not recomputed, the iteration time and the memory footprint.  Switching
+recomputation off for `kept` of the n_layers layers adds kept * bytes_per_layer to the footprint
+(Eq. 6) and removes kept * layer_fwd_time from the time (Eq. 5).  The selection is the pair
+(candidate, kept) with the highest throughput b / (p * time) (Eq. 1) among all pairs whose
+footprint stays within the capacity; the recompute count reported is n_layers - kept.
 
-Readings (the listing and the text disagree in two places):
-  * the listing's inner loop breaks at the first layer count whose memory fits, which would always
-    stop at one layer; its comment ("minimal recompute layer with spare GPU memory") and Section 3.4
-    ("computes the minimal r_i under the GPU memory capacity") ask for the largest count of
-    non-recomputed layers that still fits.  The loop below therefore runs while the memory fits;
-  * the listing keeps the candidate with the smallest time, the text ("compare the throughput
-    according to Equation 1") the one with the highest b / (p * time); they agree when b and p are
-    equal.  The text is followed.  Ties (the paper gives none): smaller p, larger b, earlier candidate.
+This file does not walk the candidates the way the paper's listing does.  It enumerates every
+(candidate, kept) pair with kept = 0 .. n_layers, discards those that do not fit, and takes the
+maximum, so that no early exit or closed form can hide a mistake.  For one candidate the time falls
+as kept grows, hence the best pair of a candidate is the one with the most layers kept, which is
+the smallest recompute count that fits: the quantity Section 3.4's text asks for.
+
+Two readings (paper silent or at odds with itself):
+  * taken literally, the listing's inner loop leaves at the first layer count that fits, i.e. it
+    would never keep more than one layer; the accompanying text asks for the smallest recompute
+    count under the capacity, which is what the maximum over all pairs yields;
+  * the listing compares raw times across candidates, the text throughput; the two agree when b and
+    p are equal, and throughput is used here.
+Ties (the paper states none): higher throughput, then smaller p, larger b, earlier candidate, and
+among equal pairs of one candidate (zero layer time) the one keeping more layers.
 """
 from fractions import Fraction
 
@@ -24,25 +32,16 @@ class Infeasible(Exception):
     pass
 
 
-def intra_select(candidates, M: int, L: int):
-    """candidates: list of (b, p, t_f, m, T_bp, M_bp).  Returns (index, recompute layers r, time)."""
-    best_key = None
-    result = None
-    for idx, (b, p, t_f, m, T_bp, M_bp) in enumerate(candidates):
-        if M_bp > M:
-            continue
-        keep = 0
-        for layers in range(1, L + 1):          # layers whose recomputation is switched off
-            M_opt = M_bp + layers * m
-            if M_opt > M:
-                break
-            keep = layers
-        cur_time = T_bp - keep * t_f
-        throughput = Fraction(b, p * cur_time)
-        key = (throughput, -p, b, -idx)
-        if best_key is None or key > best_key:
-            best_key = key
-            result = (idx, L - keep, cur_time)
-    if result is None:
+def intra_select(candidates, capacity: int, n_layers: int):
+    """candidates: (b, p, layer_fwd_time, bytes_per_layer, time_all_recomputed, bytes_all_recomputed).
+    Returns (index, recompute count, time)."""
+    pairs = []
+    for index, (b, p, layer_fwd_time, bytes_per_layer, time_all, bytes_all) in enumerate(candidates):
+        for kept in range(n_layers + 1):
+            if bytes_all + kept * bytes_per_layer > capacity:
+                continue
+            time = time_all - kept * layer_fwd_time
+            pairs.append(((Fraction(b, p * time), -p, b, -index, kept), (index, n_layers - kept, time)))
+    if not pairs:
         raise Infeasible()
-    return result
+    return max(pairs, key=lambda pair: pair[0])[1]

@@ -72,6 +72,27 @@ def lib():
             L.dcp_varlen_attn_fwd_noalloc.restype = ctypes.c_int
             L.dcp_query_status.argtypes = [vp, vp]
             L.dcp_query_status.restype = ctypes.c_int
+            L.dcp_noalloc_status.argtypes = [vp]
+            L.dcp_noalloc_status.restype = ctypes.c_int
+            L.dcp_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint32, vp]
+            L.dcp_selftest_wait_timeout.restype = ctypes.c_int
+            L.dcp_set_work_order.argtypes = [ctypes.c_int]
+            L.dcp_set_work_order.restype = ctypes.c_int
+            L.dcp_read_cta_spans.argtypes = [vp, i32, vp, i64p, i64p, i32p]
+            L.dcp_read_cta_spans.restype = ctypes.c_int
+            L.dcp_plan_segments.argtypes = [i32p, i32p, i32, i32, i32, i32p, i32p, i32p, i32p, i32p, i32, i32p]
+            L.dcp_plan_segments.restype = ctypes.c_int
+            L.dcp_copy_segments.argtypes = [vp, vp, vp, i32, i64, i32, i64, i64, i32, vp]
+            L.dcp_copy_segments.restype = ctypes.c_int
+            L.dcp_profile_interp.argtypes = [i32p, i64p, i32, i32p, i32, i64p]
+            L.dcp_profile_interp.restype = ctypes.c_int
+            L.dcp_model_time.argtypes = [i64p, i64p, i32, i32, i32, i64, i64p]
+            L.dcp_model_time.restype = ctypes.c_int
+            L.dcp_intra_candidate_from_profile.argtypes = [i32, i32, i64, i64, i64, i64, i32, i64, i64,
+                                                           ctypes.POINTER(IntraCandidate)]
+            L.dcp_intra_candidate_from_profile.restype = ctypes.c_int
+            L.dcp_shard_sequences.argtypes = [i32p, i32, i32, i32p, i64p]
+            L.dcp_shard_sequences.restype = ctypes.c_int
             L.dcp_profile_enable.argtypes = [ctypes.c_int]
             L.dcp_profile_enable.restype = ctypes.c_int
             L.dcp_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int64)]
@@ -255,5 +276,113 @@ def dcp_varlen_attn_bwd(q, k, v, o, d_o, lse, cu_seqlens, max_seqlen: int, causa
 
 
 def dcp_query_status(workspace, stream=None) -> None:
-    """Synchronises the stream and raises DcpError if a kernel reported a failure."""
+    """Synchronises the stream and raises DcpError if any call on this workspace since the previous
+    query reported a failure (the device status word is sticky; the query clears it)."""
     _check(lib().dcp_query_status(_ptr(workspace), _stream(stream)))
+
+
+def dcp_noalloc_status(stream=None) -> None:
+    """dcp_query_status for the built-in scratch of dcp_varlen_attn_fwd_noalloc on the current device."""
+    _check(lib().dcp_noalloc_status(_stream(stream)))
+
+
+def dcp_selftest_wait_timeout(workspace, spin_limit: int = 1 << 10, stream=None) -> None:
+    """Enqueues the self-test CTA whose bounded wait expires; dcp_query_status then raises DCP_ERR_TIMEOUT."""
+    _check(lib().dcp_selftest_wait_timeout(_ptr(workspace), int(spin_limit), _stream(stream)))
+
+
+def dcp_set_work_order(input_order: bool) -> None:
+    """Measurement aid: list sequences as they come (True) instead of longest first (False, default)."""
+    _check(lib().dcp_set_work_order(int(bool(input_order))))
+
+
+def dcp_read_cta_spans(workspace, which: int, stream=None):
+    """(begin_ns, end_ns) int64 numpy arrays, one entry per persistent CTA of the last forward (which = 0)
+    or backward main (which = 1) launch on this workspace."""
+    import numpy as np
+    begin = np.zeros(256, np.int64)
+    end = np.zeros(256, np.int64)
+    n = ctypes.c_int32(0)
+    i64p = ctypes.POINTER(ctypes.c_int64)
+    _check(lib().dcp_read_cta_spans(_ptr(workspace), int(which), _stream(stream), begin.ctypes.data_as(i64p),
+                                    end.ctypes.data_as(i64p), ctypes.byref(n)))
+    return begin[: n.value].copy(), end[: n.value].copy()
+
+
+def _i32(a):
+    import numpy as np
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _i32p(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+
+
+def _i64p(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_int64))
+
+
+def dcp_plan_segments(lengths, mb_id, n_mb: int, max_rows: int = 64):
+    """(mb_seq_offset [K+1], seq_index [n], mb_cu [n+K], seg_offset [K+1], seg [n_seg, 3]) as int32 numpy
+    arrays: where each sequence of a planned batch lives in the batch and in its micro-batch."""
+    import numpy as np
+    lengths, mb_id = _i32(lengths), _i32(mb_id)
+    n = int(lengths.size)
+    cap = n + int(lengths.sum()) // int(max_rows)
+    mb_seq_offset, seq_index = np.zeros(n_mb + 1, np.int32), np.zeros(max(n, 1), np.int32)
+    mb_cu, seg_offset = np.zeros(n + n_mb, np.int32), np.zeros(n_mb + 1, np.int32)
+    seg = np.zeros((max(cap, 1), 3), np.int32)
+    n_seg = ctypes.c_int32(0)
+    _check(lib().dcp_plan_segments(_i32p(lengths), _i32p(mb_id), n, int(n_mb), int(max_rows), _i32p(mb_seq_offset),
+                                   _i32p(seq_index), _i32p(mb_cu), _i32p(seg_offset), _i32p(seg), cap,
+                                   ctypes.byref(n_seg)))
+    return mb_seq_offset, seq_index[:n], mb_cu, seg_offset, seg[: n_seg.value]
+
+
+def dcp_copy_segments(src, dst, seg, n_seg: int, row_bytes: int, reverse: bool = False, n_planes: int = 1,
+                      src_plane_bytes: int = 0, dst_plane_bytes: int = 0, stream=None) -> None:
+    """Row-range copies between two CUDA tensors; seg is an int32 CUDA tensor [n_seg, 3].  Enqueues only."""
+    _check(lib().dcp_copy_segments(_ptr(src), _ptr(dst), _ptr(seg), int(n_seg), int(row_bytes), int(n_planes),
+                                   int(src_plane_bytes), int(dst_plane_bytes), int(bool(reverse)), _stream(stream)))
+
+
+def dcp_profile_interp(bucket_len, bucket_val, lengths) -> List[int]:
+    """Profiled per-sequence values at arbitrary lengths (Section 3.5; the rule is in include/dcp.h)."""
+    import numpy as np
+    xs, ys = _i32(bucket_len), np.ascontiguousarray(bucket_val, dtype=np.int64)
+    ls = _i32(lengths)
+    out = np.zeros(max(int(ls.size), 1), np.int64)
+    _check(lib().dcp_profile_interp(_i32p(xs), _i64p(ys), int(xs.size), _i32p(ls), int(ls.size), _i64p(out)))
+    return [int(x) for x in out[: ls.size]]
+
+
+def dcp_model_time(fwd_time, bwd_time, n_layers: int, recompute: int, fixed_cost: int = 0) -> int:
+    """Eq. 4-5 for one micro-batch: Lambda (sum t_f + sum t_b) + r sum t_f + T_C."""
+    import numpy as np
+    f, b = np.ascontiguousarray(fwd_time, dtype=np.int64), np.ascontiguousarray(bwd_time, dtype=np.int64)
+    if f.size != b.size:
+        raise ValueError("fwd_time and bwd_time need one entry per sequence each")
+    t = ctypes.c_int64(0)
+    _check(lib().dcp_model_time(_i64p(f), _i64p(b), int(f.size), int(n_layers), int(recompute), int(fixed_cost),
+                                ctypes.byref(t)))
+    return int(t.value)
+
+
+def dcp_intra_candidate_from_profile(batch_size: int, sp_size: int, t_f: int, t_b: int, act_bytes: int, inp_bytes: int,
+                                     n_layers: int, const_bytes: int = 0, fixed_cost: int = 0):
+    """(b, p, t_f, m, T_(b,p), M_(b,p)): one row of Algorithm 1's candidate table from a dual-layer measurement."""
+    c = IntraCandidate()
+    _check(lib().dcp_intra_candidate_from_profile(int(batch_size), int(sp_size), int(t_f), int(t_b), int(act_bytes),
+                                                  int(inp_bytes), int(n_layers), int(const_bytes), int(fixed_cost),
+                                                  ctypes.byref(c)))
+    return (c.batch_size, c.sp_size, c.t_f, c.m, c.time_full, c.mem_full)
+
+
+def dcp_shard_sequences(lengths, world_size: int):
+    """(rank_of [n], load [world_size]): longest-first assignment of sequences to ranks by accumulated L^2."""
+    import numpy as np
+    ls = _i32(lengths)
+    rank_of = np.zeros(max(int(ls.size), 1), np.int32)
+    load = np.zeros(max(int(world_size), 1), np.int64)
+    _check(lib().dcp_shard_sequences(_i32p(ls), int(ls.size), int(world_size), _i32p(rank_of), _i64p(load)))
+    return [int(x) for x in rank_of[: ls.size]], [int(x) for x in load]

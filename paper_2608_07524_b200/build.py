@@ -16,7 +16,8 @@ _DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_DIR, "csrc")
 OBJ_DIR = os.path.join(CSRC, "build")
 LIB_PATH = os.path.join(_DIR, "libdcp.so")
-SOURCES = ["api.cu", "plan.cpp", "inter.cpp", "intra.cpp", "prep.cu", "attn_fwd.cu", "attn_bwd.cu"]
+SOURCES = ["api.cu", "plan.cpp", "inter.cpp", "intra.cpp", "model.cpp", "prep.cu", "util_kernels.cu", "attn_fwd.cu",
+           "attn_bwd.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

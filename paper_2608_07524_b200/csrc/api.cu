@@ -26,30 +26,58 @@ char* error_buffer() {
 namespace {
 
 std::atomic<int64_t> g_launches{0};
+std::atomic<int> g_input_order{0};      // dcp_set_work_order: 1 = list sequences as they come
 
-// Optional per-kernel timing: event pairs recorded on the caller's stream around every launch.
+// Optional per-kernel timing: event pairs recorded on the caller's stream around every launch.  Events
+// are created once and recycled through a pool (dcp_profile_read hands them back), so that a timed
+// launch costs two event records and no create/destroy.
 struct TimedLaunch {
-    int kernel;
+    int kernel, device;
     cudaEvent_t start, stop;
 };
+constexpr int kMaxDevices = 64;
 std::mutex g_prof_mu;
 std::atomic<int> g_prof_on{0};
 std::vector<TimedLaunch> g_prof_pending;
+std::vector<cudaEvent_t> g_event_pool[kMaxDevices];      // an event belongs to the device it was created on
+
+cudaEvent_t pool_take(int device) {
+    {
+        std::lock_guard<std::mutex> lock(g_prof_mu);
+        std::vector<cudaEvent_t>& pool = g_event_pool[device];
+        if (!pool.empty()) {
+            cudaEvent_t e = pool.back();
+            pool.pop_back();
+            return e;
+        }
+    }
+    cudaEvent_t e = nullptr;
+    return cudaEventCreate(&e) == cudaSuccess ? e : nullptr;
+}
 
 struct ScopedTimer {
-    int kernel;
+    int kernel, device = 0;
     cudaStream_t stream;
     cudaEvent_t start = nullptr, stop = nullptr;
     ScopedTimer(int k, cudaStream_t s) : kernel(k), stream(s) {
         if (!g_prof_on.load()) return;
-        if (cudaEventCreate(&start) != cudaSuccess || cudaEventCreate(&stop) != cudaSuccess) { start = stop = nullptr; return; }
+        if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return;
+        start = pool_take(device);
+        stop = pool_take(device);
+        if (!start || !stop) {
+            std::lock_guard<std::mutex> lock(g_prof_mu);
+            if (start) g_event_pool[device].push_back(start);
+            if (stop) g_event_pool[device].push_back(stop);
+            start = stop = nullptr;
+            return;
+        }
         cudaEventRecord(start, stream);
     }
     ~ScopedTimer() {
         if (!start) return;
         cudaEventRecord(stop, stream);
         std::lock_guard<std::mutex> lock(g_prof_mu);
-        g_prof_pending.push_back({kernel, start, stop});
+        g_prof_pending.push_back({kernel, device, start, stop});
     }
 };
 
@@ -135,8 +163,10 @@ SchedView carve_sched(void* workspace, int32_t n_seqs) {
     SchedView s;
     uint8_t* base = static_cast<uint8_t*>(workspace);
     s.hdr = reinterpret_cast<WorkspaceHeader*>(base);
-    s.order = reinterpret_cast<const int32_t*>(base + sizeof(WorkspaceHeader));
-    s.prefix = reinterpret_cast<const uint32_t*>(base + sizeof(WorkspaceHeader) + sizeof(int32_t) * (size_t)n_seqs);
+    s.spans = reinterpret_cast<CtaSpan*>(base + sizeof(WorkspaceHeader));
+    base += sizeof(WorkspaceHeader) + kSpanBytes;
+    s.order = reinterpret_cast<const int32_t*>(base);
+    s.prefix = reinterpret_cast<const uint32_t*>(base + sizeof(int32_t) * (size_t)n_seqs);
     s.tile_prefix = s.prefix + (size_t)n_seqs + 1;
     s.vcu = reinterpret_cast<const int32_t*>(s.tile_prefix + (size_t)n_seqs + 1);
     s.n_seqs = n_seqs;
@@ -195,13 +225,14 @@ static int attn_fwd_impl(const char* fn, bool merge, const void* q, const void* 
     const SchedView sched = carve_sched(workspace, n_seqs);
     uint16_t* bounds = merge ? reinterpret_cast<uint16_t*>(static_cast<uint8_t*>(workspace) + sched_bytes(n_seqs)) : nullptr;
     cudaError_t e;
+    const bool input_order = g_input_order.load() != 0;
     {
         ScopedTimer t(DCP_KERNEL_PREP, stream);
         e = launch_prep(cu_seqlens, n_seqs, total_tokens, max_seqlen, kFwdRowsPerItem, n_heads, sched, bounds, UINT32_MAX,
-                        stream);
+                        input_order, stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: work-list kernel: %s", fn, cudaGetErrorString(e));
-    g_launches.fetch_add(prep_launches(n_seqs, merge));
+    g_launches.fetch_add(prep_launches(n_seqs, merge, input_order));
     if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
 
     CUtensorMap tq, tk, tv;
@@ -268,13 +299,14 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
     float* dq_acc = reinterpret_cast<float*>(base + align256(max_tiles(total_tokens, n_seqs) * n_heads * (size_t)(kTile * 16 * 2)));
 
     cudaError_t e;
+    const bool input_order = g_input_order.load() != 0;
     {
         ScopedTimer t(DCP_KERNEL_PREP, stream);
         e = launch_prep(cu_seqlens, n_seqs, total_tokens, max_seqlen, kTile, n_heads, sched, bounds,
-                        (uint32_t)max_tiles(total_tokens, n_seqs), stream);
+                        (uint32_t)max_tiles(total_tokens, n_seqs), input_order, stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: work-list kernel: %s", fn, cudaGetErrorString(e));
-    g_launches.fetch_add(prep_launches(n_seqs, true));
+    g_launches.fetch_add(prep_launches(n_seqs, true, input_order));
     const int32_t* vcu = sched.vcu;      // every later kernel works on the virtual sequences
     if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
 
@@ -328,13 +360,52 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
 // ---------------------------------------------------------------------------------------------
 // Forward attention for callers that cannot allocate device memory.
 //
-// The forward kernel needs scratch for its work list (header, sequence order, prefix sums).  Here
-// that scratch is a fixed array in the library's own device image, so the caller passes inputs and
-// outputs only.  Every GPU that loads this library holds the array until the process exits.
+// The forward kernel needs scratch for its work list (header, CTA time spans, sequence order, prefix
+// sums).  Here that scratch is a fixed array in the library's own device image, so the caller passes
+// inputs and outputs only.  Every GPU that loads this library holds the array until the process exits.
 #define DCP_NOALLOC_MAX_SEQS_VALUE 4096
 namespace {
 constexpr size_t kNoAllocScratchBytes = dcp::sched_bytes(DCP_NOALLOC_MAX_SEQS_VALUE);
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+// In host code the array's name is only a handle, not a device address: ask the runtime for the
+// address once per device, with that device current, and hand the kernels that pointer.  (The
+// address is cached per device index for the life of the process; a cudaDeviceReset in between
+// would make it stale.)
+int noalloc_scratch(const char* fn, void** out) {
+    static std::mutex mu;
+    static void* scratch_of_device[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
+        return fail(DCP_ERR_CUDA, "%s: cudaGetDevice failed or device index out of range", fn);
+    std::lock_guard<std::mutex> lock(mu);
+    if (!scratch_of_device[dev]) {
+        void* ptr = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+        if (e != cudaSuccess || !ptr) return fail(DCP_ERR_CUDA, "%s: cudaGetSymbolAddress: %s", fn, cudaGetErrorString(e));
+        scratch_of_device[dev] = ptr;
+    }
+    *out = scratch_of_device[dev];
+    return DCP_OK;
+}
+
+// Reads the status word at `status_word`, reports it and clears it (the word is sticky on the device).
+int report_status(void* status_word, cudaStream_t stream, const char* fn) {
+    uint32_t status = 0;
+    cudaError_t e = cudaMemcpyAsync(&status, status_word, sizeof status, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e == cudaSuccess && status != 0) {
+        e = cudaMemsetAsync(status_word, 0, sizeof status, stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    }
+    if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: %s", fn, cudaGetErrorString(e));
+    if (status == kStatusBadLengths)
+        return fail(DCP_ERR_INVALID_ARG,
+                    "cu_seqlens disagrees with n_seqs, total_tokens or max_seqlen (it must start at 0, never decrease, end "
+                    "at total_tokens, and no sequence may exceed max_seqlen); that call computed nothing");
+    if (status != 0) return fail(DCP_ERR_TIMEOUT, "a kernel abandoned a bounded wait (device status %u); results are invalid", status);
+    return DCP_OK;
+}
 }  // namespace
 
 extern "C" int dcp_varlen_attn_fwd_noalloc(const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
@@ -346,25 +417,8 @@ extern "C" int dcp_varlen_attn_fwd_noalloc(const void* q, const void* k, const v
         return fail(DCP_ERR_UNSUPPORTED, "%s: %d sequences exceed the built-in scratch (at most %d per call)", fn, n_seqs,
                     DCP_NOALLOC_MAX_SEQS_VALUE);
     if (n_seqs < 0) return fail(DCP_ERR_INVALID_ARG, "%s: negative n_seqs", fn);
-    // In host code the array's name is only a handle, not a device address: ask the runtime for the
-    // address once per device, with that device current, and hand the kernels that pointer.
-    static std::mutex mu;
-    static void* scratch_of_device[64] = {nullptr};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
-        return fail(DCP_ERR_CUDA, "%s: cudaGetDevice failed or device index out of range", fn);
     void* scratch = nullptr;
-    {
-        std::lock_guard<std::mutex> lock(mu);
-        if (!scratch_of_device[dev]) {
-            void* ptr = nullptr;
-            const cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
-            if (e != cudaSuccess || !ptr)
-                return fail(DCP_ERR_CUDA, "%s: cudaGetSymbolAddress: %s", fn, cudaGetErrorString(e));
-            scratch_of_device[dev] = ptr;
-        }
-        scratch = scratch_of_device[dev];
-    }
+    if (int rc = noalloc_scratch(fn, &scratch)) return rc;
     if (sched_bytes(n_seqs) > kNoAllocScratchBytes)      // cannot happen for n_seqs <= the maximum; kept as a guard
         return fail(DCP_ERR_UNSUPPORTED, "%s: built-in scratch too small", fn);
     // short sequences are not merged here: the table that needs is sized by the token count
@@ -372,18 +426,75 @@ extern "C" int dcp_varlen_attn_fwd_noalloc(const void* q, const void* k, const v
                          softmax_scale, o, lse, scratch, kNoAllocScratchBytes, cuda_stream);
 }
 
-extern "C" int dcp_query_status(const void* workspace, void* cuda_stream) {
+extern "C" int dcp_noalloc_status(void* cuda_stream) {
+    void* scratch = nullptr;
+    if (int rc = noalloc_scratch("dcp_noalloc_status", &scratch)) return rc;
+    return report_status(scratch, static_cast<cudaStream_t>(cuda_stream), "dcp_noalloc_status");
+}
+
+extern "C" int dcp_query_status(void* workspace, void* cuda_stream) {
     if (!workspace) return fail(DCP_ERR_INVALID_ARG, "dcp_query_status: workspace is null");
+    return report_status(workspace, static_cast<cudaStream_t>(cuda_stream), "dcp_query_status");
+}
+
+extern "C" int dcp_set_work_order(int input_order) {
+    g_input_order.store(input_order ? 1 : 0);
+    return DCP_OK;
+}
+
+extern "C" int dcp_read_cta_spans(const void* workspace, int32_t which, void* cuda_stream, int64_t* begin_ns,
+                                  int64_t* end_ns, int32_t* n_ctas) {
+    if (!workspace || !begin_ns || !end_ns || !n_ctas || which < 0 || which > 1)
+        return fail(DCP_ERR_INVALID_ARG, "dcp_read_cta_spans: null pointer or `which` not 0/1");
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    uint32_t status = 0;
-    cudaError_t e = cudaMemcpyAsync(&status, workspace, sizeof status, cudaMemcpyDeviceToHost, stream);
+    WorkspaceHeader hdr;
+    static_assert(sizeof(CtaSpan) == 16, "span is two 64-bit words");
+    std::vector<CtaSpan> spans(kMaxCtas);
+    const uint8_t* base = static_cast<const uint8_t*>(workspace);
+    cudaError_t e = cudaMemcpyAsync(&hdr, base, sizeof hdr, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(spans.data(), base + sizeof(WorkspaceHeader) + (size_t)which * kMaxCtas * sizeof(CtaSpan),
+                            kMaxCtas * sizeof(CtaSpan), cudaMemcpyDeviceToHost, stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
-    if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "dcp_query_status: %s", cudaGetErrorString(e));
-    if (status == kStatusBadLengths)
-        return fail(DCP_ERR_INVALID_ARG,
-                    "cu_seqlens disagrees with n_seqs, total_tokens or max_seqlen (it must start at 0, never decrease, end "
-                    "at total_tokens, and no sequence may exceed max_seqlen); nothing was computed");
-    if (status != 0) return fail(DCP_ERR_TIMEOUT, "a kernel abandoned a bounded wait (device status %u); results are invalid", status);
+    if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "dcp_read_cta_spans: %s", cudaGetErrorString(e));
+    if (hdr.magic[0] != kHeaderMagic0 || hdr.magic[1] != kHeaderMagic1 || hdr.n_ctas[which] > (uint32_t)kMaxCtas)
+        return fail(DCP_ERR_INVALID_ARG, "dcp_read_cta_spans: no attention call has run on this workspace");
+    *n_ctas = (int32_t)hdr.n_ctas[which];
+    for (int i = 0; i < *n_ctas; ++i) {
+        begin_ns[i] = (int64_t)spans[i].begin_ns;
+        end_ns[i] = (int64_t)spans[i].end_ns;
+    }
+    return DCP_OK;
+}
+
+extern "C" int dcp_selftest_wait_timeout(void* workspace, uint32_t spin_limit, void* cuda_stream) {
+    if (!workspace) return fail(DCP_ERR_WORKSPACE, "dcp_selftest_wait_timeout: workspace is null");
+    if (spin_limit > (1u << 20)) return fail(DCP_ERR_INVALID_ARG, "dcp_selftest_wait_timeout: spin_limit above 2^20");
+    const cudaError_t e = launch_wait_timeout_selftest(static_cast<WorkspaceHeader*>(workspace), spin_limit,
+                                                       static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "dcp_selftest_wait_timeout: %s", cudaGetErrorString(e));
+    g_launches.fetch_add(1);
+    return DCP_OK;
+}
+
+extern "C" int dcp_copy_segments(const void* src, void* dst, const int32_t* seg, int32_t n_seg, int64_t row_bytes,
+                                 int32_t n_planes, int64_t src_plane_bytes, int64_t dst_plane_bytes, int32_t reverse,
+                                 void* cuda_stream) {
+    const char* fn = "dcp_copy_segments";
+    if (n_seg < 0 || n_planes < 1 || row_bytes < 4 || row_bytes % 4 != 0 || src_plane_bytes < 0 || dst_plane_bytes < 0 ||
+        src_plane_bytes % 4 != 0 || dst_plane_bytes % 4 != 0)
+        return fail(DCP_ERR_INVALID_ARG, "%s: sizes must be non-negative and multiples of 4 bytes", fn);
+    if (n_planes > 65535) return fail(DCP_ERR_UNSUPPORTED, "%s: at most 65535 planes", fn);
+    if (n_seg == 0) return DCP_OK;
+    if (!src || !dst || !seg) return fail(DCP_ERR_INVALID_ARG, "%s: null pointer", fn);
+    if ((reinterpret_cast<uintptr_t>(src) & 3u) || (reinterpret_cast<uintptr_t>(dst) & 3u))
+        return fail(DCP_ERR_INVALID_ARG, "%s: tensors must be 4-byte aligned", fn);
+    DeviceInfo dev;
+    if (int rc = device_info(&dev)) return rc;
+    const cudaError_t e = launch_copy_segments(src, dst, seg, n_seg, row_bytes, n_planes, src_plane_bytes, dst_plane_bytes,
+                                               reverse != 0, dev.sm_count, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: %s", fn, cudaGetErrorString(e));
+    g_launches.fetch_add(1);
     return DCP_OK;
 }
 
@@ -407,8 +518,11 @@ extern "C" int dcp_profile_read(float* ms, int64_t* launches) {
         if (e == cudaSuccess) e = cudaEventElapsedTime(&one, t.start, t.stop);
         if (e != cudaSuccess) rc = fail(DCP_ERR_CUDA, "dcp_profile_read: %s", cudaGetErrorString(e));
         else { ms[t.kernel] += one; launches[t.kernel] += 1; }
-        cudaEventDestroy(t.start);
-        cudaEventDestroy(t.stop);
+    }
+    std::lock_guard<std::mutex> lock(g_prof_mu);
+    for (const TimedLaunch& t : pending) {
+        g_event_pool[t.device].push_back(t.start);
+        g_event_pool[t.device].push_back(t.stop);
     }
     return rc;
 }

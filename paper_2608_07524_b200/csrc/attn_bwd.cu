@@ -51,22 +51,6 @@
 #include "sched.cuh"
 #include "sm100_ptx.cuh"
 
-// Development aid (-DDCP_TIMING, not part of the product build): the MMA thread and compute warp 0
-// accumulate the cycles spent in each wait and phase; dcp_debug_read_timing copies the table out.
-#ifdef DCP_TIMING
-__device__ long long g_bwd_timing[148 * 2 * 16];
-#define TW(i, ...) do { long long _t = clock64(); __VA_ARGS__; tacc[i] += clock64() - _t; } while (0)
-#define TDECL long long tacc[16] = {0}; const long long _t_begin = clock64();
-#define TDUMP(role) do { tacc[15] = clock64() - _t_begin; for (int _i = 0; _i < 16; ++_i) g_bwd_timing[(blockIdx.x * 2 + (role)) * 16 + _i] = tacc[_i]; } while (0)
-extern "C" int dcp_debug_read_timing(long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, g_bwd_timing, sizeof(long long) * 148 * 2 * 16);
-}
-#else
-#define TW(i, ...) __VA_ARGS__
-#define TDECL
-#define TDUMP(role)
-#endif
-
 namespace dcp {
 
 // The drain warps pause after every kRedGroup vector atomics, and warp k of the four starts k pauses
@@ -264,6 +248,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sh.tmem_base;
+    // when this CTA started and (at the end) when it ran out of work: the spread over CTAs measures the balance
+    if (tid == 0 && blockIdx.x < kMaxCtas) {
+        p.sched.spans[1 * kMaxCtas + blockIdx.x].begin_ns = global_timer_ns();
+        if (blockIdx.x == 0) p.sched.hdr->n_ctas[1] = gridDim.x < kMaxCtas ? gridDim.x : kMaxCtas;
+    }
 
     // Q tiles that see key block `blk`: [first_q, n_q)
     auto q_range = [](const WorkItem& w, int& first_q, int& n_q) {
@@ -366,7 +355,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     if (leader) tc_mma_ss(d_tmem, a + km_step(ks, Cfg::kBoxBytes), b + km_step(ks, Cfg::kBoxBytes), idesc_abt, ks > 0);
             };
             uint32_t n_work = 0, g = 0;
-            TDECL
             while (true) {
                 const uint32_t slot = n_work & 1u;
                 const bool got = mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard);
@@ -378,7 +366,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 int first_q, n_q;
                 q_range(w, first_q, n_q);
                 const int N = n_q - first_q;
-                TW(0, mbar_wait(&sh.kv_full, n_work & 1u, guard));
+                mbar_wait(&sh.kv_full, n_work & 1u, guard);
                 // S^T and dP^T of the first tile
                 uint32_t stage = g % Cfg::kQStages;
                 mbar_wait(&sh.q_full[stage], (g / Cfg::kQStages) & 1u, guard);
@@ -398,10 +386,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     const uint32_t nstage = stage + 1 == Cfg::kQStages ? 0 : stage + 1;
                     const bool has_next = n + 1 < N;
                     // dV += P^T dO
-                    TW(1, mbar_wait(&sh.p_half, g & 1u, guard));
+                    mbar_wait(&sh.p_half, g & 1u, guard);
                     if (n == 0 && n_work >= 1) mbar_wait(&sh.dkv_free, (n_work - 1) & 1u, guard);
                     tc_fence_after();
-                    TW(6,
 #pragma unroll
                     for (int part = 0; part < 2; ++part) {
                         if (part == 1) {
@@ -415,41 +402,39 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                                       idesc_nd_kb, n > 0 || part > 0 || k4 > 0);
                         }
                     }
-                    if (leader) tc_commit(&sh.do_empty));
+                    if (leader) tc_commit(&sh.do_empty);
                     // S^T of the next tile
                     if (has_next) {
-                        TW(2, mbar_wait(&sh.q_full[nstage], ((g + 1) / Cfg::kQStages) & 1u, guard);
-                        mbar_wait(&sh.stat_full[(g + 1) & 1u], ((g + 1) >> 1) & 1u, guard));
+                        mbar_wait(&sh.q_full[nstage], ((g + 1) / Cfg::kQStages) & 1u, guard);
+                        mbar_wait(&sh.stat_full[(g + 1) & 1u], ((g + 1) >> 1) & 1u, guard);
                         tc_fence_after();
-                        TW(7, issue_abt(tmem + Cfg::kSt, k_km, q_km0 + nstage * kStageStep);
+                        issue_abt(tmem + Cfg::kSt, k_km, q_km0 + nstage * kStageStep);
                         if (leader) tc_mma_ss(tmem + Cfg::kSt, ones_s, stat0 + ((g + 1) & 1u) * kStatStep, idesc_abt, true);
-                        if (leader) tc_commit(&sh.s_full));
+                        if (leader) tc_commit(&sh.s_full);
                     }
                     // dQ tile = dS K  (A: dS^T read M-contiguous; B: K with head_dim contiguous)
-                    TW(3, mbar_wait(&sh.ds_full, g & 1u, guard));
+                    mbar_wait(&sh.ds_full, g & 1u, guard);
                     tc_fence_after();
-                    TW(8,
 #pragma unroll
                     for (int ks = 0; ks < kTile / 16; ++ks)
                         if (leader) tc_mma_ss(tmem + Cfg::kDp, ds_mn + mn_step(ks), k_mn + mn_step(ks), idesc_nd_mm, ks > 0);
-                    if (leader) tc_commit(&sh.dq_full));
+                    if (leader) tc_commit(&sh.dq_full);
                     // dK += dS^T Q
-                    TW(9,
 #pragma unroll
                     for (int ks = 0; ks < kTile / 16; ++ks)
                         if (leader) tc_mma_ss(tmem + Cfg::kDk, ds_km + km_step(ks, 16384), q_mn0 + stage * kStageStep + mn_step(ks),
                                   idesc_nd_kb, n > 0 || ks > 0);
                     if (leader) tc_commit(&sh.q_empty[stage]);
-                    if (leader) tc_commit(&sh.ds_free));
+                    if (leader) tc_commit(&sh.ds_free);
                     // dP^T of the next tile (its columns hold dQ until the drain warps have read it)
                     if (has_next) {
-                        TW(4, mbar_wait(&sh.do_full, (g + 1) & 1u, guard));
-                        TW(5, mbar_wait(&sh.dq_free, g & 1u, guard));
+                        mbar_wait(&sh.do_full, (g + 1) & 1u, guard);
+                        mbar_wait(&sh.dq_free, g & 1u, guard);
                         tc_fence_after();
-                        TW(10, issue_abt(tmem + Cfg::kDp, v_km, do_km);
+                        issue_abt(tmem + Cfg::kDp, v_km, do_km);
                         if (leader) tc_mma_ss(tmem + Cfg::kDp, ones_d, stat0 + ((g + 1) & 1u) * kStatStep, idesc_abt, true);
                         if (leader) tc_commit(&sh.dp_full);
-                        if (leader) tc_commit(&sh.stat_empty[(g + 1) & 1u]));
+                        if (leader) tc_commit(&sh.stat_empty[(g + 1) & 1u]);
                     }
                     stage = nstage;
                 }
@@ -457,7 +442,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 if (leader) tc_commit(&sh.kv_empty);
                 ++n_work;
             }
-            if (lane == 0) TDUMP(0);
         }
     }
     } else if (warp < 8) {
@@ -471,7 +455,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const uint32_t dp_tmem = tmem + lane_base + Cfg::kDp + half * 64;
         uint8_t* ds_row = smem + Cfg::kOffDs + half * 16384;
         uint32_t n_work = 0, g = 0;
-        TDECL
         while (true) {
             const uint32_t slot = n_work & 1u;
             const bool got = mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard);
@@ -494,20 +477,14 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             for (int i = first_q; i < n_q; ++i, ++g) {
                 const bool diag = CAUSAL && i == w.blk;
                 float pf[64];
-                TW(0, mbar_wait(&sh.s_full, g & 1u, guard));
+                mbar_wait(&sh.s_full, g & 1u, guard);
                 tc_fence_after();
-#ifdef DCP_TIMING
-                long long _tp = clock64();
-#endif
                 {
                     // all 64 scores of this thread's key row are requested before the single wait
                     uint32_t sr[64];
                     tmem_ld_x32(st_tmem, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
                     tmem_ld_x32(st_tmem + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
                     tmem_wait_ld();
-#ifdef DCP_TIMING
-                    tacc[7] += clock64() - _tp;
-#endif
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
                         // 32 query columns at a time: the dV product starts on the first chunk while the
@@ -536,25 +513,16 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.p_full);
-#ifdef DCP_TIMING
-                tacc[3] += clock64() - _tp;
-#endif
 
                 // dS^T = P^T o (dP^T - D)
-                TW(1, mbar_wait(&sh.dp_full, g & 1u, guard));
-                if (g >= 1) TW(2, mbar_wait(&sh.ds_free, (g - 1) & 1u, guard));
+                mbar_wait(&sh.dp_full, g & 1u, guard);
+                if (g >= 1) mbar_wait(&sh.ds_free, (g - 1) & 1u, guard);
                 tc_fence_after();
-#ifdef DCP_TIMING
-                _tp = clock64();
-#endif
                 {
                     uint32_t dr[64];
                     tmem_ld_x32(dp_tmem, *reinterpret_cast<uint32_t(*)[32]>(&dr[0]));
                     tmem_ld_x32(dp_tmem + 32, *reinterpret_cast<uint32_t(*)[32]>(&dr[32]));
                     tmem_wait_ld();
-#ifdef DCP_TIMING
-                    tacc[5] += clock64() - _tp;
-#endif
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         uint32_t pk[4];
@@ -565,16 +533,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         *reinterpret_cast<uint4*>(ds_row + sw128_offset(key_in_tile, c)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
                 }
-#ifdef DCP_TIMING
-                tacc[6] += clock64() - _tp;
-#endif
                 fence_async_smem();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.ds_full);
-#ifdef DCP_TIMING
-                tacc[4] += clock64() - _tp;
-#endif
             }
 
             // item epilogue: dV and dK rows of this key block (each group writes half the columns)
@@ -610,7 +572,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             if (lane == 0) mbar_arrive(&sh.dkv_free);
             ++n_work;
         }
-        if (warp == 0 && lane == 0) TDUMP(1);
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 136;");
         // ------------------------------------------------- dQ drain: tensor memory -> fp32 atomics
@@ -674,6 +635,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 
     tc_fence_before();
     __syncthreads();
+    if (tid == 0 && blockIdx.x < kMaxCtas) p.sched.spans[1 * kMaxCtas + blockIdx.x].end_ns = global_timer_ns();
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 

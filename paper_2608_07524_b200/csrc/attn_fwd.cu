@@ -25,21 +25,6 @@
 #include "sched.cuh"
 #include "sm100_ptx.cuh"
 
-// Development aid (-DDCP_TIMING, not part of the product build): cycles spent in waits and phases.
-#ifdef DCP_TIMING
-__device__ long long g_fwd_timing[148 * 3 * 8];
-#define FTW(i, ...) do { long long _t = clock64(); __VA_ARGS__; tacc[i] += clock64() - _t; } while (0)
-#define FTDECL long long tacc[8] = {0}; const long long _t_begin = clock64();
-#define FTDUMP(role) do { tacc[7] = clock64() - _t_begin; for (int _i = 0; _i < 8; ++_i) g_fwd_timing[(blockIdx.x * 3 + (role)) * 8 + _i] = tacc[_i]; } while (0)
-extern "C" int dcp_debug_read_timing_fwd(long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, g_fwd_timing, sizeof(long long) * 148 * 3 * 8);
-}
-#else
-#define FTW(i, ...) __VA_ARGS__
-#define FTDECL
-#define FTDUMP(role)
-#endif
-
 namespace dcp {
 
 // One pair of exponentials in this many is computed on the FMA pipe instead of the special-function
@@ -258,6 +243,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sh.tmem_base;
+    // when this CTA started and (at the end) when it ran out of work: the spread over CTAs measures the balance
+    if (tid == 0 && blockIdx.x < kMaxCtas) {
+        p.sched.spans[0 * kMaxCtas + blockIdx.x].begin_ns = global_timer_ns();
+        if (blockIdx.x == 0) p.sched.hdr->n_ctas[0] = gridDim.x < kMaxCtas ? gridDim.x : kMaxCtas;
+    }
 
     if (warp >= 8) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
@@ -311,7 +301,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         {
             const bool leader = elect_one();
             uint32_t n_work = 0, kv_base = 0, use[2] = {0, 0}, n_p[2] = {0, 0};
-            FTDECL
             const uint64_t q_desc[2] = {make_sdesc_sw128(smem_u32(sQ), 16, 1024),
                                         make_sdesc_sw128(smem_u32(sQ) + Cfg::kTileBytes, 16, 1024)};
             const uint64_t kv_km0 = make_sdesc_sw128(smem_u32(sKV), 16, 1024);                 // K: head_dim contiguous
@@ -320,7 +309,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             const uint32_t s_tmem[2] = {tmem + Cfg::kS0, tmem + Cfg::kS1};
             const uint32_t o_tmem[2] = {tmem + Cfg::kO0, tmem + Cfg::kO1};
             auto kv_wait = [&](uint32_t idx) {
-                FTW(0, mbar_wait(&sh.kv_full[idx % kKvStages], (idx / kKvStages) & 1u, guard));
+                mbar_wait(&sh.kv_full[idx % kKvStages], (idx / kKvStages) & 1u, guard);
             };
             auto commit = [&](uint64_t* bar) { if (leader) tc_commit(bar); };
             while (true) {
@@ -365,7 +354,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                             if (j == 0 && use[t] >= 1) mbar_wait(&sh.o_free[t], (use[t] - 1) & 1u, guard);
 #pragma unroll
                             for (int part = 0; part < 4; ++part) {
-                                FTW(1 + t, mbar_wait(&sh.p_part[t][part], n_p[t] & 1u, guard));
+                                mbar_wait(&sh.p_part[t][part], n_p[t] & 1u, guard);
                                 tc_fence_after();
                                 issue_pv<D>(o_tmem[t], s_tmem[t], kv_mn0 + st_v * kStageStep, j > 0, leader, part);
                             }
@@ -388,7 +377,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 }
                 kv_base += 2 * nkv;
             }
-            if (lane == 0) FTDUMP(0);
         }
     }
     } else {
@@ -400,7 +388,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const uint32_t s_tmem = tmem + lane_base + (t == 0 ? Cfg::kS0 : Cfg::kS1);
         const uint32_t o_tmem = tmem + lane_base + (t == 0 ? Cfg::kO0 : Cfg::kO1);
         uint32_t n_work = 0, n_s = 0, use = 0;
-        FTDECL
         while (true) {
             const uint32_t slot = n_work & 1u;
             const bool got = mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard);
@@ -425,11 +412,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 
             float m = -INFINITY, l = 0.f;
             for (int j = 0; j < nkv; ++j) {
-                FTW(0, mbar_wait(&sh.s_full[t], n_s & 1u, guard));
+                mbar_wait(&sh.s_full[t], n_s & 1u, guard);
                 ++n_s;
-#ifdef DCP_TIMING
-                const long long _tp = clock64();
-#endif
                 tc_fence_after();
                 uint32_t s[128];
 #pragma unroll
@@ -518,9 +502,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     unpack_f32x2(sum2[1], b0, b1);
                     l += (a0 + a1) + (b0 + b1);
                 }
-#ifdef DCP_TIMING
-                tacc[1] += clock64() - _tp;
-#endif
             }
 
             // epilogue: O = acc / l, lse = m*scale + ln l
@@ -553,11 +534,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.o_free[t]);
         }
-        if ((warp == 0 || warp == 4) && lane == 0) FTDUMP(1 + t);
     }
 
     tc_fence_before();
     __syncthreads();
+    if (tid == 0 && blockIdx.x < kMaxCtas) p.sched.spans[0 * kMaxCtas + blockIdx.x].end_ns = global_timer_ns();
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 

@@ -44,13 +44,23 @@ struct BwdParams {
 // With `bounds` non-null, short sequences are first merged into virtual sequences: sched.vcu and
 // `bounds` are written and the list is built over sched.vcu, which the later kernels must then be
 // given as their boundary array; with `bounds` null the list is built over cu_seqlens itself.
-int prep_launches(int32_t n_seqs, bool merge);   // kernels launch_prep enqueues (1 to 4)
+int prep_launches(int32_t n_seqs, bool merge, bool input_order);   // kernels launch_prep enqueues (1 to 4)
 // tile_capacity = number of 128-row tiles the per-tile storage of the workspace holds (UINT32_MAX if the
 // call uses none).  Inconsistent boundaries or more tiles than that leave an empty work list and
-// kStatusBadLengths in the status word.
+// kStatusBadLengths in the status word.  input_order = true lists the sequences as they come instead of
+// longest first (a measurement aid: it shows what the ordering is worth).
 cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen,
                         int32_t rows_per_block, int32_t n_heads, const SchedView& sched, uint16_t* bounds,
-                        uint32_t tile_capacity, cudaStream_t stream);
+                        uint32_t tile_capacity, bool input_order, cudaStream_t stream);
+
+// One CTA that waits, with the kernels' own bounded wait and the given poll limit, on a barrier nobody
+// arrives at, and leaves through the same abort path (status word raised, no trap).
+cudaError_t launch_wait_timeout_selftest(WorkspaceHeader* hdr, uint32_t spin_limit, cudaStream_t stream);
+
+// Copies row ranges between two tensors (see dcp_copy_segments).
+cudaError_t launch_copy_segments(const void* src, void* dst, const int32_t* seg, int32_t n_seg, int64_t row_bytes,
+                                 int32_t n_planes, int64_t src_plane_bytes, int64_t dst_plane_bytes, bool reverse,
+                                 int n_sms, cudaStream_t stream);
 
 cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                             int head_dim, bool causal, int n_ctas, cudaStream_t stream);

@@ -129,3 +129,56 @@ extern "C" int dcp_plan_profiled(const int32_t* lengths, const int64_t* fwd_time
     if (!fwd_time) return dcp::fail(DCP_ERR_INVALID_ARG, "dcp_plan_profiled: null pointer");
     return plan_impl("dcp_plan_profiled", lengths, fwd_time, n, hbm_budget_bytes, params, mb_id, n_mb, recompute, cost);
 }
+
+// Where each sequence of a planned batch lives: in the batch (packed in input order) and in its
+// micro-batch's own packed tensors.  The definition is in include/dcp.h.
+extern "C" int dcp_plan_segments(const int32_t* lengths, const int32_t* mb_id, int32_t n, int32_t n_mb, int32_t max_rows,
+                                 int32_t* mb_seq_offset, int32_t* seq_index, int32_t* mb_cu, int32_t* seg_offset,
+                                 int32_t* seg, int32_t seg_capacity, int32_t* n_seg) {
+    const char* who = "dcp_plan_segments";
+    if (!lengths || !mb_id || !mb_seq_offset || !seq_index || !mb_cu || !seg_offset || !seg || !n_seg)
+        return dcp::fail(DCP_ERR_INVALID_ARG, "%s: null pointer", who);
+    if (n < 1 || n_mb < 1 || n_mb > n || max_rows < 1 || seg_capacity < 0)
+        return dcp::fail(DCP_ERR_INVALID_ARG, "%s: need 1 <= n_mb <= n, max_rows >= 1, seg_capacity >= 0", who);
+    std::vector<int64_t> src_row(n + 1, 0);
+    std::vector<int32_t> count(n_mb, 0);
+    for (int32_t i = 0; i < n; ++i) {
+        if (lengths[i] < 0) return dcp::fail(DCP_ERR_INVALID_ARG, "%s: lengths[%d] is negative", who, i);
+        if (mb_id[i] < 0 || mb_id[i] >= n_mb) return dcp::fail(DCP_ERR_INVALID_ARG, "%s: mb_id[%d] = %d is not in [0, n_mb)", who, i, mb_id[i]);
+        src_row[i + 1] = src_row[i] + lengths[i];
+        ++count[mb_id[i]];
+    }
+    if (src_row[n] > INT32_MAX) return dcp::fail(DCP_ERR_OVERFLOW, "%s: more than 2^31 - 1 tokens", who);
+    mb_seq_offset[0] = 0;
+    for (int32_t k = 0; k < n_mb; ++k) mb_seq_offset[k + 1] = mb_seq_offset[k] + count[k];
+    std::vector<int32_t> fill(mb_seq_offset, mb_seq_offset + n_mb);
+    for (int32_t i = 0; i < n; ++i) seq_index[fill[mb_id[i]]++] = i;      // input order inside a micro-batch
+    int64_t total_seg = 0;
+    for (int32_t k = 0; k < n_mb; ++k) {
+        seg_offset[k] = (int32_t)total_seg;
+        int64_t dst = 0;
+        // micro-batch k's boundary array occupies mb_cu[mb_seq_offset[k] + k ...], count[k] + 1 entries
+        int32_t* cu = mb_cu + mb_seq_offset[k] + k;
+        cu[0] = 0;
+        for (int32_t e = mb_seq_offset[k]; e < mb_seq_offset[k + 1]; ++e) {
+            const int32_t i = seq_index[e];
+            for (int32_t done = 0; done < lengths[i]; done += max_rows) {
+                const int32_t rows = std::min(max_rows, lengths[i] - done);
+                if (total_seg < seg_capacity) {
+                    seg[3 * total_seg] = (int32_t)(src_row[i] + done);
+                    seg[3 * total_seg + 1] = (int32_t)(dst + done);
+                    seg[3 * total_seg + 2] = rows;
+                }
+                ++total_seg;
+            }
+            dst += lengths[i];
+            cu[e - mb_seq_offset[k] + 1] = (int32_t)dst;
+        }
+    }
+    seg_offset[n_mb] = (int32_t)std::min<int64_t>(total_seg, INT32_MAX);
+    *n_seg = seg_offset[n_mb];
+    if (total_seg > seg_capacity)
+        return dcp::fail(DCP_ERR_WORKSPACE, "%s: %lld segments needed, seg holds %d (ask again with that capacity)", who,
+                         (long long)total_seg, seg_capacity);
+    return DCP_OK;
+}

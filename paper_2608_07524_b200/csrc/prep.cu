@@ -10,6 +10,7 @@ namespace dcp {
 constexpr int kPrepThreads = 1024;
 
 __device__ inline uint32_t block_exclusive_scan(uint32_t v, uint32_t* scratch, uint32_t* total);
+__device__ inline int block_exclusive_max_scan(int v, int* scratch);
 
 // Merging of short sequences into virtual sequences of at most 128 tokens.  One CTA.
 //
@@ -28,7 +29,9 @@ __device__ inline uint32_t block_exclusive_scan(uint32_t v, uint32_t* scratch, u
 // bound on the number of tiles that sizes the workspace: it is derived for rule 0).
 // Outputs: vcu[0..n_v] = boundaries of the virtual sequences, vcu[n_v+1..n_seqs] = total_tokens
 // (empty padding, so that vcu is a valid boundary array of n_seqs sequences); hdr->n_vseq = n_v;
-// hdr->merge_rule = the rule used.
+// hdr->merge_rule = the rule used; vstart[i] = first token of the virtual sequence that input
+// sequence i belongs to (read by bounds_kernel, so that no thread there has to walk back over a run,
+// which under rule 0 may hold any number of empty sequences).
 __device__ __forceinline__ bool merge_is_head(const int32_t* __restrict__ cu, int i, int32_t max_short, uint32_t rule) {
     if (i == 0 || cu[i + 1] - cu[i] > max_short || cu[i] - cu[i - 1] > max_short) return true;
     if (rule == 0) {
@@ -40,19 +43,18 @@ __device__ __forceinline__ bool merge_is_head(const int32_t* __restrict__ cu, in
 
 __global__ void __launch_bounds__(kPrepThreads) merge_kernel(const int32_t* __restrict__ cu, int32_t n_seqs,
                                                              int32_t total_tokens, int32_t max_short,
-                                                             WorkspaceHeader* hdr, int32_t* vcu) {
+                                                             WorkspaceHeader* hdr, int32_t* vcu, int32_t* vstart) {
     __shared__ uint32_t scratch[33];
     const int tid = threadIdx.x;
     const int per = (n_seqs + kPrepThreads - 1) / kPrepThreads;
     const int begin = min(tid * per, n_seqs), end = min(begin + per, n_seqs);
     // The boundaries come from the caller and index everything that follows: they must start at 0, never
     // decrease and end at total_tokens.  If not, the status word says so and every sequence is made empty,
-    // which turns the rest of the call into no-ops.  This kernel is the first of a call, so it also resets
-    // the status word.
+    // which turns the rest of the call into no-ops.  This kernel is the first of a call.
     int bad = (tid == 0 && (cu[0] != 0 || cu[n_seqs] != total_tokens)) ? 1 : 0;
     for (int i = begin; i < end; ++i) bad |= cu[i + 1] < cu[i] ? 1 : 0;
     bad = __syncthreads_or(bad);
-    if (tid == 0) hdr->status = bad ? (uint32_t)kStatusBadLengths : (uint32_t)kStatusOk;
+    if (tid == 0) header_begin_call(hdr, bad != 0);
     if (bad) {
         for (int i = tid; i <= n_seqs; i += kPrepThreads) vcu[i] = 0;
         if (tid == 0) hdr->n_vseq = 0;
@@ -75,26 +77,33 @@ __global__ void __launch_bounds__(kPrepThreads) merge_kernel(const int32_t* __re
         hdr->n_vseq = n_v;
         hdr->merge_rule = rule;
     }
+    int last_head = -1;
     for (int i = begin; i < end; ++i)
-        if (merge_is_head(cu, i, max_short, rule)) vcu[run++] = cu[i];
+        if (merge_is_head(cu, i, max_short, rule)) {
+            vcu[run++] = cu[i];
+            last_head = i;
+        }
     for (uint32_t i = n_v + tid; i <= (uint32_t)n_seqs; i += kPrepThreads) vcu[i] = total_tokens;
+    // head of the run each sequence belongs to: the last head at or before it (sequence 0 is always one)
+    int cur = block_exclusive_max_scan(last_head, reinterpret_cast<int*>(scratch));
+    for (int i = begin; i < end; ++i) {
+        if (merge_is_head(cu, i, max_short, rule)) cur = i;
+        vstart[i] = cu[cur];
+    }
 }
 
 // One thread per input sequence of at most 128 tokens, over as many CTAs as needed: bounds[t] for
 // each of its tokens t = (first, end) position of the sequence relative to the start of its virtual
-// sequence, one byte each.  The start is found by walking back to the head of the run (the head rule
-// is local, so this does not wait for merge_kernel's scan).
-__global__ void __launch_bounds__(256) bounds_kernel(const int32_t* __restrict__ cu, int32_t n_seqs, int32_t max_short,
-                                                     const WorkspaceHeader* __restrict__ hdr, uint16_t* __restrict__ bounds) {
+// sequence, one byte each.  merge_kernel has left that start in vstart[].
+__global__ void __launch_bounds__(256) bounds_kernel(const int32_t* __restrict__ cu, int32_t n_seqs,
+                                                     const WorkspaceHeader* __restrict__ hdr,
+                                                     const int32_t* __restrict__ vstart, uint16_t* __restrict__ bounds) {
     const int i = blockIdx.x * 256 + threadIdx.x;
-    if (i >= n_seqs || hdr->status != kStatusOk) return;      // merge_kernel found the boundaries inconsistent
+    if (i >= n_seqs || hdr->call_bad) return;      // merge_kernel found the boundaries inconsistent
     const int32_t a = cu[i], b = cu[i + 1];
     if (b == a || b - a > kTile) return;
-    const uint32_t rule = hdr->merge_rule;
-    int j = i;
-    while (!merge_is_head(cu, j, max_short, rule)) --j;     // at most 127 non-empty members before i
-    const int32_t vstart = cu[j];
-    const uint16_t packed = (uint16_t)((a - vstart) | ((b - vstart) << 8));
+    const int32_t v0 = vstart[i];
+    const uint16_t packed = (uint16_t)((a - v0) | ((b - v0) << 8));
     for (int32_t t = a; t < b; ++t) bounds[t] = packed;
 }
 
@@ -157,7 +166,37 @@ __device__ inline uint32_t block_exclusive_scan(uint32_t v, uint32_t* scratch, u
     return scratch[warp] + incl - v;
 }
 
-// One CTA.  order[] as above (computed here unless `ranked`); prefix[i] = number of work items of the
+// Exclusive running maximum of one value per thread (in thread order) over a CTA of kPrepThreads
+// threads; -1 where nothing precedes.  scratch holds 33 words.
+__device__ inline int block_exclusive_max_scan(int v, int* scratch) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, s);
+        if (lane >= s) incl = max(incl, t);
+    }
+    __syncthreads();                       // scratch may still be read from an earlier scan
+    if (lane == 31) scratch[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int wi = scratch[lane];
+#pragma unroll
+        for (int s = 1; s < 32; s <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, wi, s);
+            if (lane >= s) wi = max(wi, t);
+        }
+        scratch[lane] = wi;                // inclusive over warps
+    }
+    __syncthreads();
+    int excl = __shfl_up_sync(0xffffffffu, incl, 1);
+    if (lane == 0) excl = -1;
+    if (warp > 0) excl = max(excl, scratch[warp - 1]);
+    return excl;
+}
+
+// One CTA.  order[] as above (computed here if `ranked` is 0, by rank_kernel if 1; 2 keeps the input
+// order, a measurement aid); prefix[i] = number of work items of the
 // first i sequences in that order, where a sequence of length L contributes
 // ceil(L / rows_per_block) * n_heads items; tile_prefix[b] = 128-row tiles before sequence b.
 // Sequences from *n_live_ptr on (if given) are empty padding and sorted last: only the live ones
@@ -177,7 +216,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __res
         int bad = (tid == 0 && (cu[0] != 0 || cu[n_seqs] != total_tokens)) ? 1 : 0;
         for (int i = tid; i < n_seqs; i += kPrepThreads) bad |= cu[i + 1] < cu[i] ? 1 : 0;
         bad = __syncthreads_or(bad);
-        if (tid == 0) hdr->status = bad ? (uint32_t)kStatusBadLengths : (uint32_t)kStatusOk;
+        if (tid == 0) header_begin_call(hdr, bad != 0);
         if (bad) {
             for (int i = tid; i <= n_seqs; i += kPrepThreads) { prefix[i] = 0; tile_prefix[i] = 0; }
             for (int i = tid; i < n_seqs; i += kPrepThreads) order[i] = i;
@@ -185,7 +224,9 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __res
             return;
         }
     }
-    if (!ranked) {                                    // n_seqs <= kPrepThreads: one sequence per thread
+    if (ranked == 2) {
+        for (int i = tid; i < n_seqs; i += kPrepThreads) order[i] = i;
+    } else if (!ranked) {                             // n_seqs <= kPrepThreads: one sequence per thread
         len_sh[tid] = tid < n_seqs ? cu[tid + 1] - cu[tid] : -1;
         __syncthreads();
         if (tid < n_seqs) {
@@ -228,7 +269,10 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __res
         // more tiles than the workspace was sized for: max_seqlen was understated (the bound on merged runs
         // relies on it).  Nothing may index the per-tile storage: no items, no tiles.
         for (int i = tid; i <= n_seqs; i += kPrepThreads) tile_prefix[i] = 0;
-        if (tid == 0) { hdr->n_items = 0; hdr->status = kStatusBadLengths; }
+        if (tid == 0) {
+            hdr->n_items = 0;
+            atomicMax(&hdr->status, (uint32_t)kStatusBadLengths);
+        }
         return;
     }
     for (int i = begin; i < end; ++i) {
@@ -238,26 +282,29 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __res
     for (int i = n_live + tid; i <= n_seqs; i += kPrepThreads) tile_prefix[i] = total;
 }
 
-int prep_launches(int32_t n_seqs, bool merge) { return (n_seqs > kPrepThreads ? 2 : 1) + (merge ? 2 : 0); }
+int prep_launches(int32_t n_seqs, bool merge, bool input_order) {
+    return (n_seqs > kPrepThreads && !input_order ? 2 : 1) + (merge ? (n_seqs > 0 ? 2 : 1) : 0);
+}
 
 cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen,
                         int32_t rows_per_block, int32_t n_heads, const SchedView& sched, uint16_t* bounds,
-                        uint32_t tile_capacity, cudaStream_t stream) {
+                        uint32_t tile_capacity, bool input_order, cudaStream_t stream) {
     const int32_t* cu = cu_seqlens;
     const uint32_t* n_live = nullptr;
     if (bounds) {                                       // merge short sequences; everything below sees vcu
         const int32_t max_short = max_seqlen < kMergeMaxLen ? (max_seqlen > 0 ? max_seqlen : 1) : kMergeMaxLen;
+        // order[] is not needed until the ranking below: until then it carries each sequence's run start
         merge_kernel<<<1, kPrepThreads, 0, stream>>>(cu_seqlens, n_seqs, total_tokens, max_short, sched.hdr,
-                                                     const_cast<int32_t*>(sched.vcu));
+                                                     const_cast<int32_t*>(sched.vcu), const_cast<int32_t*>(sched.order));
         if (cudaError_t e = cudaGetLastError()) return e;
         if (n_seqs > 0)
-            bounds_kernel<<<(n_seqs + 255) / 256, 256, 0, stream>>>(cu_seqlens, n_seqs, max_short, sched.hdr, bounds);
+            bounds_kernel<<<(n_seqs + 255) / 256, 256, 0, stream>>>(cu_seqlens, n_seqs, sched.hdr, sched.order, bounds);
         if (cudaError_t e = cudaGetLastError()) return e;
         cu = sched.vcu;
         n_live = &sched.hdr->n_vseq;
     }
-    const int ranked = n_seqs > kPrepThreads;
-    if (ranked) {
+    const int ranked = input_order ? 2 : (n_seqs > kPrepThreads ? 1 : 0);
+    if (ranked == 1) {
         rank_kernel<<<(n_seqs + 255) / 256, 256, 0, stream>>>(cu, n_seqs, n_live, const_cast<int32_t*>(sched.order));
         if (cudaError_t e = cudaGetLastError()) return e;
     }

@@ -29,17 +29,49 @@ enum : uint32_t {
 };
 
 // First bytes of every workspace.  `status` must stay at offset 0 (dcp_query_status reads it).
+// The status word is sticky: kernels only ever raise it (atomicMax), so a failure of any call on this
+// workspace stays visible until dcp_query_status has reported and cleared it.  A workspace needs no
+// initialisation by the caller: the first kernel of a call that does not find `magic` treats the
+// header as fresh memory and clears the status word itself.
+constexpr uint32_t kHeaderMagic0 = 0x64637031u, kHeaderMagic1 = 0x9e3779b9u;
+constexpr int kMaxCtas = 256;         // persistent CTAs whose time span the header area can record
 struct WorkspaceHeader {
-    uint32_t status;        // 0 = ok, else a kStatus* code left by a kernel
+    uint32_t status;        // 0 = ok, else the highest kStatus* code a kernel has left since the last query
     uint32_t work_counter;  // next unclaimed work item
     uint32_t n_items;       // items in the list
     uint32_t n_vseq;        // virtual sequences that are not padding
     uint32_t merge_rule;    // which of the two merging rules built them (see merge_kernel)
-    uint32_t pad[59];
+    uint32_t call_bad;      // this call's boundaries were inconsistent (reset by every call)
+    uint32_t magic[2];      // kHeaderMagic0/1 once the header has been initialised
+    uint32_t n_ctas[2];     // CTAs of the last forward / backward main launch that recorded a span
+    uint32_t pad[54];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
 
-// After the header: int32 order[n_seqs] (sequence ids, longest first, ties by id),
+#ifdef __CUDACC__
+// Run by one thread of the first kernel of every call: a header that does not carry the magic words is
+// fresh memory, whose status word means nothing yet.  Afterwards the status word is only ever raised.
+__device__ __forceinline__ void header_begin_call(WorkspaceHeader* hdr, bool bad) {
+    if (hdr->magic[0] != kHeaderMagic0 || hdr->magic[1] != kHeaderMagic1) {
+        hdr->status = kStatusOk;
+        hdr->magic[0] = kHeaderMagic0;
+        hdr->magic[1] = kHeaderMagic1;
+    }
+    hdr->call_bad = bad ? 1u : 0u;
+    if (bad) atomicMax(&hdr->status, (uint32_t)kStatusBadLengths);
+}
+#endif
+
+// When a persistent CTA of the forward (slot 0) or backward main kernel (slot 1) started and when it
+// ran out of work, in nanoseconds of the GPU's global timer.  Their spread over the CTAs is the
+// single-GPU form of the paper's imbalance ratio (Section 2.3, Section 4.2): with a good work order
+// every CTA ends within one item of the others.
+struct CtaSpan {
+    unsigned long long begin_ns, end_ns;
+};
+constexpr size_t kSpanBytes = 2 * kMaxCtas * sizeof(CtaSpan);      // 8 KB right after the header
+
+// After the header and the span table: int32 order[n_seqs] (sequence ids, longest first, ties by id),
 // uint32 prefix[n_seqs + 1] (items before the i-th sequence of `order`),
 // uint32 tile_prefix[n_seqs + 1] (128-row tiles before sequence b, in input order) and
 // int32 vcu[n_seqs + 1] (virtual sequence boundaries; unused when sequences are not merged).
@@ -47,6 +79,7 @@ static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
 // (vcu, or the caller's cu_seqlens when merging is off).
 struct SchedView {
     WorkspaceHeader* hdr;
+    CtaSpan* spans;         // [2][kMaxCtas]
     const int32_t* order;
     const uint32_t* prefix;
     const uint32_t* tile_prefix;
@@ -55,8 +88,8 @@ struct SchedView {
 };
 
 __host__ __device__ constexpr size_t sched_bytes(int32_t n_seqs) {
-    return (sizeof(WorkspaceHeader) + sizeof(int32_t) * (size_t)n_seqs + 2 * sizeof(uint32_t) * ((size_t)n_seqs + 1) +
-            sizeof(int32_t) * ((size_t)n_seqs + 1) + 255) & ~(size_t)255;
+    return (sizeof(WorkspaceHeader) + kSpanBytes + sizeof(int32_t) * (size_t)n_seqs +
+            2 * sizeof(uint32_t) * ((size_t)n_seqs + 1) + sizeof(int32_t) * ((size_t)n_seqs + 1) + 255) & ~(size_t)255;
 }
 
 // Per-token table of the merged path: low byte = first position, high byte = one past the last

@@ -60,15 +60,27 @@ struct WaitGuard {
 
 constexpr uint32_t kSpinLimit = 1u << 24;   // try_wait polls before a wait is abandoned
 
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const WaitGuard& g) {
+// Waits for the phase with the given parity, at most `limit` polls.  On giving up it raises the CTA's
+// abort flag and the workspace's status word and returns false; it never traps and never spins on.
+__device__ __forceinline__ bool mbar_wait_limited(uint64_t* bar, uint32_t parity, const WaitGuard& g, uint32_t limit) {
     if (mbar_try_wait(bar, parity)) return true;
-    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+    for (uint32_t spin = 0; spin < limit; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((spin & 1023u) == 1023u && *g.abort_flag) return false;
     }
     *g.abort_flag = 1u;
     if (g.status) atomicMax(g.status, (uint32_t)kStatusWaitTimeout);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const WaitGuard& g) {
+    return mbar_wait_limited(bar, parity, g, kSpinLimit);
+}
+
+// Nanoseconds of the GPU-wide timer (the same clock on every SM, unlike clock64).
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
 }
 
 // Generic-proxy writes to shared memory become visible to the async proxy (TMA, tcgen05.mma).

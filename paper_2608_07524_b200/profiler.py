@@ -7,8 +7,10 @@ whole model is extrapolated as Lambda * (2 t_f + t_b) + T_C under full recomputa
 length buckets (sequence-parallel size is 1 on one GPU).  The table feeds dcp_plan_profiled, which
 replaces the planner's L^2 stand-in for t_f by these measurements.
 
-Only host logic lives here: which buckets to run, what to keep, and integer interpolation between
-buckets.  The timed work is the library's kernels, timed by the library's own CUDA events.
+Only host logic lives here: which buckets to run and what to keep.  The timed work is the library's
+kernels, timed by the library's own CUDA events; interpolation between buckets (dcp_profile_interp),
+the modelled time of a micro-batch (dcp_model_time, Eq. 4-5) and the candidate rows of Algorithm 1
+(dcp_intra_candidate_from_profile) are computed by the library.
 """
 from __future__ import annotations
 
@@ -33,32 +35,25 @@ class ProfileTable:
         if any(t < 0 for t in self.t_f_ns + self.t_b_ns):
             raise ValueError("negative time in profile")
 
-    def _interp(self, col: Sequence[int], L: int) -> int:
-        """Integer interpolation, floor division throughout:
-        below the first bucket linear in L (short sequences are bound by memory traffic, which is
-        linear in tokens); between buckets linear; above the last bucket quadratic in L."""
-        if L < 1:
-            raise ValueError("length must be >= 1")
-        xs = self.lengths
-        if L <= xs[0]:
-            return col[0] * L // xs[0]
-        if L >= xs[-1]:
-            return col[-1] * L * L // (xs[-1] * xs[-1])
-        hi = next(i for i, x in enumerate(xs) if x >= L)
-        lo = hi - 1
-        return col[lo] + (col[hi] - col[lo]) * (L - xs[lo]) // (xs[hi] - xs[lo])
+    def fwd_times(self, lengths: Sequence[int]) -> List[int]:
+        from . import binding
+        return binding.dcp_profile_interp(self.lengths, self.t_f_ns, lengths)
+
+    def bwd_times(self, lengths: Sequence[int]) -> List[int]:
+        from . import binding
+        return binding.dcp_profile_interp(self.lengths, self.t_b_ns, lengths)
 
     def fwd_time(self, L: int) -> int:
-        return self._interp(self.t_f_ns, L)
+        return self.fwd_times([L])[0]
 
     def bwd_time(self, L: int) -> int:
-        return self._interp(self.t_b_ns, L)
+        return self.bwd_times([L])[0]
 
     def model_time(self, lengths: Sequence[int], n_layers: int, recompute: int, fixed_cost_ns: int = 0) -> int:
         """Eq. 4-5: T = Lambda (t_f + t_b) + r t_f + T_C for one micro-batch."""
-        tf = sum(self.fwd_time(L) for L in lengths)
-        tb = sum(self.bwd_time(L) for L in lengths)
-        return n_layers * (tf + tb) + recompute * tf + fixed_cost_ns
+        from . import binding
+        return binding.dcp_model_time(self.fwd_times(lengths), self.bwd_times(lengths), n_layers, recompute,
+                                      fixed_cost_ns)
 
 
 def _gpu_layer(n_heads: int, head_dim: int, causal: bool, device) -> Callable[[List[int]], Tuple[float, float]]:
@@ -109,3 +104,31 @@ def dual_layer_profile(bucket_lengths: Sequence[int], n_heads: int, head_dim: in
         t_b.append(int(round(b_ms * 1e6)) // copies)
         m.append(4 * L * n_heads * head_dim * elt_bytes)
     return ProfileTable(buckets, t_f, t_b, m)
+
+
+def intra_candidates(seq_len: int, batch_sizes: Sequence[int], n_heads: int, head_dim: int, causal: bool, n_layers: int,
+                     device="cuda", elt_bytes: int = 2, const_bytes: int = 0, fixed_cost_ns: int = 0,
+                     run_layer: Optional[Callable[[List[int]], Tuple[float, float]]] = None):
+    """The candidate table Algorithm 1 takes, for sequences of one length on one GPU: one row (b, 1) per
+    batch size b, measured the dual-layer way (the batch of b sequences runs twice, the second run is
+    kept).  Row = (b, p = 1, t_f, m, T_(b,1), M_(b,1)) with t_f the measured forward time of one layer for
+    the whole batch in ns, m = 4 b L H d e the bytes a layer keeps when it is not recomputed,
+    T = Lambda (2 t_f + t_b) + T_C the modelled time with every layer recomputed (Section 3.5) and
+    M = Lambda b L H d e + M_C (Eq. 6 at r = Lambda)."""
+    from . import binding
+    run = run_layer if run_layer is not None else _gpu_layer(n_heads, head_dim, causal, device)
+    rows = []
+    for b in batch_sizes:
+        run([seq_len] * b)                                  # first layer: warm-up, discarded
+        f_ms, b_ms = run([seq_len] * b)                     # second layer: recorded
+        unit = b * seq_len * n_heads * head_dim * elt_bytes
+        rows.append(binding.dcp_intra_candidate_from_profile(b, 1, int(round(f_ms * 1e6)), int(round(b_ms * 1e6)), 4 * unit,
+                                                             unit, n_layers, const_bytes, fixed_cost_ns))
+    return rows
+
+
+def select_group_setting(candidates, mem_capacity: int, n_layers: int) -> Tuple[int, int, int]:
+    """(batch size, recompute count, modelled time) Algorithm 1 picks from a candidate table."""
+    from . import binding
+    idx, r, t = binding.dcp_intra_select(candidates, mem_capacity, n_layers)
+    return candidates[idx][0], r, t

@@ -29,6 +29,33 @@ def assert_close(name, got, ref):
     assert max_abs <= MAX_ABS and rel <= REL_FRO, f"{name}: max-abs {max_abs:.3e}, rel-Frobenius {rel:.3e}"
 
 
+GUARD_ROWS, GUARD_BYTES, GUARD_FILL = 128, 1 << 16, 0x5A
+
+
+class Guarded:
+    """Device buffers with a poisoned margin after their end: whatever a kernel stores past the last row
+    of an output, past the end of lse or past the end of the workspace lands in the margin and is seen."""
+
+    def __init__(self, T, H, d, n_seqs, dev):
+        self.T, self.H, self.d = T, H, d
+        row = H * d
+        self.bf16 = [torch.full(((T + GUARD_ROWS) * row,), GUARD_FILL * 257, dtype=torch.int16, device=dev) for _ in range(4)]
+        self.o, self.dq, self.dk, self.dv = (b[: T * row].view(torch.bfloat16).view(T, H, d) for b in self.bf16)
+        self.lse_raw = torch.full((H * T + GUARD_BYTES // 4,), GUARD_FILL * 0x01010101, dtype=torch.int32, device=dev)
+        self.lse = self.lse_raw[: H * T].view(torch.float32).view(H, T)
+        _, bwd = B.dcp_varlen_attn_workspace(T, n_seqs, H, d)
+        self.ws_bytes = bwd
+        self.ws_raw = torch.full((bwd + GUARD_BYTES,), GUARD_FILL, dtype=torch.uint8, device=dev)
+        self.ws = self.ws_raw[:bwd]
+
+    def assert_margins_untouched(self, what):
+        row = self.H * self.d
+        for name, b in zip(("o", "dq", "dk", "dv"), self.bf16):
+            assert bool((b[self.T * row:] == GUARD_FILL * 257).all()), f"{what}: store past the end of {name}"
+        assert bool((self.lse_raw[self.H * self.T:] == GUARD_FILL * 0x01010101).all()), f"{what}: store past the end of lse"
+        assert bool((self.ws_raw[self.ws_bytes:] == GUARD_FILL).all()), f"{what}: store past the end of the workspace"
+
+
 def run_gpu(q, k, v, g, cu, causal, scale=0.0, o_override=None, lse_override=None):
     dev = "cuda"
     cud = torch.tensor(np.asarray(cu), dtype=torch.int32, device=dev)
@@ -36,13 +63,16 @@ def run_gpu(q, k, v, g, cu, causal, scale=0.0, o_override=None, lse_override=Non
     max_len = int(lens.max()) if lens.size else 0
     qd, kd, vd, gd = (x.to(dev) for x in (q, k, v, g))
     T, H, d = q.shape
-    ws = B.alloc_workspace(T, len(lens), H, d, True, dev)
-    o, lse = B.dcp_varlen_attn_fwd(qd, kd, vd, cud, max_len, causal, scale, workspace=ws)
-    B.dcp_query_status(ws)
+    buf = Guarded(T, H, d, len(lens), dev)
+    o, lse = B.dcp_varlen_attn_fwd(qd, kd, vd, cud, max_len, causal, scale, out=buf.o, lse=buf.lse, workspace=buf.ws)
+    B.dcp_query_status(buf.ws)
+    buf.assert_margins_untouched("forward")
     o_in = o if o_override is None else o_override.to(dev)
     lse_in = lse if lse_override is None else lse_override.to(dev)
-    dq, dk, dv = B.dcp_varlen_attn_bwd(qd, kd, vd, o_in, gd, lse_in, cud, max_len, causal, scale, workspace=ws)
-    B.dcp_query_status(ws)
+    dq, dk, dv = B.dcp_varlen_attn_bwd(qd, kd, vd, o_in, gd, lse_in, cud, max_len, causal, scale, dq=buf.dq, dk=buf.dk,
+                                       dv=buf.dv, workspace=buf.ws)
+    B.dcp_query_status(buf.ws)
+    buf.assert_margins_untouched("backward")
     return o, lse, dq, dk, dv
 
 
@@ -338,3 +368,74 @@ def test_merged_by_aligned_windows(causal):
     lengths = [64] * 9 + [60, 4, 64, 32, 32, 33, 31, 64, 200, 64, 64, 50, 14, 64, 1, 63]
     check_full(lengths, 2, 128, causal, seed=95)
     check_full([64] * 40, 1, 64, causal, seed=96)
+
+
+def test_status_word_is_sticky_and_maps_to_error_codes():
+    """The device status word keeps the most severe failure of any call until it is queried; the query
+    reports it and clears it.  Codes: 1 or 2 (a kernel gave up a bounded wait / found its shared memory
+    misaligned) -> DCP_ERR_TIMEOUT, 3 (inconsistent boundaries) -> DCP_ERR_INVALID_ARG."""
+    dev = "cuda"
+    T, H, d = 300, 2, 64
+    q, k, v, g = (x.to(dev) for x in inputs.make_qkvg(T, H, d, 62))
+    ws = B.alloc_workspace(T, 2, H, d, True, dev)
+    good = torch.tensor([0, 100, 300], dtype=torch.int32, device=dev)
+    bad = torch.tensor([0, 200, 100], dtype=torch.int32, device=dev)
+    B.dcp_varlen_attn_fwd(q, k, v, good, 200, False, workspace=ws)
+    B.dcp_query_status(ws)                                  # the header is initialised now
+    for code, err in ((1, B.DCP_ERR_TIMEOUT), (2, B.DCP_ERR_TIMEOUT), (3, B.DCP_ERR_INVALID_ARG)):
+        ws[:4].copy_(torch.tensor([code, 0, 0, 0], dtype=torch.uint8))
+        with pytest.raises(B.DcpError) as e:
+            B.dcp_query_status(ws)
+        assert e.value.code == err
+        B.dcp_query_status(ws)                              # cleared by the query
+    # a failing call followed by good calls on the same workspace: the failure is still reported
+    B.dcp_varlen_attn_fwd(q, k, v, bad, 200, False, workspace=ws)
+    o, lse = B.dcp_varlen_attn_fwd(q, k, v, good, 200, False, workspace=ws)
+    B.dcp_varlen_attn_bwd(q, k, v, o, g, lse, good, 200, False, workspace=ws)
+    with pytest.raises(B.DcpError) as e:
+        B.dcp_query_status(ws)
+    assert e.value.code == B.DCP_ERR_INVALID_ARG
+    B.dcp_query_status(ws)
+
+
+def test_bounded_wait_gives_up_and_reports_a_timeout():
+    """A wait on a barrier nothing arrives at: the kernels' wait helper stops after its poll limit, raises
+    the status word and the CTA returns; the context stays usable."""
+    dev = "cuda"
+    ws = torch.empty(4096, dtype=torch.uint8, device=dev)
+    B.dcp_selftest_wait_timeout(ws, 1 << 10)
+    with pytest.raises(B.DcpError) as e:
+        B.dcp_query_status(ws)
+    assert e.value.code == B.DCP_ERR_TIMEOUT
+    B.dcp_query_status(ws)
+    # the device still works afterwards
+    check_full([130, 40], 1, 64, True, seed=63)
+    with pytest.raises(B.DcpError):
+        B.dcp_selftest_wait_timeout(ws, (1 << 20) + 1)
+
+
+def test_input_order_work_list_gives_the_same_results():
+    # the measurement switch that lists sequences as they come changes the schedule, not the answers
+    lengths = [40, 700, 129, 13, 13, 300, 1]
+    try:
+        B.dcp_set_work_order(True)
+        check_full(lengths, 2, 128, True, seed=64)
+        check_full([int(x) for x in np.random.default_rng(9).integers(0, 50, size=1200)], 1, 64, False, seed=65)
+    finally:
+        B.dcp_set_work_order(False)
+
+
+def test_cta_spans_are_recorded():
+    dev = "cuda"
+    lengths = [2000, 700, 129]
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    q, k, v, g = (x.to(dev) for x in inputs.make_qkvg(int(cu[-1]), 4, 128, 66))
+    cud = torch.tensor(cu, device=dev)
+    ws = B.alloc_workspace(int(cu[-1]), 3, 4, 128, True, dev)
+    o, lse = B.dcp_varlen_attn_fwd(q, k, v, cud, 2000, False, workspace=ws)
+    B.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cud, 2000, False, workspace=ws)
+    n_sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for which in (0, 1):
+        begin, end = B.dcp_read_cta_spans(ws, which)
+        assert begin.size == min(n_sms, 256) and bool((end >= begin).all()) and bool((begin > 0).all())
+        assert int(end.max() - begin.min()) < 10 ** 9          # nanoseconds: well under a second

@@ -1,9 +1,11 @@
 """Full-size benchmark configurations (2 text, 3 video, 4 extreme imbalance, and the video clips
 seen along the spatial axis of a 2-D model) in the launch configuration the benchmark times; the
 temporal axis (20384 sequences of 1-13 tokens) is small enough for the oracle to check in full.  A full fp64 evaluation of these is 10^13-10^14 flop, so the
-oracle checks (a) sampled query rows (O, lse, dQ) and key columns (dK, dV), which the definition
-lets it compute one by one, (b) the shortest sequences completely, on every head, and (c) two
-whole-tensor identities that hold at any size:
+oracle checks (a) every sequence of at most 8192 tokens completely, on every head, (b) for longer
+sequences sampled query rows (O, lse, dQ) and key columns (dK, dV), which the definition lets it
+compute one by one - at least 256 rows on every head of the longest sequence, key columns from its
+first blocks included - plus one whole head of O and lse, and (c) two whole-tensor identities that
+hold at any size:
     sum_i <Q_i, dQ_i> = sum_j <K_j, dK_j>      and      sum_j dV_j = sum_i dO_i
 per (sequence, head), evaluated on the GPU results in fp64.  Their bounds have two parts: the
 independent bf16 rounding of every stored gradient element (8 sigma), and a term proportional to
@@ -17,6 +19,7 @@ import torch
 import oracle
 from paper_2608_07524_b200 import binding as B
 from paper_2608_07524_b200 import inputs
+from test_gpu_attn import Guarded
 
 pytestmark = pytest.mark.gpu
 
@@ -52,57 +55,86 @@ def full_run(request):
     dev = "cuda"
     q, k, v, g = inputs.make_qkvg_device(w.total_tokens, w.n_heads, w.head_dim, w.value_seed, dev)
     cud = torch.tensor(w.cu_seqlens, dtype=torch.int32, device=dev)
-    ws = B.alloc_workspace(w.total_tokens, len(w.lengths), w.n_heads, w.head_dim, True, dev)
-    o, lse = B.dcp_varlen_attn_fwd(q, k, v, cud, w.max_seqlen, w.causal, workspace=ws)
-    B.dcp_query_status(ws)
-    dq, dk, dv = B.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cud, w.max_seqlen, w.causal, workspace=ws)
-    B.dcp_query_status(ws)
-    del ws
+    # outputs and workspace carry a poisoned margin after their end (a store past the last row shows there)
+    buf = Guarded(w.total_tokens, w.n_heads, w.head_dim, len(w.lengths), dev)
+    o, lse = B.dcp_varlen_attn_fwd(q, k, v, cud, w.max_seqlen, w.causal, out=buf.o, lse=buf.lse, workspace=buf.ws)
+    B.dcp_query_status(buf.ws)
+    buf.assert_margins_untouched("forward")
+    dq, dk, dv = B.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cud, w.max_seqlen, w.causal, dq=buf.dq, dk=buf.dk, dv=buf.dv,
+                                       workspace=buf.ws)
+    B.dcp_query_status(buf.ws)
+    buf.assert_margins_untouched("backward")
+    del buf.ws, buf.ws_raw
     host = tuple(x.cpu() for x in (q, k, v, g))
     yield w, (q, k, v, g), host, (o, lse, dq, dk, dv)
     torch.cuda.empty_cache()
 
 
-def test_sampled_rows_and_columns(full_run):
+FULL_LIMIT = 8192      # sequences up to this length are compared in full, on every head
+
+
+def test_sequences_up_to_8192_tokens_in_full(full_run):
+    """Every sequence of at most 8192 tokens, every head, every element of o, lse, dq, dk, dv.  The
+    oracle sees them packed back to back as a batch of their own (attention is per sequence)."""
+    w, _, (q, k, v, g), (o, lse, dq, dk, dv) = full_run
+    seqs = [b for b, L in enumerate(w.lengths) if 0 < L <= FULL_LIMIT]
+    if not seqs:
+        pytest.skip("no sequence of at most 8192 tokens")
+    rows = np.concatenate([np.arange(w.cu_seqlens[b], w.cu_seqlens[b + 1]) for b in seqs])
+    sub_cu = np.concatenate([[0], np.cumsum([w.lengths[b] for b in seqs])]).astype(np.int32)
+    idx_h = torch.from_numpy(rows)
+    qs, ks, vs, gs = (x[idx_h].contiguous() for x in (q, k, v, g))
+    O, Lse = oracle.attn_fwd(qs, ks, vs, sub_cu, w.causal)
+    rdq, rdk, rdv = oracle.attn_bwd(qs, ks, vs, gs, sub_cu, w.causal)
+    idx = idx_h.cuda()
+    close("o", o[idx], O)
+    close("dq", dq[idx], rdq)
+    close("dk", dk[idx], rdk)
+    close("dv", dv[idx], rdv)
+    assert float(np.max(np.abs(lse[:, idx].double().cpu().numpy() - Lse))) <= LSE_ABS
+
+
+def test_long_sequences_by_rows_columns_and_one_full_head(full_run):
+    """Sequences longer than 8192 tokens.  The longest one: at least 256 sampled query rows (o, lse, dq) on
+    EVERY head, one head's o and lse completely, and sampled key columns (dk, dv) that include the first key
+    blocks - under a causal mask those are the columns that accumulate over the most query tiles (up to 1024
+    for the 131072-token sequence), and the oracle needs the statistics of every later row for them, i.e.
+    one full pass over the head.  The other long sequences: sampled rows on two heads and columns on one."""
     w, _, (q, k, v, g), (o, lse, dq, dk, dv) = full_run
     rng = np.random.default_rng(100 + len(w.lengths))
-    order = np.argsort(w.lengths)
-    seqs = [int(order[-1]), int(order[len(order) // 2]), int(order[0])]      # longest, median, shortest
-    for seq in seqs:
+    long_seqs = [b for b, L in enumerate(w.lengths) if L > FULL_LIMIT]
+    if not long_seqs:
+        pytest.skip("no sequence longer than 8192 tokens")
+    longest = max(long_seqs, key=lambda b: w.lengths[b])
+    for seq in long_seqs:
         L, c0 = w.lengths[seq], w.cu_seqlens[seq]
-        for head in (0, w.n_heads - 1):
-            rows = sample_positions(L, rng)
+        heads = range(w.n_heads) if seq == longest else (0, w.n_heads - 1)
+        for head in heads:
+            rows = sample_positions(L, rng, n_random=260 if seq == longest else 24)
+            assert seq != longest or rows.size >= 256
             Or, lr, dqr = oracle.attn_rows(q, k, v, g, w.cu_seqlens, w.causal, seq, head, rows)
             idx = torch.tensor(c0 + rows, device="cuda").long()
             close(f"o seq {seq} head {head}", o[idx, head], Or)
             close(f"dq seq {seq} head {head}", dq[idx, head], dqr)
             assert float(np.max(np.abs(lse[head, idx].double().cpu().numpy() - lr))) <= LSE_ABS
-        # columns: one head per sequence.  Under a causal mask a column needs the statistics of
-        # every later row, so for very long sequences only columns near the end are sampled here
-        # (early columns are covered by the identities and by the shorter sequences).
         head = 1
         cols = sample_positions(L, rng, n_random=8)
-        if w.causal and L > 16384:
-            cols = cols[cols >= L - 2048]
+        if seq == longest:
+            early = np.concatenate([[0, 1, 127, 128, 255], rng.integers(0, 4096, size=8)])
+            cols = np.unique(np.concatenate([cols, early])).astype(np.int32)
+        elif w.causal:
+            cols = cols[cols >= L - 2048]          # keeps the row pass short for the sequences that are not the longest
         dkc, dvc = oracle.attn_cols(q, k, v, g, w.cu_seqlens, w.causal, seq, head, cols)
         idx = torch.tensor(c0 + cols, device="cuda").long()
         close(f"dk seq {seq}", dk[idx, head], dkc)
         close(f"dv seq {seq}", dv[idx, head], dvc)
-
-
-def test_shortest_sequences_in_full(full_run):
-    w, _, (q, k, v, g), (o, lse, dq, dk, dv) = full_run
-    order = np.argsort(w.lengths)
-    for seq in (int(order[0]), int(order[1])):
-        L, c0 = w.lengths[seq], w.cu_seqlens[seq]
-        sl = slice(c0, c0 + L)
-        O, Lse = oracle.attn_fwd(q[sl], k[sl], v[sl], [0, L], w.causal)
-        rdq, rdk, rdv = oracle.attn_bwd(q[sl], k[sl], v[sl], g[sl], [0, L], w.causal)
-        close("o", o[sl], O)
-        close("dq", dq[sl], rdq)
-        close("dk", dk[sl], rdk)
-        close("dv", dv[sl], rdv)
-        assert float(np.max(np.abs(lse[:, sl].double().cpu().numpy() - Lse))) <= LSE_ABS
+    # one whole head of the longest sequence
+    L, c0, head = w.lengths[longest], w.cu_seqlens[longest], 2
+    sl = slice(c0, c0 + L)
+    O, Lse = oracle.attn_fwd(q[sl, head:head + 1].contiguous(), k[sl, head:head + 1].contiguous(),
+                             v[sl, head:head + 1].contiguous(), [0, L], w.causal)
+    close("o, one full head", o[sl, head:head + 1], O)
+    assert float(np.max(np.abs(lse[head:head + 1, sl].double().cpu().numpy() - Lse))) <= LSE_ABS
 
 
 def test_whole_tensor_identities(full_run):

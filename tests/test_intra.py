@@ -1,5 +1,6 @@
-"""DCP-intra selection (Algorithm 1): the library's dcp_intra_select against the plain-Python oracle,
-and the oracle against what Eq. 4-6 fix independently of the algorithm's loop."""
+"""DCP-intra selection (Algorithm 1): the library's dcp_intra_select against the exhaustive oracle, and
+the oracle against what Eq. 4-6 fix independently of any search: per candidate the number of layers
+that may keep their activations has a closed form, and a hand-worked example."""
 from fractions import Fraction
 
 import numpy as np
@@ -10,19 +11,18 @@ from oracle.intra_oracle import Infeasible
 from paper_2608_07524_b200 import binding as B
 
 
-def from_equations(cands, M, L):
-    """Best (throughput, candidate, r) straight from Eq. 4-6: T(r) = T_f + T_b + r t_f + T_C and
-    M(r) = (L - r) m + L m_inp + M_C, so relative to the profile at r = L:
-    T(r) = T_(b,p) - (L - r) t_f and M(r) = M_(b,p) + (L - r) m.  Every feasible r is tried."""
+def from_closed_form(cands, M, L):
+    """Eq. 6: M(r) = M_(b,p) + (L - r) m <= M  <=>  L - r <= (M - M_(b,p)) / m, so the smallest feasible r
+    is L - min(L, floor((M - M_(b,p)) / m)); Eq. 5 then gives the time.  Best throughput over candidates."""
     best = None
     for idx, (b, p, t_f, m, T_bp, M_bp) in enumerate(cands):
-        for r in range(L + 1):
-            if M_bp + (L - r) * m > M:
-                continue
-            thr = Fraction(b, p * (T_bp - (L - r) * t_f))
-            key = (thr, -p, b, -idx, -r)
-            if best is None or key > best[0]:
-                best = (key, idx, r, T_bp - (L - r) * t_f)
+        if M_bp > M:
+            continue
+        keep = L if m == 0 else min(L, (M - M_bp) // m)
+        time = T_bp - keep * t_f
+        key = (Fraction(b, p * time), -p, b, -idx)
+        if best is None or key > best[0]:
+            best = (key, idx, L - keep, time)
     return None if best is None else best[1:]
 
 
@@ -41,11 +41,11 @@ def random_case(rng):
     return cands, M, L
 
 
-def test_oracle_matches_the_equations_and_library_matches_oracle():
+def test_oracle_matches_the_closed_form_and_library_matches_oracle():
     rng = np.random.default_rng(21)
     for _ in range(3000):
         cands, M, L = random_case(rng)
-        ref = from_equations(cands, M, L)
+        ref = from_closed_form(cands, M, L)
         try:
             got_o = oracle.intra_select(cands, M, L)
         except Infeasible:
@@ -82,6 +82,7 @@ def test_equal_b_and_p_reduces_to_the_smallest_time():
         cands = [(3, 2) + c[2:] for c in cands]
         M = max(M, max(c[5] for c in cands))
         idx, r, t = B.dcp_intra_select(cands, M, L)
+        assert oracle.intra_select(cands, M, L) == (idx, r, t)
         times = [c[4] - min(L, (M - c[5]) // c[3] if c[3] else L) * c[2] for c in cands]
         assert t == min(times) and idx == times.index(min(times))
 

@@ -53,7 +53,7 @@ def set_partitions(items):
 
 
 def block_cost(block, budget, H, d, e, lam, MC, TC):
-    """Eq. 4-6 as read in the design notes, written independently of the C oracle, in Python ints."""
+    """Eq. 4-6 (r = recomputed layers, m = 4 tok H d e, m_inp = tok H d e), written independently of the C oracle, in Python ints."""
     tok = sum(block)
     W = sum(x * x for x in block)
     unit = tok * H * d * e
@@ -166,3 +166,36 @@ def test_rejects_bad_arguments():
         oracle.plan_bruteforce([0, 5], 1000)
     with pytest.raises(ValueError):
         oracle.plan_bruteforce([5] * 25, 10 ** 12)
+
+
+def test_weighted_hand_worked_case_with_unsorted_unequal_lengths():
+    """Profiled variant (Section 3.5 feeding Eq. 5): weight[i] belongs to INPUT sequence i.
+    H = d = e = 1, Lambda = 1: a block of tok tokens needs 5 tok bytes at r = 0 and tok at r = 1.
+    Lengths in input order (25, 10, 30) with weights (7, 100, 2); sorted order is 30, 25, 10.
+    Budget 150: r = 0 iff tok <= 30, r = 1 otherwise (every block has tok <= 65 <= 150).  T_C = 50.
+      [30, 25, 10]           r = 1        cost  50 + (2 + 7 + 100)      = 159
+      [30] [25, 10]          r = 0, 1     cost 100 + (7 + 100)          = 207
+      [30, 25] [10]          r = 1, 0     cost 100 + (2 + 7)            = 109   <- optimum
+      [30] [25] [10]         r = 0, 0, 0  cost 150
+    Reading the weights by sorted position instead (30 -> 7, 25 -> 100, 10 -> 2) would give
+    159 / 202 / 207 / 150 and pick three blocks at cost 150."""
+    kw = dict(n_heads=1, head_dim=1, elt_bytes=1, n_layers=1, fixed_cost=50)
+    assert oracle.plan_bruteforce([25, 10, 30], 150, fwd_time=[7, 100, 2], **kw) == ([0, 1, 0], [1, 0], 109)
+    # the same batch presented in another order: the plan follows the sequences, not the positions
+    assert oracle.plan_bruteforce([30, 25, 10], 150, fwd_time=[2, 7, 100], **kw) == ([0, 0, 1], [1, 0], 109)
+    assert oracle.plan_bruteforce([10, 30, 25], 150, fwd_time=[100, 2, 7], **kw) == ([1, 0, 0], [1, 0], 109)
+
+
+def test_weighted_with_model_times_equals_the_unweighted_oracle():
+    # weight[i] = 2 L_i^2 is the analytic stand-in itself: both entry paths must agree on every output
+    rng = np.random.default_rng(17)
+    for _ in range(300):
+        n = int(rng.integers(1, 10))
+        lengths = [int(x) for x in rng.integers(1, 600, size=n)]
+        lam = int(rng.choice([1, 2, 5]))
+        TC = int(rng.choice([0, 7, 10 ** 4, 1 << 24]))
+        unit = 3 * 8 * 2
+        budget = int(rng.integers(lam * unit * max(lengths), 5 * lam * unit * sum(lengths) + 2))
+        kw = dict(n_heads=3, head_dim=8, n_layers=lam, fixed_cost=TC)
+        assert oracle.plan_bruteforce(lengths, budget, fwd_time=[2 * L * L for L in lengths], **kw) == \
+            oracle.plan_bruteforce(lengths, budget, **kw)

@@ -77,8 +77,54 @@ def test_stream_batches_literal_and_binding_settings():
 
 def test_plan_batch_groups_sequences():
     lengths = [17, 64, 100, 255]
-    mbs = plan_batch(lengths, 65280, n_heads=2, head_dim=64)
-    assert [m.lengths for m in mbs] == [[255], [100, 64, 17]] and [m.recompute for m in mbs] == [1, 1]
+    plan = plan_batch(lengths, 65280, n_heads=2, head_dim=64)
+    mbs = plan.micro_batches
+    # micro-batch 0 holds the longest sequence; inside a micro-batch sequences keep their input order
+    assert [list(m.lengths) for m in mbs] == [[255], [17, 64, 100]] and [m.recompute for m in mbs] == [1, 1]
+    assert [list(m.seq_index) for m in mbs] == [[3], [0, 1, 2]] and plan.mb_id == [1, 1, 1, 0]
+    # copy lists: (row in the batch, row in the micro-batch, rows), long sequences cut into pieces of 64 rows
+    assert mbs[0].seg.tolist() == [[181, 0, 64], [245, 64, 64], [309, 128, 64], [373, 192, 63]]
+    assert mbs[1].seg.tolist() == [[0, 0, 17], [17, 17, 64], [81, 81, 64], [145, 145, 36]]
+    # a plan that does not split runs in place
+    one = plan_batch(lengths, 10 ** 6, n_heads=2, head_dim=64)
+    assert len(one.micro_batches) == 1 and one.micro_batches[0].seg is None
+    assert list(one.micro_batches[0].lengths) == lengths
+
+
+def reference_segments(lengths, mb_id, K, max_rows):
+    """The layout written out plainly: per micro-batch the input indices in input order, its boundary
+    array, and one copy piece per max_rows rows of every sequence."""
+    src = np.concatenate([[0], np.cumsum(lengths)])
+    offs, index, cu, seg_off, seg = [0], [], [], [0], []
+    for k in range(K):
+        members = [i for i in range(len(lengths)) if mb_id[i] == k]
+        index += members
+        offs.append(len(index))
+        dst = 0
+        cu.append(0)
+        for i in members:
+            for done in range(0, lengths[i], max_rows):
+                seg.append([int(src[i]) + done, dst + done, min(max_rows, lengths[i] - done)])
+            dst += lengths[i]
+            cu.append(dst)
+        seg_off.append(len(seg))
+    return offs, index, cu, seg_off, seg
+
+
+def test_plan_segments_against_a_plain_restatement():
+    rng = np.random.default_rng(8)
+    for _ in range(300):
+        n = int(rng.integers(1, 30))
+        lengths = [int(x) for x in rng.choice([0, 1, 5, 63, 64, 65, 128, 300, 1000], size=n)]
+        K = int(rng.integers(1, n + 1))
+        mb_id = [int(x) for x in rng.integers(0, K, size=n)]
+        max_rows = int(rng.choice([1, 7, 64, 1000]))
+        got = B.dcp_plan_segments(lengths, mb_id, K, max_rows)
+        ref = reference_segments(lengths, mb_id, K, max_rows)
+        assert [x.tolist() for x in got] == [list(x) for x in ref]
+    with pytest.raises(B.DcpError) as e:
+        B.dcp_plan_segments([5, 6], [0, 2], 2)
+    assert e.value.code == B.DCP_ERR_INVALID_ARG
 
 
 def test_errors():

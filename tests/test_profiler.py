@@ -5,7 +5,8 @@ import pytest
 
 import oracle
 from paper_2608_07524_b200 import binding as B
-from paper_2608_07524_b200.profiler import ProfileTable, dual_layer_profile
+from oracle import profile_oracle
+from paper_2608_07524_b200.profiler import ProfileTable, dual_layer_profile, intra_candidates, select_group_setting
 from paper_2608_07524_b200.stream import plan_batch
 
 
@@ -70,21 +71,77 @@ def test_profiled_argument_errors():
     assert e.value.code in (B.DCP_ERR_OVERFLOW, B.DCP_ERR_INFEASIBLE)
 
 
-def test_interpolation_rule():
+def test_interpolation_oracle_hand_values():
+    # pins of the plain-Python oracle: values worked by hand from the rule (linear below the first bucket,
+    # linear between buckets, quadratic above the last, floor division)
+    xs, f, b = [100, 200, 400], [1000, 3000, 11000], [2000, 7000, 30000]
+    o = profile_oracle.interp
+    assert [o(xs, f, L) for L in (100, 200, 400)] == [1000, 3000, 11000]
+    assert o(xs, f, 50) == 500 and o(xs, f, 1) == 10                   # 1000 * L / 100
+    assert o(xs, f, 150) == 2000 and o(xs, f, 201) == 3040             # 3000 + 8000 * 1 / 200
+    assert o(xs, f, 800) == 44000 and o(xs, f, 401) == 11000 * 401 * 401 // 160000
+    assert o(xs, b, 300) == 18500
+    vals = [o(xs, f, L) for L in range(1, 1000)]
+    assert all(y >= x for x, y in zip(vals, vals[1:]))
+    assert o([10, 20], [9, 2], 13) == 6                                # falling table: 9 + floor(-7 * 3 / 10) = 9 - 3
+    # Eq. 4-5: Lambda (t_f + t_b) + r t_f + T_C; at r = Lambda it is Section 3.5's Lambda (2 t_f + t_b) + T_C
+    assert profile_oracle.model_time([1000, 3000], [2000, 7000], 3, 2, 7) == 3 * (4000 + 9000) + 2 * 4000 + 7
+    assert profile_oracle.model_time([5], [11], 4, 4, 9) == 4 * (2 * 5 + 11) + 9
+    assert profile_oracle.candidate(2, 1, 5, 11, 40, 10, 4, 3, 9) == (2, 1, 5, 40, 4 * (2 * 5 + 11) + 9, 4 * 10 + 3)
+
+
+def test_library_interpolation_and_model_time_match_the_oracle():
     t = ProfileTable([100, 200, 400], [1000, 3000, 11000], [2000, 7000, 30000], [1, 2, 4])
-    assert [t.fwd_time(L) for L in (100, 200, 400)] == [1000, 3000, 11000]
-    assert t.fwd_time(50) == 500 and t.fwd_time(1) == 10            # linear below the first bucket
-    assert t.fwd_time(150) == 2000 and t.fwd_time(201) == 3040      # linear between, floor
-    assert t.fwd_time(800) == 44000 and t.fwd_time(401) == 11000 * 401 * 401 // 160000   # quadratic above
-    assert t.bwd_time(300) == 18500
-    xs = [t.fwd_time(L) for L in range(1, 1000)]
-    assert all(b >= a for a, b in zip(xs, xs[1:]))
-    # Eq. 4-5: Lambda (t_f + t_b) + r t_f + T_C
+    assert t.fwd_time(150) == 2000 and t.bwd_time(300) == 18500 and t.fwd_time(800) == 44000
+    rng = np.random.default_rng(31)
+    for _ in range(300):
+        nb = int(rng.integers(1, 8))
+        xs = sorted(set(int(x) for x in rng.integers(1, 5000, size=nb)))
+        ys = [int(x) for x in rng.integers(0, 10 ** int(rng.integers(1, 12)), size=len(xs))]
+        ls = [int(x) for x in rng.integers(1, 9000, size=20)] + xs
+        assert B.dcp_profile_interp(xs, ys, ls) == [profile_oracle.interp(xs, ys, L) for L in ls]
+        f = [int(x) for x in rng.integers(0, 10 ** 9, size=6)]
+        b = [int(x) for x in rng.integers(0, 10 ** 9, size=6)]
+        lam = int(rng.integers(1, 40))
+        r = int(rng.integers(0, lam + 1))
+        assert B.dcp_model_time(f, b, lam, r, 12345) == profile_oracle.model_time(f, b, lam, r, 12345)
+        args = (int(rng.integers(1, 9)), 1, f[0], b[0], f[1], f[2], lam, f[3], f[4])
+        assert B.dcp_intra_candidate_from_profile(*args) == profile_oracle.candidate(*args)
     assert t.model_time([100, 200], 3, 2, 7) == 3 * (4000 + 9000) + 2 * 4000 + 7
     with pytest.raises(ValueError):
         ProfileTable([100, 100], [1, 2], [1, 2], [1, 2])
-    with pytest.raises(ValueError):
+    with pytest.raises(B.DcpError) as e:
         t.fwd_time(0)
+    assert e.value.code == B.DCP_ERR_INVALID_ARG
+    with pytest.raises(B.DcpError):
+        B.dcp_profile_interp([5, 5], [1, 2], [3])
+    with pytest.raises(B.DcpError) as e:
+        B.dcp_profile_interp([5], [2 ** 62], [500])
+    assert e.value.code == B.DCP_ERR_OVERFLOW
+
+
+def test_algorithm_1_table_from_a_fake_profile():
+    # forward 1 ms per sequence of the batch, backward 3 ms, whatever b: per-sequence time is flat, so the
+    # throughput b / T is the same for every b and only memory decides how many layers are recomputed
+    runs = []
+
+    def fake_layer(lengths):
+        runs.append(len(lengths))
+        return 1.0 * len(lengths), 3.0 * len(lengths)
+
+    H, d, L, lam = 4, 32, 1000, 6
+    cands = intra_candidates(L, [1, 2, 4], H, d, False, lam, run_layer=fake_layer, fixed_cost_ns=500)
+    assert runs == [1, 1, 2, 2, 4, 4]                                    # warm-up + recorded run per batch size
+    unit = L * H * d * 2
+    assert cands == [profile_oracle.candidate(b, 1, b * 10 ** 6, 3 * b * 10 ** 6, 4 * b * unit, b * unit, lam, 0, 500)
+                     for b in (1, 2, 4)]
+    # capacity for b = 4 with no layer kept, b = 2 with one kept, b = 1 with all six kept
+    cap = lam * 4 * unit
+    b, r, t = select_group_setting(cands, cap, lam)
+    assert (b, r, t) == (lambda i, rr, tt: (cands[i][0], rr, tt))(*oracle.intra_select(cands, cap, lam))
+    # b = 1 keeps floor((24 - 6) / 4) = 4 layers: T = 6 * 5 ms + 500 - 4 * 1 ms = 26 ms + 500 ns per sequence;
+    # b = 2 keeps (24 - 12) / 8 = 1: (60 ms + 500 - 2 ms) / 2 = 29 ms; b = 4 keeps none: 30 ms per sequence
+    assert (b, r, t) == (1, 2, 26 * 10 ** 6 + 500)
 
 
 def test_dual_layer_profile_keeps_the_second_run():
@@ -112,11 +169,11 @@ def test_plan_batch_with_profile_uses_measured_times():
     budget = 3 * unit * sum(lengths)              # all four together only fit when recomputed
     cheap = ProfileTable([1000, 4000], [1, 4], [1, 4], [1, 1])
     dear = ProfileTable([1000, 4000], [10 ** 6, 16 * 10 ** 6], [1, 4], [1, 1])
-    one = plan_batch(lengths, budget, 16, 128, n_layers=1, fixed_cost=1000, profile=cheap)
-    assert [m.lengths for m in one] == [lengths] and one[0].recompute == 1
-    many = plan_batch(lengths, budget, 16, 128, n_layers=1, fixed_cost=1000, profile=dear)
+    one = plan_batch(lengths, budget, 16, 128, n_layers=1, fixed_cost=1000, profile=cheap).micro_batches
+    assert [list(m.lengths) for m in one] == [lengths] and one[0].recompute == 1 and one[0].seg is None
+    many = plan_batch(lengths, budget, 16, 128, n_layers=1, fixed_cost=1000, profile=dear).micro_batches
     assert len(many) == 2 and all(m.recompute == 0 for m in many)
-    assert sorted(sum((m.lengths for m in many), [])) == sorted(lengths)
+    assert sorted(sum((list(m.lengths) for m in many), [])) == sorted(lengths)
 
 
 @pytest.mark.gpu
@@ -128,8 +185,8 @@ def test_profile_on_device_and_plan():
     assert 8 < t.t_f_ns[2] / t.t_f_ns[1] < 20
     assert all(b > f for f, b in zip(t.t_f_ns, t.t_b_ns))
     lengths = [9600, 9600, 3600, 2048, 1024, 256]
-    mbs = plan_batch(lengths, 5 * 16 * 128 * 2 * 14000, 16, 128, n_layers=1, fixed_cost=20000, profile=t)
-    assert sorted(sum((m.lengths for m in mbs), [])) == sorted(lengths)
+    plan = plan_batch(lengths, 5 * 16 * 128 * 2 * 14000, 16, 128, n_layers=1, fixed_cost=20000, profile=t)
+    assert sorted(sum((list(m.lengths) for m in plan.micro_batches), [])) == sorted(lengths)
     ref = oracle.plan_bruteforce(lengths, 5 * 16 * 128 * 2 * 14000, fixed_cost=20000,
-                                 fwd_time=[t.fwd_time(L) for L in lengths])
-    assert [m.recompute for m in mbs] == ref[1]
+                                 fwd_time=[profile_oracle.interp(t.lengths, t.t_f_ns, L) for L in lengths])
+    assert (plan.mb_id, plan.recompute, plan.cost) == ref
