@@ -247,7 +247,10 @@ class Job:
         from paper_2608_07524_b200 import binding as B
         out = {}
         for which, key in ((0, "fwd"), (1, "bwd_main")):
-            begin, end = B.dcp_read_cta_spans(self.runner.ws, which)
+            try:
+                begin, end = B.dcp_read_cta_spans(self.runner.ws, which)
+            except B.DcpError:
+                continue
             if begin.size == 0:
                 continue
             busy = self.np.sort((end - begin).astype(self.np.float64)) / 1e6

@@ -54,6 +54,7 @@ static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
 __device__ __forceinline__ void header_begin_call(WorkspaceHeader* hdr, bool bad) {
     if (hdr->magic[0] != kHeaderMagic0 || hdr->magic[1] != kHeaderMagic1) {
         hdr->status = kStatusOk;
+        hdr->n_ctas[0] = hdr->n_ctas[1] = 0;
         hdr->magic[0] = kHeaderMagic0;
         hdr->magic[1] = kHeaderMagic1;
     }

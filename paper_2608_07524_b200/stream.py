@@ -68,6 +68,25 @@ def plan_batch(lengths: Sequence[int], hbm_budget_bytes: int, n_heads: int, head
     return plan
 
 
+def plan_length_group(n_seqs: int, seq_len: int, batch_size: int, recompute: int) -> BatchPlan:
+    """The plan of a group of n_seqs sequences of one length run with the setting Algorithm 1 selected
+    for that length (Section 3.4): micro-batches of `batch_size` sequences each, every one with
+    `recompute` recomputed layers.  Consecutive sequences share a micro-batch."""
+    if n_seqs < 1 or batch_size < 1 or recompute < 0:
+        raise ValueError("need n_seqs >= 1, batch_size >= 1, recompute >= 0")
+    lengths = [int(seq_len)] * n_seqs
+    mb_id = [i // batch_size for i in range(n_seqs)]
+    K = mb_id[-1] + 1
+    mb_seq_offset, seq_index, _, seg_offset, seg = binding.dcp_plan_segments(lengths, mb_id, K, SEG_ROWS)
+    lens = np.asarray(lengths, dtype=np.int32)
+    plan = BatchPlan(mb_id, [int(recompute)] * K, 0)
+    for k in range(K):
+        idx = seq_index[mb_seq_offset[k]: mb_seq_offset[k + 1]]
+        plan.micro_batches.append(MicroBatch(lens[idx], int(recompute), idx,
+                                             None if K == 1 else seg[seg_offset[k]: seg_offset[k + 1]]))
+    return plan
+
+
 class _Buffers:
     """q, k, v, dO, o, dq, dk, dv [tokens, H, d] bf16 and lse [H * tokens] fp32 on the device."""
 

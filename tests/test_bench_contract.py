@@ -58,3 +58,7 @@ def test_cuda_arm_prints_the_contract_line():
     assert line["clocks"]["sm_max_mhz"] >= line["clocks"]["sm_mhz"] > 0
     base = line["cpu_baseline"]
     assert base["kind"] == "oracle" and base["value"] > 0 and base["cores"] >= 1
+    busy = line["sm_busy"]
+    assert busy["fwd"]["ctas"] > 0 and busy["bwd_main"]["max_over_mean"] >= 1.0
+    assert set(line["others"]) == {"video", "extreme", "stream", "spatial2d", "temporal2d"}
+    assert all("error" not in o and o["value"] > 0 for o in line["others"].values())

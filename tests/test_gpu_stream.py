@@ -11,7 +11,8 @@ import torch
 import oracle
 from paper_2608_07524_b200 import binding as B
 from paper_2608_07524_b200 import inputs
-from paper_2608_07524_b200.stream import StreamRunner, plan_batch
+from paper_2608_07524_b200.profiler import intra_candidates, select_group_setting
+from paper_2608_07524_b200.stream import StreamRunner, plan_batch, plan_length_group
 
 pytestmark = pytest.mark.gpu
 
@@ -118,3 +119,42 @@ def test_copy_segments_gathers_and_scatters():
         B.dcp_copy_segments(lk, lse_back, segk, segk.shape[0], 4, reverse=True, n_planes=5, src_plane_bytes=4 * Tk,
                             dst_plane_bytes=4 * T)
     assert torch.equal(back, x) and torch.equal(lse_back, lse)
+
+
+def test_algorithm_1_setting_measured_on_the_device_and_applied():
+    """DCP-intra on one GPU (p = 1): the candidate table (b, 1) for one sequence length is measured the
+    dual-layer way on this device, Algorithm 1 selects batch size and recompute count under a memory
+    capacity, the selection is compared with the exhaustive oracle on the SAME measured table, and a group
+    of sequences of that length is then run with the selected setting and compared with the attention
+    oracle."""
+    L, n_seqs, lam = 384, 7, 4
+    cands = intra_candidates(L, [1, 2, 4], H, D, False, lam, fixed_cost_ns=20000)
+    assert all(c[2] > 0 and c[4] > lam * 2 * c[2] for c in cands)
+    unit = L * H * D * 2
+    # room for b = 4 with nothing kept, for b = 2 with two layers kept, for b = 1 with all four kept
+    capacity = lam * 4 * unit + 4 * unit
+    b, r, t = select_group_setting(cands, capacity, lam)
+    idx, r_ref, t_ref = oracle.intra_select(cands, capacity, lam)
+    assert (b, r, t) == (cands[idx][0], r_ref, t_ref)
+    if r == 0:                                     # make sure the recompute path runs whatever the device measured
+        capacity = lam * b * unit + b * unit * 4 * (lam - 1)
+        b2, r, t = select_group_setting([c for c in cands if c[0] == b], capacity, lam)
+        assert b2 == b and r == 1
+    plan = plan_length_group(n_seqs, L, b, r)
+    assert len(plan.micro_batches) == -(-n_seqs // b) and all(m.recompute == r for m in plan.micro_batches)
+    T = n_seqs * L
+    cu = np.arange(0, T + 1, L, dtype=np.int32)
+    q, k, v, g = inputs.make_qkvg(T, H, D, 71)
+    runner = StreamRunner(T, n_seqs, H, D, False, "cuda")
+    runner.verify_recompute = True
+    load_batch(runner, q, k, v, g)
+    assert runner.run_batch(plan, T) == T
+    runner.check()
+    assert runner.recompute_mismatches == 0
+    O, Lse = oracle.attn_fwd(q, k, v, cu, False)
+    rdq, rdk, rdv = oracle.attn_bwd(q, k, v, g, cu, False)
+    close("o", runner.o[:T], O)
+    close("dq", runner.dq[:T], rdq)
+    close("dk", runner.dk[:T], rdk)
+    close("dv", runner.dv[:T], rdv)
+    assert float(np.max(np.abs(runner.lse[: H * T].view(H, T).double().cpu().numpy() - Lse))) <= LSE_ABS
