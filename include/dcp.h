@@ -149,6 +149,17 @@ int dcp_intra_candidate_from_profile(int32_t batch_size, int32_t sp_size, int64_
                                      int64_t inp_bytes, int32_t n_layers, int64_t const_bytes, int64_t fixed_cost,
                                      dcp_intra_candidate* out);
 
+/* The planner's memory model for `tokens` tokens of one micro-batch (Eq. 6 with the sizes this build's
+ * benchmark fixes): a layer that is not recomputed keeps act_bytes = m = 4 * tokens * H * d * e (q, k, v, o),
+ * every layer keeps its input, inp_bytes = m_inp = tokens * H * d * e.  Host pointers. */
+int dcp_activation_bytes(int64_t tokens, int32_t n_heads, int32_t head_dim, int32_t elt_bytes, int64_t* act_bytes,
+                         int64_t* inp_bytes);
+
+/* Micro-batches of a group of n_seqs sequences of one length run with the batch size Algorithm 1 selected
+ * for that length (Section 3.4): consecutive sequences share a micro-batch, mb_id [n_seqs] (host) = i / b,
+ * *n_mb = ceil(n_seqs / b).  Feed mb_id to dcp_plan_segments. */
+int dcp_length_group_plan(int32_t n_seqs, int32_t batch_size, int32_t* mb_id, int32_t* n_mb);
+
 /* Which rank owns which sequence when a batch is sharded over world_size GPUs without any
  * data-path collective (every (sequence, head) is independent).
  *

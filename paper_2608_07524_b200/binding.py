@@ -91,6 +91,10 @@ def lib():
             L.dcp_intra_candidate_from_profile.argtypes = [i32, i32, i64, i64, i64, i64, i32, i64, i64,
                                                            ctypes.POINTER(IntraCandidate)]
             L.dcp_intra_candidate_from_profile.restype = ctypes.c_int
+            L.dcp_activation_bytes.argtypes = [i64, i32, i32, i32, i64p, i64p]
+            L.dcp_activation_bytes.restype = ctypes.c_int
+            L.dcp_length_group_plan.argtypes = [i32, i32, i32p, i32p]
+            L.dcp_length_group_plan.restype = ctypes.c_int
             L.dcp_shard_sequences.argtypes = [i32p, i32, i32, i32p, i64p]
             L.dcp_shard_sequences.restype = ctypes.c_int
             L.dcp_profile_enable.argtypes = [ctypes.c_int]
@@ -376,6 +380,23 @@ def dcp_intra_candidate_from_profile(batch_size: int, sp_size: int, t_f: int, t_
                                                   int(inp_bytes), int(n_layers), int(const_bytes), int(fixed_cost),
                                                   ctypes.byref(c)))
     return (c.batch_size, c.sp_size, c.t_f, c.m, c.time_full, c.mem_full)
+
+
+def dcp_activation_bytes(tokens: int, n_heads: int, head_dim: int, elt_bytes: int = 2) -> Tuple[int, int]:
+    """(m, m_inp) of the planner's memory model for `tokens` tokens: bytes a layer keeps when it is not
+    recomputed, and the bytes of its input."""
+    act, inp = ctypes.c_int64(0), ctypes.c_int64(0)
+    _check(lib().dcp_activation_bytes(int(tokens), int(n_heads), int(head_dim), int(elt_bytes), ctypes.byref(act),
+                                      ctypes.byref(inp)))
+    return int(act.value), int(inp.value)
+
+
+def dcp_length_group_plan(n_seqs: int, batch_size: int) -> Tuple[List[int], int]:
+    """(mb_id [n_seqs], n_mb): consecutive sequences of a length group in micro-batches of batch_size."""
+    mb = (ctypes.c_int32 * max(n_seqs, 1))()
+    n_mb = ctypes.c_int32(0)
+    _check(lib().dcp_length_group_plan(int(n_seqs), int(batch_size), mb, ctypes.byref(n_mb)))
+    return list(mb[:n_seqs]), int(n_mb.value)
 
 
 def dcp_shard_sequences(lengths, world_size: int):

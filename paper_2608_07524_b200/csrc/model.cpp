@@ -98,6 +98,28 @@ extern "C" int dcp_intra_candidate_from_profile(int32_t batch_size, int32_t sp_s
     return DCP_OK;
 }
 
+extern "C" int dcp_activation_bytes(int64_t tokens, int32_t n_heads, int32_t head_dim, int32_t elt_bytes, int64_t* act_bytes,
+                                    int64_t* inp_bytes) {
+    const char* who = "dcp_activation_bytes";
+    if (!act_bytes || !inp_bytes) return dcp::fail(DCP_ERR_INVALID_ARG, "%s: null pointer", who);
+    if (tokens < 0 || n_heads < 1 || head_dim < 1 || elt_bytes < 1)
+        return dcp::fail(DCP_ERR_INVALID_ARG, "%s: need tokens >= 0 and H, d, e >= 1", who);
+    const i128 unit = (i128)tokens * n_heads * head_dim * elt_bytes;
+    if (4 * unit > kMax) return dcp::fail(DCP_ERR_OVERFLOW, "%s: size does not fit in int64", who);
+    *act_bytes = (int64_t)(4 * unit);
+    *inp_bytes = (int64_t)unit;
+    return DCP_OK;
+}
+
+extern "C" int dcp_length_group_plan(int32_t n_seqs, int32_t batch_size, int32_t* mb_id, int32_t* n_mb) {
+    const char* who = "dcp_length_group_plan";
+    if (!mb_id || !n_mb) return dcp::fail(DCP_ERR_INVALID_ARG, "%s: null pointer", who);
+    if (n_seqs < 1 || batch_size < 1) return dcp::fail(DCP_ERR_INVALID_ARG, "%s: need n_seqs >= 1 and batch_size >= 1", who);
+    for (int32_t i = 0; i < n_seqs; ++i) mb_id[i] = i / batch_size;
+    *n_mb = (n_seqs + batch_size - 1) / batch_size;
+    return DCP_OK;
+}
+
 extern "C" int dcp_shard_sequences(const int32_t* lengths, int32_t n, int32_t world_size, int32_t* rank_of,
                                    int64_t* load) {
     const char* who = "dcp_shard_sequences";

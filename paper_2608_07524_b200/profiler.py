@@ -100,9 +100,10 @@ def dual_layer_profile(bucket_lengths: Sequence[int], n_heads: int, head_dim: in
         copies = max(1, -(-fill_tokens // L))
         run([L] * copies)                                   # first layer: warm-up, discarded
         f_ms, b_ms = run([L] * copies)                      # second layer: recorded
+        from . import binding
         t_f.append(int(round(f_ms * 1e6)) // copies)
         t_b.append(int(round(b_ms * 1e6)) // copies)
-        m.append(4 * L * n_heads * head_dim * elt_bytes)
+        m.append(binding.dcp_activation_bytes(L, n_heads, head_dim, elt_bytes)[0])
     return ProfileTable(buckets, t_f, t_b, m)
 
 
@@ -121,9 +122,9 @@ def intra_candidates(seq_len: int, batch_sizes: Sequence[int], n_heads: int, hea
     for b in batch_sizes:
         run([seq_len] * b)                                  # first layer: warm-up, discarded
         f_ms, b_ms = run([seq_len] * b)                     # second layer: recorded
-        unit = b * seq_len * n_heads * head_dim * elt_bytes
-        rows.append(binding.dcp_intra_candidate_from_profile(b, 1, int(round(f_ms * 1e6)), int(round(b_ms * 1e6)), 4 * unit,
-                                                             unit, n_layers, const_bytes, fixed_cost_ns))
+        act, inp = binding.dcp_activation_bytes(b * seq_len, n_heads, head_dim, elt_bytes)
+        rows.append(binding.dcp_intra_candidate_from_profile(b, 1, int(round(f_ms * 1e6)), int(round(b_ms * 1e6)), act, inp,
+                                                             n_layers, const_bytes, fixed_cost_ns))
     return rows
 
 

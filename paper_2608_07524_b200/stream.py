@@ -72,11 +72,10 @@ def plan_length_group(n_seqs: int, seq_len: int, batch_size: int, recompute: int
     """The plan of a group of n_seqs sequences of one length run with the setting Algorithm 1 selected
     for that length (Section 3.4): micro-batches of `batch_size` sequences each, every one with
     `recompute` recomputed layers.  Consecutive sequences share a micro-batch."""
-    if n_seqs < 1 or batch_size < 1 or recompute < 0:
-        raise ValueError("need n_seqs >= 1, batch_size >= 1, recompute >= 0")
+    if recompute < 0:
+        raise ValueError("need recompute >= 0")
     lengths = [int(seq_len)] * n_seqs
-    mb_id = [i // batch_size for i in range(n_seqs)]
-    K = mb_id[-1] + 1
+    mb_id, K = binding.dcp_length_group_plan(n_seqs, batch_size)
     mb_seq_offset, seq_index, _, seg_offset, seg = binding.dcp_plan_segments(lengths, mb_id, K, SEG_ROWS)
     lens = np.asarray(lengths, dtype=np.int32)
     plan = BatchPlan(mb_id, [int(recompute)] * K, 0)

@@ -108,6 +108,13 @@ def test_library_interpolation_and_model_time_match_the_oracle():
         args = (int(rng.integers(1, 9)), 1, f[0], b[0], f[1], f[2], lam, f[3], f[4])
         assert B.dcp_intra_candidate_from_profile(*args) == profile_oracle.candidate(*args)
     assert t.model_time([100, 200], 3, 2, 7) == 3 * (4000 + 9000) + 2 * 4000 + 7
+    # memory model of a micro-batch (config 5: 4 * L * H * d * 2 bytes of activations per sequence) and the
+    # grouping of a length group into micro-batches of b sequences
+    assert B.dcp_activation_bytes(1000, 16, 128) == (4 * 1000 * 16 * 128 * 2, 1000 * 16 * 128 * 2)
+    assert B.dcp_activation_bytes(0, 1, 8, 4) == (0, 0)
+    assert B.dcp_length_group_plan(7, 3) == ([0, 0, 0, 1, 1, 1, 2], 3) and B.dcp_length_group_plan(4, 8) == ([0] * 4, 1)
+    with pytest.raises(B.DcpError):
+        B.dcp_length_group_plan(0, 3)
     with pytest.raises(ValueError):
         ProfileTable([100, 100], [1, 2], [1, 2], [1, 2])
     with pytest.raises(B.DcpError) as e:
