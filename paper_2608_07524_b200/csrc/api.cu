@@ -175,6 +175,9 @@ SchedView carve_sched(void* workspace, int32_t n_seqs) {
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// Batches whose longest sequence has at most this many tokens (64 key tiles) run the forward variant for short items.
+constexpr int32_t kShortItemMaxLen = 8192;
+
 // The kernels work on 64 or 128 columns per head; other head dimensions run zero-padded to the next of the two.
 size_t padded_dim(int32_t head_dim) { return head_dim <= 64 ? 64 : 128; }
 
@@ -253,7 +256,7 @@ static int attn_fwd_impl(const char* fn, bool merge, const void* q, const void* 
     p.scale_log2 = p.scale * 1.4426950408889634f;
     {
         ScopedTimer t(DCP_KERNEL_FWD, stream);
-        e = launch_attn_fwd(tq, tk, tv, p, head_dim, causal != 0, dev.sm_count, stream);
+        e = launch_attn_fwd(tq, tk, tv, p, head_dim, causal != 0, max_seqlen <= kShortItemMaxLen, dev.sm_count, stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: attention kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(1);

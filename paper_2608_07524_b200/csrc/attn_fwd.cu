@@ -201,7 +201,8 @@ __device__ __noinline__ void softmax_single_tile_item(FwdShared& sh, const FwdPa
     if (lane == 0) mbar_arrive(&sh.o_free[0]);
 }
 
-template <int D, bool CAUSAL>
+// EARLY_Q: release a Q tile's slot as soon as its last S product has been issued (see the MMA warp).
+template <int D, bool CAUSAL, bool EARLY_Q>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ FwdParams p) {
@@ -334,12 +335,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     tc_fence_after();
                     issue_qk<D>(s_tmem[t], q_desc[t], kv_km0 + (kv_base % kKvStages) * kStageStep, leader);
                     commit(&sh.s_full[t]);
-                    // Under a causal mask (short items: a query block sees a few key tiles) a Q tile is released as
-                    // soon as its last S product is issued, so that the next item's Q load runs while this item's
-                    // last PV products do instead of after them (config 2 forward 1.05 -> 1.01 ms).  Without a mask
-                    // items are long and the two extra tests per key step cost the MMA warp more than the early
-                    // load gains (config 3 forward 16.4 -> 16.9 ms), so there the tiles are released at the end.
-                    if (CAUSAL && nkv_t[t] == 1) commit(&sh.q_empty[t]);
+                    // When items are short (a query block sees a few key tiles: causal masks, batches of short
+                    // sequences) a Q tile is released as soon as its last S product is issued, so that the next
+                    // item's Q load runs while this item's last PV products do instead of after them (config 2
+                    // forward 1.05 -> 1.01 ms, spatial axis of the 2-D workload 1.97 -> 1.84 ms).  On long items the
+                    // two extra tests per key step cost the MMA warp more than the early load gains (config 3
+                    // forward 16.4 -> 16.9 ms), so the host picks the variant by mask and longest sequence.
+                    if (EARLY_Q && nkv_t[t] == 1) commit(&sh.q_empty[t]);
                 }
                 commit(&sh.kv_empty[kv_base % kKvStages]);
 
@@ -355,7 +357,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                             tc_fence_after();
                             issue_qk<D>(s_tmem[0], q_desc[0], kv_km0 + st_k * kStageStep, leader);
                             commit(&sh.s_full[0]);
-                            if (CAUSAL && j + 2 == nkv_t[0]) commit(&sh.q_empty[0]);
+                            if (EARLY_Q && j + 2 == nkv_t[0]) commit(&sh.q_empty[0]);
                         }
                         if (j < nkv_t[t]) {
                             if (j == 0 && use[t] >= 1) mbar_wait(&sh.o_free[t], (use[t] - 1) & 1u, guard);
@@ -373,14 +375,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     if (j + 1 < nkv_t[1]) {
                         issue_qk<D>(s_tmem[1], q_desc[1], kv_km0 + st_k * kStageStep, leader);
                         commit(&sh.s_full[1]);
-                        if (CAUSAL && j + 2 == nkv_t[1]) commit(&sh.q_empty[1]);
+                        if (EARLY_Q && j + 2 == nkv_t[1]) commit(&sh.q_empty[1]);
                     }
                     if (has_next) commit(&sh.kv_empty[st_k]);
                 }
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     if (nkv_t[t] == 0) continue;
-                    if (!CAUSAL) commit(&sh.q_empty[t]);
+                    if (!EARLY_Q) commit(&sh.q_empty[t]);
                     ++use[t];
                 }
                 kv_base += 2 * nkv;
@@ -550,10 +552,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
-template <int D, bool CAUSAL>
+template <int D, bool CAUSAL, bool EARLY_Q>
 static cudaError_t launch_one(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                               int n_ctas, cudaStream_t stream) {
-    auto kern = attn_fwd_kernel<D, CAUSAL>;
+    auto kern = attn_fwd_kernel<D, CAUSAL, EARLY_Q>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<D>::kSmemBytes);
     if (e != cudaSuccess) return e;
     kern<<<n_ctas, kFwdThreads, FwdCfg<D>::kSmemBytes, stream>>>(tq, tk, tv, p);
@@ -561,10 +563,15 @@ static cudaError_t launch_one(const CUtensorMap& tq, const CUtensorMap& tk, cons
 }
 
 cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
-                            int head_dim, bool causal, int n_ctas, cudaStream_t stream) {
-    if (head_dim > 64)
-        return causal ? launch_one<128, true>(tq, tk, tv, p, n_ctas, stream) : launch_one<128, false>(tq, tk, tv, p, n_ctas, stream);
-    return causal ? launch_one<64, true>(tq, tk, tv, p, n_ctas, stream) : launch_one<64, false>(tq, tk, tv, p, n_ctas, stream);
+                            int head_dim, bool causal, bool short_items, int n_ctas, cudaStream_t stream) {
+    if (head_dim > 64) {
+        if (causal) return launch_one<128, true, true>(tq, tk, tv, p, n_ctas, stream);
+        return short_items ? launch_one<128, false, true>(tq, tk, tv, p, n_ctas, stream)
+                           : launch_one<128, false, false>(tq, tk, tv, p, n_ctas, stream);
+    }
+    if (causal) return launch_one<64, true, true>(tq, tk, tv, p, n_ctas, stream);
+    return short_items ? launch_one<64, false, true>(tq, tk, tv, p, n_ctas, stream)
+                       : launch_one<64, false, false>(tq, tk, tv, p, n_ctas, stream);
 }
 
 }  // namespace dcp
