@@ -181,7 +181,10 @@ __device__ __noinline__ void compute_single_tile_item(BwdControl& sh, const BwdP
     if (lane == 0) mbar_arrive(&sh.ds_full);
 }
 
-template <int D, bool CAUSAL>
+// TRIM: head_dim is at most D - 16, so the products skip the zero-padded columns: S^T and dP^T sum over
+// ceil(head_dim / 16) steps instead of D / 16; dV, dK and dQ are 16 * ceil(head_dim / 16) columns wide, and so
+// is what the drain warps add to the accumulator.
+template <int D, bool CAUSAL, bool TRIM>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_do,
@@ -329,8 +332,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             // Shared-memory descriptors are built once; a k-step only adds a constant to the address
             // field (the issuing thread is on the critical path: MMA issue blocks while the pipe is busy).
             constexpr uint32_t idesc_abt = make_idesc_bf16(128, 128, false, false);  // both operands K-contiguous
-            constexpr uint32_t idesc_nd_kb = make_idesc_bf16(128, D, false, true);   // A K-contig / tmem, B N-contig
-            constexpr uint32_t idesc_nd_mm = make_idesc_bf16(128, D, true, true);    // A M-contig, B N-contig
+            const int n_ks = TRIM ? (p.head_dim + 15) >> 4 : D / 16;                // steps of 16 head_dim columns that hold data
+            const uint32_t idesc_nd_kb = make_idesc_bf16(128, TRIM ? n_ks * 16 : D, false, true);   // A K-contig / tmem, B N-contig
+            const uint32_t idesc_nd_mm = make_idesc_bf16(128, TRIM ? n_ks * 16 : D, true, true);    // A M-contig, B N-contig
             constexpr uint32_t kStageStep = Cfg::kTileBytes >> 4;
             const uint64_t k_km = make_sdesc_sw128(smem_u32(smem + Cfg::kOffK), 16, 1024);
             const uint64_t k_mn = make_sdesc_sw128(smem_u32(smem + Cfg::kOffK), Cfg::kBoxBytes, 1024);
@@ -352,7 +356,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             auto issue_abt = [&](uint32_t d_tmem, uint64_t a, uint64_t b) {
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks)
-                    if (leader) tc_mma_ss(d_tmem, a + km_step(ks, Cfg::kBoxBytes), b + km_step(ks, Cfg::kBoxBytes), idesc_abt, ks > 0);
+                    if (leader && (!TRIM || ks < n_ks))
+                        tc_mma_ss(d_tmem, a + km_step(ks, Cfg::kBoxBytes), b + km_step(ks, Cfg::kBoxBytes), idesc_abt, ks > 0);
             };
             uint32_t n_work = 0, g = 0;
             while (true) {
@@ -622,8 +627,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 } else {
                     const bool live = qrow < w.len;
                     if ((warp & 3) > 0) __nanosleep((warp & 3) * kRedStaggerNs + 64);
+                    const int n_c4 = TRIM ? ((p.head_dim + 15) >> 4) * 4 : D / 4;     // groups of four columns that hold data
 #pragma unroll
                     for (int c = 0; c < D / 4; ++c) {
+                        if (TRIM && c >= n_c4) break;
                         if (live) red_add_v4(dst + c * (kTile * 4), __uint_as_float(acc[c * 4]), __uint_as_float(acc[c * 4 + 1]),
                                    __uint_as_float(acc[c * 4 + 2]), __uint_as_float(acc[c * 4 + 3]));
                         if ((c % kRedGroup) == kRedGroup - 1) __nanosleep(kRedSleepNs);
@@ -639,10 +646,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
-template <int D, bool CAUSAL>
+template <int D, bool CAUSAL, bool TRIM>
 static cudaError_t launch_one(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
                               const BwdParams& p, int n_ctas, cudaStream_t stream) {
-    auto kern = attn_bwd_kernel<D, CAUSAL>;
+    auto kern = attn_bwd_kernel<D, CAUSAL, TRIM>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<D>::kSmemBytes);
     if (e != cudaSuccess) return e;
     kern<<<n_ctas, kBwdThreads, BwdCfg<D>::kSmemBytes, stream>>>(tq, tk, tv, tdo, p);
@@ -651,11 +658,14 @@ static cudaError_t launch_one(const CUtensorMap& tq, const CUtensorMap& tk, cons
 
 cudaError_t launch_attn_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
                             const BwdParams& p, int head_dim, bool causal, int n_ctas, cudaStream_t stream) {
+    if (head_dim > 112)
+        return causal ? launch_one<128, true, false>(tq, tk, tv, tdo, p, n_ctas, stream)
+                      : launch_one<128, false, false>(tq, tk, tv, tdo, p, n_ctas, stream);
     if (head_dim > 64)
-        return causal ? launch_one<128, true>(tq, tk, tv, tdo, p, n_ctas, stream)
-                      : launch_one<128, false>(tq, tk, tv, tdo, p, n_ctas, stream);
-    return causal ? launch_one<64, true>(tq, tk, tv, tdo, p, n_ctas, stream)
-                  : launch_one<64, false>(tq, tk, tv, tdo, p, n_ctas, stream);
+        return causal ? launch_one<128, true, true>(tq, tk, tv, tdo, p, n_ctas, stream)
+                      : launch_one<128, false, true>(tq, tk, tv, tdo, p, n_ctas, stream);
+    return causal ? launch_one<64, true, false>(tq, tk, tv, tdo, p, n_ctas, stream)
+                  : launch_one<64, false, false>(tq, tk, tv, tdo, p, n_ctas, stream);
 }
 
 }  // namespace dcp

@@ -79,24 +79,27 @@ __device__ __forceinline__ void load_tile(uint8_t* dst, const CUtensorMap* map, 
 // dependent instructions several cycles apart, so each instruction between two MMAs is pipe idle time.)
 
 // S = Q K^T for one 128x128 tile: both operands K-contiguous in shared memory.
-template <int D>
-__device__ __forceinline__ void issue_qk(uint32_t d_tmem, uint64_t q_desc, uint64_t k_desc, bool leader) {
+// TRIM: the head dimension is smaller than the D columns the tiles hold (the rest are zeros), so only the
+// first n_ks steps of 16 columns are multiplied; without it the loop is the full, compile-time one.
+template <int D, bool TRIM>
+__device__ __forceinline__ void issue_qk(uint32_t d_tmem, uint64_t q_desc, uint64_t k_desc, bool leader, int n_ks) {
     constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, false);
 #pragma unroll
     for (int ks = 0; ks < D / 16; ++ks) {
         constexpr int kBox = FwdCfg<D>::kBoxBytes;
         const uint64_t off = (uint64_t)(((ks / 4) * kBox + (ks % 4) * 32) >> 4);
-        if (leader) tc_mma_ss(d_tmem, q_desc + off, k_desc + off, idesc, ks > 0);
+        if (leader && (!TRIM || ks < n_ks)) tc_mma_ss(d_tmem, q_desc + off, k_desc + off, idesc, ks > 0);
     }
 }
 
 // O (+)= P V: P from tensor memory (bf16 pairs per column), V with head_dim contiguous.
 // `part` selects 32 of the tile's 128 keys: the product starts on the first part of P while the softmax
 // group is still producing the rest, which shortens the chain S -> softmax -> PV -> next S.
-template <int D>
+// TRIM: only the first 16 * n_ks columns of O are computed (idesc_trim carries that width).
+template <int D, bool TRIM>
 __device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint64_t v_desc, bool accumulate, bool leader,
-                                         int part) {
-    constexpr uint32_t idesc = make_idesc_bf16(128, D, false, true);
+                                         int part, uint32_t idesc_trim) {
+    const uint32_t idesc = TRIM ? idesc_trim : make_idesc_bf16(128, D, false, true);
 #pragma unroll
     for (int k4 = 0; k4 < 2; ++k4) {
         const int ks = part * 2 + k4;
@@ -202,7 +205,10 @@ __device__ __noinline__ void softmax_single_tile_item(FwdShared& sh, const FwdPa
 }
 
 // EARLY_Q: release a Q tile's slot as soon as its last S product has been issued (see the MMA warp).
-template <int D, bool CAUSAL, bool EARLY_Q>
+// TRIM: head_dim is at most D - 16, so the products skip the zero-padded columns: S sums over
+// ceil(head_dim / 16) steps instead of D / 16 and O is 16 * ceil(head_dim / 16) columns wide (head_dim 72,
+// the width of the paper's second model, does 5/8 of the padded work).
+template <int D, bool CAUSAL, bool EARLY_Q, bool TRIM>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ FwdParams p) {
@@ -309,6 +315,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             constexpr uint32_t kStageStep = Cfg::kTileBytes >> 4;
             const uint32_t s_tmem[2] = {tmem + Cfg::kS0, tmem + Cfg::kS1};
             const uint32_t o_tmem[2] = {tmem + Cfg::kO0, tmem + Cfg::kO1};
+            const int n_ks = TRIM ? (p.head_dim + 15) >> 4 : D / 16;
+            const uint32_t idesc_pv = make_idesc_bf16(128, n_ks * 16, false, true);
             auto kv_wait = [&](uint32_t idx) {
                 mbar_wait(&sh.kv_full[idx % kKvStages], (idx / kKvStages) & 1u, guard);
             };
@@ -333,7 +341,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     if (nkv_t[t] == 0) continue;
                     mbar_wait(&sh.q_full[t], use[t] & 1u, guard);
                     tc_fence_after();
-                    issue_qk<D>(s_tmem[t], q_desc[t], kv_km0 + (kv_base % kKvStages) * kStageStep, leader);
+                    issue_qk<D, TRIM>(s_tmem[t], q_desc[t], kv_km0 + (kv_base % kKvStages) * kStageStep, leader, n_ks);
                     commit(&sh.s_full[t]);
                     // When items are short (a query block sees a few key tiles: causal masks, batches of short
                     // sequences) a Q tile is released as soon as its last S product is issued, so that the next
@@ -355,7 +363,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         if (t == 1 && has_next) kv_wait(ik);
                         if (t == 1 && j + 1 < nkv_t[0]) {      // S_0(j+1) goes between the two PV products
                             tc_fence_after();
-                            issue_qk<D>(s_tmem[0], q_desc[0], kv_km0 + st_k * kStageStep, leader);
+                            issue_qk<D, TRIM>(s_tmem[0], q_desc[0], kv_km0 + st_k * kStageStep, leader, n_ks);
                             commit(&sh.s_full[0]);
                             if (EARLY_Q && j + 2 == nkv_t[0]) commit(&sh.q_empty[0]);
                         }
@@ -365,7 +373,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                             for (int part = 0; part < 4; ++part) {
                                 mbar_wait(&sh.p_part[t][part], n_p[t] & 1u, guard);
                                 tc_fence_after();
-                                issue_pv<D>(o_tmem[t], s_tmem[t], kv_mn0 + st_v * kStageStep, j > 0, leader, part);
+                                issue_pv<D, TRIM>(o_tmem[t], s_tmem[t], kv_mn0 + st_v * kStageStep, j > 0, leader, part, idesc_pv);
                             }
                             ++n_p[t];
                             if (j == nkv_t[t] - 1) commit(&sh.o_full[t]);
@@ -373,7 +381,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     }
                     commit(&sh.kv_empty[st_v]);
                     if (j + 1 < nkv_t[1]) {
-                        issue_qk<D>(s_tmem[1], q_desc[1], kv_km0 + st_k * kStageStep, leader);
+                        issue_qk<D, TRIM>(s_tmem[1], q_desc[1], kv_km0 + st_k * kStageStep, leader, n_ks);
                         commit(&sh.s_full[1]);
                         if (EARLY_Q && j + 2 == nkv_t[1]) commit(&sh.q_empty[1]);
                     }
@@ -552,26 +560,29 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
-template <int D, bool CAUSAL, bool EARLY_Q>
+template <int D, bool CAUSAL, bool EARLY_Q, bool TRIM>
 static cudaError_t launch_one(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                               int n_ctas, cudaStream_t stream) {
-    auto kern = attn_fwd_kernel<D, CAUSAL, EARLY_Q>;
+    auto kern = attn_fwd_kernel<D, CAUSAL, EARLY_Q, TRIM>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<D>::kSmemBytes);
     if (e != cudaSuccess) return e;
     kern<<<n_ctas, kFwdThreads, FwdCfg<D>::kSmemBytes, stream>>>(tq, tk, tv, p);
     return cudaGetLastError();
 }
 
+template <int D, bool TRIM>
+static cudaError_t launch_masked(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
+                                 bool causal, bool short_items, int n_ctas, cudaStream_t stream) {
+    if (causal) return launch_one<D, true, true, TRIM>(tq, tk, tv, p, n_ctas, stream);
+    return short_items ? launch_one<D, false, true, TRIM>(tq, tk, tv, p, n_ctas, stream)
+                       : launch_one<D, false, false, TRIM>(tq, tk, tv, p, n_ctas, stream);
+}
+
 cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                             int head_dim, bool causal, bool short_items, int n_ctas, cudaStream_t stream) {
-    if (head_dim > 64) {
-        if (causal) return launch_one<128, true, true>(tq, tk, tv, p, n_ctas, stream);
-        return short_items ? launch_one<128, false, true>(tq, tk, tv, p, n_ctas, stream)
-                           : launch_one<128, false, false>(tq, tk, tv, p, n_ctas, stream);
-    }
-    if (causal) return launch_one<64, true, true>(tq, tk, tv, p, n_ctas, stream);
-    return short_items ? launch_one<64, false, true>(tq, tk, tv, p, n_ctas, stream)
-                       : launch_one<64, false, false>(tq, tk, tv, p, n_ctas, stream);
+    if (head_dim > 112) return launch_masked<128, false>(tq, tk, tv, p, causal, short_items, n_ctas, stream);
+    if (head_dim > 64) return launch_masked<128, true>(tq, tk, tv, p, causal, short_items, n_ctas, stream);
+    return launch_masked<64, false>(tq, tk, tv, p, causal, short_items, n_ctas, stream);
 }
 
 }  // namespace dcp

@@ -301,7 +301,7 @@ def test_many_sequences_mixed_with_long_ones(causal):
 
 
 @pytest.mark.parametrize("causal", [False, True])
-@pytest.mark.parametrize("d", [8, 40, 72, 96, 120])
+@pytest.mark.parametrize("d", [8, 40, 72, 80, 96, 104, 112, 120])
 def test_head_dims_between_the_native_ones(causal, d):
     # head dimensions other than 64 and 128 run zero-padded to the next of the two (72 is the head
     # dimension of the paper's second model: hidden size 1152 over 16 heads)
