@@ -241,6 +241,27 @@ int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, const void*
                         float softmax_scale, void* dq, void* dk, void* dv, void* workspace,
                         size_t workspace_bytes, void* cuda_stream);
 
+/* The same two calls on a group of heads inside wider tensors: consecutive tokens of q, k, v, o, d_o, dq,
+ * dk, dv are token_stride elements apart (a multiple of 8, at least n_heads * head_dim; the plain calls are
+ * the case token_stride = n_heads * head_dim); each pointer addresses the group's first head of token 0; lse
+ * stays [n_heads, total_tokens] for the group.
+ *
+ * Paper: Section 3.2 (sequence-parallel size p_i) and Section 4.1 (the head-sharded scheme: every rank of
+ * a group holds a slice of the tokens with all heads, attention needs all tokens of some heads).  With these
+ * calls rank r of p computes heads [r H/p, (r+1) H/p) directly on the token-sharded [T, H, d] tensors - its
+ * own slice and its peers', mapped into one address range (peer or fabric mappings; the kernels read them
+ * with plain TMA loads, no multicast, and write results with plain stores) - so the re-sharding all-to-all
+ * on either side of attention is never materialised: a tile crosses the link when the kernel needs it. */
+int dcp_varlen_attn_fwd_strided(const void* q, const void* k, const void* v, const int32_t* cu_seqlens, int32_t n_seqs,
+                                int32_t total_tokens, int32_t max_seqlen, int32_t n_heads, int32_t head_dim,
+                                int64_t token_stride, int32_t causal, float softmax_scale, void* o, float* lse,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream);
+int dcp_varlen_attn_bwd_strided(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                                const float* lse, const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens,
+                                int32_t max_seqlen, int32_t n_heads, int32_t head_dim, int64_t token_stride,
+                                int32_t causal, float softmax_scale, void* dq, void* dk, void* dv, void* workspace,
+                                size_t workspace_bytes, void* cuda_stream);
+
 /* Forward attention without a workspace argument (the paper has no counterpart; this exists for
  * callers that must not allocate device memory - code running inside a memory-pool callback or a
  * real-time loop, a plug-in handed fixed buffers by its host program, a process whose allocator is

@@ -68,6 +68,12 @@ def lib():
             L.dcp_varlen_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32,
                                               vp, vp, vp, vp, ctypes.c_size_t, vp]
             L.dcp_varlen_attn_bwd.restype = ctypes.c_int
+            L.dcp_varlen_attn_fwd_strided.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i64, i32, f32, vp, vp, vp,
+                                                      ctypes.c_size_t, vp]
+            L.dcp_varlen_attn_fwd_strided.restype = ctypes.c_int
+            L.dcp_varlen_attn_bwd_strided.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i64, i32, f32,
+                                                      vp, vp, vp, vp, ctypes.c_size_t, vp]
+            L.dcp_varlen_attn_bwd_strided.restype = ctypes.c_int
             L.dcp_varlen_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, vp, vp, vp]
             L.dcp_varlen_attn_fwd_noalloc.restype = ctypes.c_int
             L.dcp_query_status.argtypes = [vp, vp]
@@ -236,6 +242,57 @@ def dcp_varlen_attn_fwd(q, k, v, cu_seqlens, max_seqlen: int, causal: bool, soft
                                      int(bool(causal)), float(softmax_scale), _ptr(o), _ptr(lse), _ptr(ws),
                                      ws.numel(), _stream(stream)))
     return o, lse
+
+
+def _require_head_group(t, name, stride=None):
+    """A bf16 CUDA view [T, Hg, d] of a group of heads inside a wider [T, H, d] tensor: unit stride along
+    d, heads d apart, tokens `stride` apart.  Returns the token stride."""
+    import torch
+    if not t.is_cuda or t.dtype != torch.bfloat16 or t.dim() != 3:
+        raise TypeError(f"{name} must be a bf16 CUDA tensor [T, heads, head_dim]")
+    T, Hg, d = t.shape
+    st = t.stride()
+    if st[2] != 1 or (Hg > 1 and st[1] != d) or (T > 1 and st[0] < Hg * d) or (stride is not None and T > 1 and st[0] != stride):
+        raise TypeError(f"{name} must be a group of adjacent heads of a [T, H, d] tensor (same token stride for all tensors)")
+    return int(st[0]) if T > 1 else (stride if stride is not None else Hg * d)
+
+
+def dcp_varlen_attn_fwd_strided(q, k, v, cu_seqlens, max_seqlen: int, causal: bool, out, softmax_scale: float = 0.0,
+                                lse=None, workspace=None, stream=None):
+    """Forward attention on a group of heads inside wider tensors (views such as x[:, h0:h1, :]); `out` is a
+    view of the same kind.  lse [Hg, T] fp32 is contiguous and belongs to the group.  Enqueues only."""
+    import torch
+    stride = _require_head_group(q, "q")
+    for name, t in (("k", k), ("v", v), ("out", out)):
+        _require_head_group(t, name, stride)
+    _require(cu_seqlens, torch.int32, "cu_seqlens")
+    T, Hg, d = q.shape
+    n_seqs = cu_seqlens.numel() - 1
+    lse = torch.empty((Hg, T), dtype=torch.float32, device=q.device) if lse is None else lse
+    ws = alloc_workspace(T, n_seqs, Hg, d, False, q.device) if workspace is None else workspace
+    _check(lib().dcp_varlen_attn_fwd_strided(_ptr(q), _ptr(k), _ptr(v), _ptr(cu_seqlens), n_seqs, T, int(max_seqlen), Hg,
+                                             d, stride, int(bool(causal)), float(softmax_scale), _ptr(out), _ptr(lse),
+                                             _ptr(ws), ws.numel(), _stream(stream)))
+    return out, lse
+
+
+def dcp_varlen_attn_bwd_strided(q, k, v, o, d_o, lse, cu_seqlens, max_seqlen: int, causal: bool, dq, dk, dv,
+                                softmax_scale: float = 0.0, workspace=None, stream=None):
+    """Backward attention on a group of heads inside wider tensors; dq, dk, dv are views of the same kind."""
+    import torch
+    stride = _require_head_group(q, "q")
+    for name, t in (("k", k), ("v", v), ("o", o), ("d_o", d_o), ("dq", dq), ("dk", dk), ("dv", dv)):
+        _require_head_group(t, name, stride)
+    _require(lse, torch.float32, "lse")
+    _require(cu_seqlens, torch.int32, "cu_seqlens")
+    T, Hg, d = q.shape
+    n_seqs = cu_seqlens.numel() - 1
+    ws = alloc_workspace(T, n_seqs, Hg, d, True, q.device) if workspace is None else workspace
+    _check(lib().dcp_varlen_attn_bwd_strided(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), _ptr(cu_seqlens),
+                                             n_seqs, T, int(max_seqlen), Hg, d, stride, int(bool(causal)),
+                                             float(softmax_scale), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(ws), ws.numel(),
+                                             _stream(stream)))
+    return dq, dk, dv
 
 
 NOALLOC_MAX_SEQS = 4096

@@ -126,12 +126,14 @@ int device_info(DeviceInfo* out) {
 
 // [T, H, d] bf16 viewed as a 3-D tensor (d, H, T); a box is 64 columns x 1 head x 128 tokens,
 // written to shared memory as 128 rows of 128 bytes with the 128-byte swizzle.  Rows past T are
-// zero-filled.
-int make_map(CUtensorMap* map, const void* base, int32_t total_tokens, int32_t n_heads, int32_t head_dim) {
+// zero-filled.  Consecutive tokens are row_stride elements apart (n_heads * head_dim when the tensor is
+// contiguous; more when it is a group of heads inside a wider tensor).
+int make_map(CUtensorMap* map, const void* base, int32_t total_tokens, int32_t n_heads, int32_t head_dim,
+             int64_t row_stride) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return fail(DCP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the CUDA driver");
     const cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)n_heads, (cuuint64_t)total_tokens};
-    const cuuint64_t strides[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)n_heads * head_dim * 2};
+    const cuuint64_t strides[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)row_stride * 2};
     const cuuint32_t box[3] = {64, 1, (cuuint32_t)kTile};
     const cuuint32_t elem_strides[3] = {1, 1, 1};
     const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
@@ -156,6 +158,13 @@ int check_shape(const char* fn, int32_t n_seqs, int32_t total_tokens, int32_t ma
         return fail(DCP_ERR_INVALID_ARG, "%s: softmax_scale must be finite and >= 0 (0 selects 1/sqrt(d))", fn);
     if ((int64_t)total_tokens * n_heads >= ((int64_t)1 << 31))
         return fail(DCP_ERR_UNSUPPORTED, "%s: total_tokens * n_heads must be below 2^31", fn);
+    return DCP_OK;
+}
+
+int check_stride(const char* fn, int64_t token_stride, int32_t n_heads, int32_t head_dim) {
+    if (token_stride < (int64_t)n_heads * head_dim || token_stride % 8 != 0)
+        return fail(DCP_ERR_INVALID_ARG, "%s: token_stride must be a multiple of 8 elements and at least n_heads * head_dim", fn);
+    if (token_stride >= ((int64_t)1 << 38)) return fail(DCP_ERR_UNSUPPORTED, "%s: token_stride too large", fn);
     return DCP_OK;
 }
 
@@ -207,9 +216,10 @@ extern "C" int dcp_varlen_attn_workspace(int32_t total_tokens, int32_t n_seqs, i
 // the results are the same either way.
 static int attn_fwd_impl(const char* fn, bool merge, const void* q, const void* k, const void* v,
                          const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen,
-                         int32_t n_heads, int32_t head_dim, int32_t causal, float softmax_scale, void* o, float* lse,
-                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+                         int32_t n_heads, int32_t head_dim, int64_t token_stride, int32_t causal, float softmax_scale,
+                         void* o, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     if (int rc = check_shape(fn, n_seqs, total_tokens, max_seqlen, n_heads, head_dim, softmax_scale)) return rc;
+    if (int rc = check_stride(fn, token_stride, n_heads, head_dim)) return rc;
     if (!cu_seqlens) return fail(DCP_ERR_INVALID_ARG, "%s: cu_seqlens is null", fn);
     if (!workspace) return fail(DCP_ERR_WORKSPACE, "%s: workspace is null", fn);
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
@@ -239,9 +249,9 @@ static int attn_fwd_impl(const char* fn, bool merge, const void* q, const void* 
     if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
 
     CUtensorMap tq, tk, tv;
-    if (int rc = make_map(&tq, q, total_tokens, n_heads, head_dim)) return rc;
-    if (int rc = make_map(&tk, k, total_tokens, n_heads, head_dim)) return rc;
-    if (int rc = make_map(&tv, v, total_tokens, n_heads, head_dim)) return rc;
+    if (int rc = make_map(&tq, q, total_tokens, n_heads, head_dim, token_stride)) return rc;
+    if (int rc = make_map(&tk, k, total_tokens, n_heads, head_dim, token_stride)) return rc;
+    if (int rc = make_map(&tv, v, total_tokens, n_heads, head_dim, token_stride)) return rc;
 
     FwdParams p;
     p.cu_seqlens = merge ? sched.vcu : cu_seqlens;
@@ -252,6 +262,7 @@ static int attn_fwd_impl(const char* fn, bool merge, const void* q, const void* 
     p.n_heads = n_heads;
     p.head_dim = head_dim;
     p.total_tokens = total_tokens;
+    p.row_stride = token_stride;
     p.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
     p.scale_log2 = p.scale * 1.4426950408889634f;
     {
@@ -268,16 +279,27 @@ extern "C" int dcp_varlen_attn_fwd(const void* q, const void* k, const void* v, 
                                    int32_t head_dim, int32_t causal, float softmax_scale, void* o, float* lse,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
     return attn_fwd_impl("dcp_varlen_attn_fwd", true, q, k, v, cu_seqlens, n_seqs, total_tokens, max_seqlen, n_heads,
-                         head_dim, causal, softmax_scale, o, lse, workspace, workspace_bytes, cuda_stream);
+                         head_dim, (int64_t)n_heads * head_dim, causal, softmax_scale, o, lse, workspace, workspace_bytes,
+                         cuda_stream);
 }
 
-extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
-                                   const float* lse, const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens,
-                                   int32_t max_seqlen, int32_t n_heads, int32_t head_dim, int32_t causal,
-                                   float softmax_scale, void* dq, void* dk, void* dv, void* workspace,
-                                   size_t workspace_bytes, void* cuda_stream) {
-    const char* fn = "dcp_varlen_attn_bwd";
+extern "C" int dcp_varlen_attn_fwd_strided(const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
+                                           int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen, int32_t n_heads,
+                                           int32_t head_dim, int64_t token_stride, int32_t causal, float softmax_scale,
+                                           void* o, float* lse, void* workspace, size_t workspace_bytes,
+                                           void* cuda_stream) {
+    return attn_fwd_impl("dcp_varlen_attn_fwd_strided", true, q, k, v, cu_seqlens, n_seqs, total_tokens, max_seqlen,
+                         n_heads, head_dim, token_stride, causal, softmax_scale, o, lse, workspace, workspace_bytes,
+                         cuda_stream);
+}
+
+static int attn_bwd_impl(const char* fn, const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                         const float* lse, const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens,
+                         int32_t max_seqlen, int32_t n_heads, int32_t head_dim, int64_t token_stride, int32_t causal,
+                         float softmax_scale, void* dq, void* dk, void* dv, void* workspace, size_t workspace_bytes,
+                         void* cuda_stream) {
     if (int rc = check_shape(fn, n_seqs, total_tokens, max_seqlen, n_heads, head_dim, softmax_scale)) return rc;
+    if (int rc = check_stride(fn, token_stride, n_heads, head_dim)) return rc;
     if (!cu_seqlens) return fail(DCP_ERR_INVALID_ARG, "%s: cu_seqlens is null", fn);
     if (!workspace) return fail(DCP_ERR_WORKSPACE, "%s: workspace is null", fn);
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
@@ -314,16 +336,16 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
     if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
 
     CUtensorMap tq, tk, tv, tg;
-    if (int rc = make_map(&tq, q, total_tokens, n_heads, head_dim)) return rc;
-    if (int rc = make_map(&tk, k, total_tokens, n_heads, head_dim)) return rc;
-    if (int rc = make_map(&tv, v, total_tokens, n_heads, head_dim)) return rc;
-    if (int rc = make_map(&tg, d_o, total_tokens, n_heads, head_dim)) return rc;
+    if (int rc = make_map(&tq, q, total_tokens, n_heads, head_dim, token_stride)) return rc;
+    if (int rc = make_map(&tk, k, total_tokens, n_heads, head_dim, token_stride)) return rc;
+    if (int rc = make_map(&tv, v, total_tokens, n_heads, head_dim, token_stride)) return rc;
+    if (int rc = make_map(&tg, d_o, total_tokens, n_heads, head_dim, token_stride)) return rc;
 
     {
         ScopedTimer t(DCP_KERNEL_BWD_PRE, stream);
         e = launch_bwd_pre(static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, vcu,
                            sched, stats, dq_acc, max_tiles(total_tokens, n_seqs) * kTile * n_heads * padded_dim(head_dim),
-                           total_tokens, n_heads, head_dim,
+                           total_tokens, n_heads, head_dim, token_stride,
                            softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim), dev.sm_count, stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: pre kernel: %s", fn, cudaGetErrorString(e));
@@ -341,6 +363,7 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
     p.n_heads = n_heads;
     p.head_dim = head_dim;
     p.total_tokens = total_tokens;
+    p.row_stride = token_stride;
     p.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
     p.scale_log2 = p.scale * 1.4426950408889634f;
     {
@@ -352,12 +375,32 @@ extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, 
 
     {
         ScopedTimer t(DCP_KERNEL_BWD_POST, stream);
-        e = launch_bwd_post(dq_acc, static_cast<__nv_bfloat16*>(dq), vcu, sched, n_heads, head_dim, p.scale,
+        e = launch_bwd_post(dq_acc, static_cast<__nv_bfloat16*>(dq), vcu, sched, n_heads, head_dim, token_stride, p.scale,
                             dev.sm_count, stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: post kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(1);
     return DCP_OK;
+}
+
+extern "C" int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                                   const float* lse, const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens,
+                                   int32_t max_seqlen, int32_t n_heads, int32_t head_dim, int32_t causal,
+                                   float softmax_scale, void* dq, void* dk, void* dv, void* workspace,
+                                   size_t workspace_bytes, void* cuda_stream) {
+    return attn_bwd_impl("dcp_varlen_attn_bwd", q, k, v, o, d_o, lse, cu_seqlens, n_seqs, total_tokens, max_seqlen, n_heads,
+                         head_dim, (int64_t)n_heads * head_dim, causal, softmax_scale, dq, dk, dv, workspace, workspace_bytes,
+                         cuda_stream);
+}
+
+extern "C" int dcp_varlen_attn_bwd_strided(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                                           const float* lse, const int32_t* cu_seqlens, int32_t n_seqs,
+                                           int32_t total_tokens, int32_t max_seqlen, int32_t n_heads, int32_t head_dim,
+                                           int64_t token_stride, int32_t causal, float softmax_scale, void* dq, void* dk,
+                                           void* dv, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return attn_bwd_impl("dcp_varlen_attn_bwd_strided", q, k, v, o, d_o, lse, cu_seqlens, n_seqs, total_tokens, max_seqlen,
+                         n_heads, head_dim, token_stride, causal, softmax_scale, dq, dk, dv, workspace, workspace_bytes,
+                         cuda_stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -425,8 +468,9 @@ extern "C" int dcp_varlen_attn_fwd_noalloc(const void* q, const void* k, const v
     if (sched_bytes(n_seqs) > kNoAllocScratchBytes)      // cannot happen for n_seqs <= the maximum; kept as a guard
         return fail(DCP_ERR_UNSUPPORTED, "%s: built-in scratch too small", fn);
     // short sequences are not merged here: the table that needs is sized by the token count
-    return attn_fwd_impl(fn, false, q, k, v, cu_seqlens, n_seqs, total_tokens, max_seqlen, n_heads, head_dim, causal,
-                         softmax_scale, o, lse, scratch, kNoAllocScratchBytes, cuda_stream);
+    return attn_fwd_impl(fn, false, q, k, v, cu_seqlens, n_seqs, total_tokens, max_seqlen, n_heads, head_dim,
+                         (int64_t)n_heads * head_dim, causal, softmax_scale, o, lse, scratch, kNoAllocScratchBytes,
+                         cuda_stream);
 }
 
 extern "C" int dcp_noalloc_status(void* cuda_stream) {

@@ -548,7 +548,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             mbar_wait(&sh.dkv_full, n_work & 1u, guard);
             tc_fence_after();
             const size_t tok = (size_t)w.tok0 + (size_t)key;
-            const size_t out_off = (tok * p.n_heads + w.head) * p.head_dim + half * (D / 2);
+            const size_t out_off = tok * p.row_stride + w.head * p.head_dim + half * (D / 2);
 #pragma unroll
             for (int which = 0; which < 2; ++which) {
                 const uint32_t src = tmem + lane_base + (which == 0 ? Cfg::kDv : Cfg::kDk) + half * (D / 2);
@@ -613,7 +613,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 if (w.len <= kTile) {
                     // the sequence's only tile pair: this is the whole dQ, no accumulation needed
                     if (qrow < w.len) {
-                        __nv_bfloat16* out = p.dq + (((size_t)w.tok0 + qrow) * p.n_heads + w.head) * p.head_dim;
+                        __nv_bfloat16* out = p.dq + ((size_t)w.tok0 + qrow) * p.row_stride + w.head * p.head_dim;
 #pragma unroll
                         for (int c = 0; c < D / 8; ++c) {
                             uint4 val;

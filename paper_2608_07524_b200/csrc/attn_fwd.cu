@@ -180,7 +180,7 @@ __device__ __noinline__ void softmax_single_tile_item(FwdShared& sh, const FwdPa
     tc_fence_after();
     const float inv_l = 1.0f / l;
     const size_t tok = (size_t)w.tok0 + (size_t)row;
-    __nv_bfloat16* out = p.o + (tok * p.n_heads + w.head) * p.head_dim;
+    __nv_bfloat16* out = p.o + tok * p.row_stride + w.head * p.head_dim;
 #pragma unroll
     for (int c = 0; c < D / 32; ++c) {
         uint32_t acc[32];
@@ -529,7 +529,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             const float inv_l = 1.0f / l;
             const bool valid = row < w.len;
             const size_t tok = (size_t)w.tok0 + (size_t)row;
-            __nv_bfloat16* out = p.o + (tok * p.n_heads + w.head) * p.head_dim;
+            __nv_bfloat16* out = p.o + tok * p.row_stride + w.head * p.head_dim;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t acc[32];

@@ -18,6 +18,7 @@ struct FwdParams {
     int32_t head_dim;     // columns of a row in global memory (a multiple of 8); the kernels work on 64 or 128
                           // columns, those past head_dim read as zeros (TMA fills them) and are never stored
     int32_t total_tokens;
+    int64_t row_stride; // elements between consecutive tokens of q, k, v, o (n_heads * head_dim when contiguous)
     float scale;        // softmax scale
     float scale_log2;   // scale * log2(e)
 };
@@ -36,6 +37,7 @@ struct BwdParams {
     int32_t n_heads;
     int32_t head_dim;     // as in FwdParams
     int32_t total_tokens;
+    int64_t row_stride;   // as in FwdParams; the same for q, k, v, dO, dq, dk, dv
     float scale;
     float scale_log2;
 };
@@ -70,14 +72,15 @@ cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const 
 // Tile-aligned row statistics for the backward kernel (see BwdParams::stats) and dq_acc = 0.
 cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, const float* lse, const int32_t* cu_seqlens,
                            const SchedView& sched, __nv_bfloat16* stats, float* dq_acc, size_t dq_acc_elems,
-                           int32_t total_tokens, int32_t n_heads, int32_t head_dim, float scale, int n_sms,
-                           cudaStream_t stream);
+                           int32_t total_tokens, int32_t n_heads, int32_t head_dim, int64_t row_stride, float scale,
+                           int n_sms, cudaStream_t stream);
 
 cudaError_t launch_attn_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
                             const BwdParams& p, int head_dim, bool causal, int n_ctas, cudaStream_t stream);
 
 // dq[T, H, d] = bf16(scale * dq_acc), undoing the tile-blocked layout
 cudaError_t launch_bwd_post(const float* dq_acc, __nv_bfloat16* dq, const int32_t* cu_seqlens, const SchedView& sched,
-                            int32_t n_heads, int32_t head_dim, float scale, int n_sms, cudaStream_t stream);
+                            int32_t n_heads, int32_t head_dim, int64_t row_stride, float scale, int n_sms,
+                            cudaStream_t stream);
 
 }  // namespace dcp

@@ -330,7 +330,7 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
                                                       int32_t n_seqs, __nv_bfloat16* __restrict__ stats,
                                                       float* __restrict__ dq_acc, size_t dq_acc_vec4,
                                                       int32_t total_tokens, int32_t n_heads, int32_t head_dim,
-                                                      float inv_scale) {
+                                                      int64_t row_stride, float inv_scale) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t n_blocks = tile_prefix[n_seqs] * (uint32_t)n_heads;
     for (uint32_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
@@ -375,7 +375,7 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
                     const size_t tok = (size_t)cu[lo] + row0 + r;
                     // rows hold head_dim <= D columns; lanes past them re-read column 0 and drop it, so that the
                     // loads stay unconditional and eight of them are in flight per lane
-                    const size_t row = (tok * n_heads + h) * (size_t)head_dim + lane_col;
+                    const size_t row = tok * (size_t)row_stride + (size_t)h * head_dim + lane_col;
                     if (kPer == 4) {
                         a[u] = *reinterpret_cast<const uint2*>(o + row);
                         b[u] = *reinterpret_cast<const uint2*>(d_o + row);
@@ -426,17 +426,17 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
 
 cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, const float* lse, const int32_t* cu_seqlens,
                            const SchedView& sched, __nv_bfloat16* stats, float* dq_acc, size_t dq_acc_elems,
-                           int32_t total_tokens, int32_t n_heads, int32_t head_dim, float scale, int n_sms,
-                           cudaStream_t stream) {
+                           int32_t total_tokens, int32_t n_heads, int32_t head_dim, int64_t row_stride, float scale,
+                           int n_sms, cudaStream_t stream) {
     const int blocks = n_sms * 8;
     if (head_dim > 64)
         bwd_pre_kernel<128><<<blocks, 256, 0, stream>>>(o, d_o, lse, cu_seqlens, sched.tile_prefix, sched.n_seqs, stats,
                                                         dq_acc, dq_acc_elems / 4, total_tokens, n_heads, head_dim,
-                                                        1.0f / scale);
+                                                        row_stride, 1.0f / scale);
     else
         bwd_pre_kernel<64><<<blocks, 256, 0, stream>>>(o, d_o, lse, cu_seqlens, sched.tile_prefix, sched.n_seqs, stats,
                                                        dq_acc, dq_acc_elems / 4, total_tokens, n_heads, head_dim,
-                                                       1.0f / scale);
+                                                       row_stride, 1.0f / scale);
     return cudaGetLastError();
 }
 
@@ -447,7 +447,8 @@ cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, con
 template <int D>
 __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict__ dq,
                                                        const int32_t* __restrict__ cu, const uint32_t* __restrict__ tile_prefix,
-                                                       int32_t n_seqs, int32_t n_heads, int32_t head_dim, float scale) {
+                                                       int32_t n_seqs, int32_t n_heads, int32_t head_dim, int64_t row_stride,
+                                                       float scale) {
     constexpr int kRowBytes = D * 2 + 16;                    // padded row of bf16
     __shared__ __align__(16) uint8_t tile[kTile * kRowBytes];
     const uint32_t n_blocks = tile_prefix[n_seqs] * (uint32_t)n_heads;
@@ -486,7 +487,7 @@ __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__
         for (int e = threadIdx.x; e < rows * kChunks; e += blockDim.x) {
             const int r = e / kChunks, c = e % kChunks;
             const uint4 v = *reinterpret_cast<const uint4*>(tile + r * kRowBytes + c * 16);
-            __nv_bfloat16* out = dq + (((size_t)cu[lo] + row0 + r) * n_heads + h) * (size_t)head_dim;
+            __nv_bfloat16* out = dq + ((size_t)cu[lo] + row0 + r) * (size_t)row_stride + (size_t)h * head_dim;
             reinterpret_cast<uint4*>(out)[c] = v;
         }
         __syncthreads();
@@ -495,14 +496,15 @@ __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__
 }
 
 cudaError_t launch_bwd_post(const float* dq_acc, __nv_bfloat16* dq, const int32_t* cu_seqlens, const SchedView& sched,
-                            int32_t n_heads, int32_t head_dim, float scale, int n_sms, cudaStream_t stream) {
+                            int32_t n_heads, int32_t head_dim, int64_t row_stride, float scale, int n_sms,
+                            cudaStream_t stream) {
     const int blocks = n_sms * 4;
     if (head_dim > 64)
         bwd_post_kernel<128><<<blocks, 256, 0, stream>>>(dq_acc, dq, cu_seqlens, sched.tile_prefix, sched.n_seqs, n_heads,
-                                                         head_dim, scale);
+                                                         head_dim, row_stride, scale);
     else
         bwd_post_kernel<64><<<blocks, 256, 0, stream>>>(dq_acc, dq, cu_seqlens, sched.tile_prefix, sched.n_seqs, n_heads,
-                                                        head_dim, scale);
+                                                        head_dim, row_stride, scale);
     return cudaGetLastError();
 }
 

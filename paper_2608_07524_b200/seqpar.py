@@ -9,6 +9,11 @@ dk, dv) back.  There is no other collective, and no peer memory is touched by an
 library: the exchanges are torch.distributed calls (NCCL on GPUs, gloo in the CPU tests).
 
 Only host logic and data movement live here; the attention itself is the library's kernels.
+
+Two forms: the first re-shards with a library all-to-all around the unchanged kernels
+(scatter_heads / gather_heads / sp_attention_fwd / sp_attention_bwd); the second, at the end of this file,
+needs no all-to-all at all: the kernels work in place on token-sharded tensors that every rank has mapped
+into one address range (vmm.py) and fetch each tile from its owner when they need it.
 """
 from __future__ import annotations
 
@@ -89,3 +94,57 @@ def sp_attention_bwd(do_local, ctx, cu_seqlens, max_seqlen: int, causal: bool, g
     do = scatter_heads(do_local, slices, group)
     dq, dk, dv = attn_bwd(q, k, v, o, do, lse, cu_seqlens, max_seqlen, causal)
     return tuple(gather_heads(x, slices, group) for x in (dq, dk, dv))
+
+
+# ---- the same scheme without materialising the all-to-all ---------------------------------------------------------------
+#
+# When the token-sharded tensors of the group live in one address range on every rank (vmm.py: each rank maps
+# its own slice and its peers' slices back to back), rank r can run attention for its heads [r H/p, (r+1) H/p)
+# directly on those tensors: the strided entry points read every tile from wherever it lives (plain TMA loads,
+# no multicast) and write o / dq / dk / dv rows straight into their owners' slices.  Nothing is re-sharded and
+# no collective moves data; the ranks only have to agree on WHEN: inputs complete before anyone reads them,
+# outputs complete before anyone uses them.  `fence` is that agreement - a device synchronise followed by a
+# barrier of the group on multiple GPUs, nothing at all for virtual ranks run one after the other on one GPU.
+
+def head_group(rank: int, p: int, n_heads: int) -> slice:
+    """Heads that rank `rank` of `p` computes."""
+    if n_heads % p or not 0 <= rank < p:
+        raise ValueError("heads must divide by the group size and the rank must lie in the group")
+    hp = n_heads // p
+    return slice(rank * hp, (rank + 1) * hp)
+
+
+def group_fence(group=None):
+    """Everything this rank has enqueued is done, and every rank of the group has said the same."""
+    import torch
+    import torch.distributed as dist
+    torch.cuda.synchronize()
+    dist.barrier(group)
+
+
+def sp_attention_fwd_mapped(q, k, v, o, cu_seqlens, max_seqlen: int, causal: bool, rank: int, p: int,
+                            fence: Optional[Callable[[], None]] = None, workspace=None):
+    """Forward of rank `rank` on mapped token-sharded tensors q, k, v, o [T, H, d] (all ranks pass views of
+    the same memory).  Returns lse [H/p, T] of this rank's heads (rank-local)."""
+    from . import binding
+    hs = head_group(rank, p, q.shape[1])
+    if fence is not None:
+        fence()                       # every slice of q, k, v is complete
+    _, lse = binding.dcp_varlen_attn_fwd_strided(q[:, hs], k[:, hs], v[:, hs], cu_seqlens, max_seqlen, causal, o[:, hs],
+                                                 workspace=workspace)
+    if fence is not None:
+        fence()                       # every head group of o is complete
+    return lse
+
+
+def sp_attention_bwd_mapped(q, k, v, o, d_o, lse, dq, dk, dv, cu_seqlens, max_seqlen: int, causal: bool, rank: int, p: int,
+                            fence: Optional[Callable[[], None]] = None, workspace=None):
+    """Backward of rank `rank` on mapped token-sharded tensors; dq, dk, dv [T, H, d] receive this rank's heads."""
+    from . import binding
+    hs = head_group(rank, p, q.shape[1])
+    if fence is not None:
+        fence()                       # every slice of dO is complete
+    binding.dcp_varlen_attn_bwd_strided(q[:, hs], k[:, hs], v[:, hs], o[:, hs], d_o[:, hs], lse, cu_seqlens, max_seqlen,
+                                        causal, dq[:, hs], dk[:, hs], dv[:, hs], workspace=workspace)
+    if fence is not None:
+        fence()

@@ -439,3 +439,45 @@ def test_cta_spans_are_recorded():
         begin, end = B.dcp_read_cta_spans(ws, which)
         assert begin.size == min(n_sms, 256) and bool((end >= begin).all()) and bool((begin > 0).all())
         assert int(end.max() - begin.min()) < 10 ** 9          # nanoseconds: well under a second
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_head_groups_inside_wider_tensors(causal):
+    """The strided entry points run a group of heads in place inside [T, H, d] tensors (the form the head-
+    sharded sequence-parallel scheme needs): every group must give, bit for bit, what the plain calls give on
+    a contiguous copy of that group, and must leave the other heads' outputs alone."""
+    dev = "cuda"
+    lengths = [300, 5, 13, 129, 64, 700]
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    T, H, d, p = int(cu[-1]), 6, 128, 3
+    q, k, v, g = (x.to(dev) for x in inputs.make_qkvg(T, H, d, 97))
+    cud = torch.tensor(cu, device=dev)
+    o = torch.full_like(q, float("nan"))
+    dq, dk, dv = (torch.full_like(q, float("nan")) for _ in range(3))
+    Hg = H // p
+    for r in range(p):
+        hs = slice(r * Hg, (r + 1) * Hg)
+        qc, kc, vc, gc = (x[:, hs].contiguous() for x in (q, k, v, g))
+        ref_o, ref_lse = B.dcp_varlen_attn_fwd(qc, kc, vc, cud, max(lengths), causal)
+        ref_dq, ref_dk, ref_dv = B.dcp_varlen_attn_bwd(qc, kc, vc, ref_o, gc, ref_lse, cud, max(lengths), causal)
+        _, lse = B.dcp_varlen_attn_fwd_strided(q[:, hs], k[:, hs], v[:, hs], cud, max(lengths), causal, o[:, hs])
+        B.dcp_varlen_attn_bwd_strided(q[:, hs], k[:, hs], v[:, hs], o[:, hs], g[:, hs], lse, cud, max(lengths), causal,
+                                      dq[:, hs], dk[:, hs], dv[:, hs])
+        torch.cuda.synchronize()
+        assert torch.equal(o[:, hs], ref_o) and torch.equal(lse, ref_lse)
+        assert torch.equal(dk[:, hs], ref_dk) and torch.equal(dv[:, hs], ref_dv)
+        assert float((dq[:, hs].float() - ref_dq.float()).abs().max()) <= 2e-2       # atomics: order may differ
+        if r + 1 < p:       # heads of later groups are still untouched
+            rest = slice((r + 1) * Hg, H)
+            assert bool(torch.isnan(o[:, rest].float()).all()) and bool(torch.isnan(dk[:, rest].float()).all())
+    O, L = oracle.attn_fwd(q.cpu(), k.cpu(), v.cpu(), cu, causal)
+    rdq, rdk, rdv = oracle.attn_bwd(q.cpu(), k.cpu(), v.cpu(), g.cpu(), cu, causal)
+    assert_close("o", o, O)
+    assert_close("dq", dq, rdq)
+    assert_close("dk", dk, rdk)
+    assert_close("dv", dv, rdv)
+    # a stride smaller than the group's own width is refused
+    rc = B.lib().dcp_varlen_attn_fwd_strided(q.data_ptr(), k.data_ptr(), v.data_ptr(), cud.data_ptr(), len(lengths), T,
+                                             max(lengths), Hg, d, Hg * d - 8, 0, 0.0, o.data_ptr(), lse.data_ptr(),
+                                             B.alloc_workspace(T, len(lengths), Hg, d, False, dev).data_ptr(), 1 << 20, None)
+    assert rc == B.DCP_ERR_INVALID_ARG
