@@ -427,13 +427,13 @@ def run_ours(args):
                 "traffic": load_dram_traffic(args.workload) if plain else None,
                 "launches": bwd_n, "avg_launch_ms": bwd_ms / max(bwd_n, 1)}
     if axis == "temporal" and bwd_n:
-        # sequences of 1-13 tokens: a tile pair does ~1 % useful arithmetic, the kernel is bound by HBM.
-        # Algorithmic bytes of the backward main kernel per (token, head): q, k, v, dO read and dq, dk, dv
-        # written (7 d bf16; a sequence of one tile gets its dq written directly), lse and D read (8).
+        # sequences of 1-13 tokens run on the short-sequence kernels, which are bound by HBM.  Algorithmic bytes of
+        # the backward kernel per (token, head): q, k, v, dO read and dq, dk, dv written (7 d bf16), lse read (4);
+        # D is formed in registers and o is not read.
         tok_per_launch = tokens_all / world / max(bwd_n, 1)
-        gbs = tok_per_launch * H * (7 * d * 2 + 8) / (bwd_ms / bwd_n * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": "attn_bwd_kernel (backward main)", "achieved": gbs, "peak": peaks["hbm_gbs"],
-                    "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+        gbs = tok_per_launch * H * (7 * d * 2 + 4) / (bwd_ms / bwd_n * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "small_attn_kernel (backward, short sequences)", "achieved": gbs,
+                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                     "peak_source": f"hbm_gbs of {peaks['source']} MEASURED_PEAKS.json",
                     "traffic": load_dram_traffic("temporal2d") if d == 128 else None,
                     "launches": bwd_n, "avg_launch_ms": bwd_ms / bwd_n}

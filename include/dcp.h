@@ -312,6 +312,17 @@ int dcp_selftest_wait_timeout(void* workspace, uint32_t spin_limit, void* cuda_s
  * backward main (which = 1) launch on `workspace`, when each persistent CTA started and when it ran
  * out of work, in nanoseconds of the GPU's global timer: begin_ns, end_ns [256] (host), *n_ctas valid. */
 int dcp_set_work_order(int input_order);
+
+/* Batches of very short sequences (Section 4.1: the temporal axis of a 2-D model has sequences of a handful
+ * of tokens).  When the declared max_seqlen is at most 32, dcp_varlen_attn_fwd/bwd (and their strided and
+ * no-allocation forms) run one small CTA per (sequence, group of heads) that fetches exactly the sequence's
+ * rows, instead of the work list and the 128-row tile kernels: such a batch is bound by HBM, and what it needs
+ * is many sequences in flight per SM.  Results are the same within rounding; the backward then forms
+ * D_i = sum_j P_ij dP_ij itself and does not read `o`; a sequence longer than the declared max_seqlen makes
+ * dcp_query_status report DCP_ERR_INVALID_ARG and nothing is computed (as on the other path).
+ * dcp_set_short_sequence_path(0) sends such batches through the tile kernels instead (a measurement aid and
+ * a test hook); 1 restores the default.  Process-wide. */
+int dcp_set_short_sequence_path(int enabled);
 int dcp_read_cta_spans(const void* workspace, int32_t which, void* cuda_stream, int64_t* begin_ns, int64_t* end_ns,
                        int32_t* n_ctas);
 

@@ -84,6 +84,8 @@ def lib():
             L.dcp_selftest_wait_timeout.restype = ctypes.c_int
             L.dcp_set_work_order.argtypes = [ctypes.c_int]
             L.dcp_set_work_order.restype = ctypes.c_int
+            L.dcp_set_short_sequence_path.argtypes = [ctypes.c_int]
+            L.dcp_set_short_sequence_path.restype = ctypes.c_int
             L.dcp_read_cta_spans.argtypes = [vp, i32, vp, i64p, i64p, i32p]
             L.dcp_read_cta_spans.restype = ctypes.c_int
             L.dcp_plan_segments.argtypes = [i32p, i32p, i32, i32, i32, i32p, i32p, i32p, i32p, i32p, i32, i32p]
@@ -355,6 +357,12 @@ def dcp_selftest_wait_timeout(workspace, spin_limit: int = 1 << 10, stream=None)
 def dcp_set_work_order(input_order: bool) -> None:
     """Measurement aid: list sequences as they come (True) instead of longest first (False, default)."""
     _check(lib().dcp_set_work_order(int(bool(input_order))))
+
+
+def dcp_set_short_sequence_path(enabled: bool) -> None:
+    """Measurement aid and test hook: batches whose declared max_seqlen is at most 32 run on the small per-sequence
+    kernels (True, default) or on the tile kernels like every other batch (False)."""
+    _check(lib().dcp_set_short_sequence_path(int(bool(enabled))))
 
 
 def dcp_read_cta_spans(workspace, which: int, stream=None):

@@ -17,7 +17,7 @@ CSRC = os.path.join(_DIR, "csrc")
 OBJ_DIR = os.path.join(CSRC, "build")
 LIB_PATH = os.path.join(_DIR, "libdcp.so")
 SOURCES = ["api.cu", "plan.cpp", "inter.cpp", "intra.cpp", "model.cpp", "prep.cu", "util_kernels.cu", "attn_fwd.cu",
-           "attn_bwd.cu"]
+           "attn_bwd.cu", "attn_small.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

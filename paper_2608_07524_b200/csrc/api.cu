@@ -27,6 +27,7 @@ namespace {
 
 std::atomic<int64_t> g_launches{0};
 std::atomic<int> g_input_order{0};      // dcp_set_work_order: 1 = list sequences as they come
+std::atomic<int> g_short_path{1};       // dcp_set_short_sequence_path: 0 = batches of very short sequences run on the tile kernels
 
 // Optional per-kernel timing: event pairs recorded on the caller's stream around every launch.  Events
 // are created once and recycled through a pool (dcp_profile_read hands them back), so that a timed
@@ -184,6 +185,11 @@ SchedView carve_sched(void* workspace, int32_t n_seqs) {
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// Whether a call takes the path for batches of very short sequences (see attn_small.cu).
+bool short_sequence_path(int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen) {
+    return g_short_path.load() != 0 && small_path_fits(n_seqs, total_tokens, max_seqlen);
+}
+
 // Batches whose longest sequence has at most this many tokens (64 key tiles) run the forward variant for short items.
 constexpr int32_t kShortItemMaxLen = 8192;
 
@@ -238,6 +244,28 @@ static int attn_fwd_impl(const char* fn, bool merge, const void* q, const void* 
     const SchedView sched = carve_sched(workspace, n_seqs);
     uint16_t* bounds = merge ? reinterpret_cast<uint16_t*>(static_cast<uint8_t*>(workspace) + sched_bytes(n_seqs)) : nullptr;
     cudaError_t e;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
+    if (short_sequence_path(n_seqs, total_tokens, max_seqlen)) {
+        int32_t* first_seq = const_cast<int32_t*>(sched.order);      // the work list's arrays are free on this path
+        {
+            ScopedTimer t(DCP_KERNEL_PREP, stream);
+            e = launch_small_check(false, cu_seqlens, n_seqs, total_tokens, max_seqlen, n_heads, sched.hdr, first_seq, dev.sm_count,
+                                   stream);
+        }
+        if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: boundary check kernel: %s", fn, cudaGetErrorString(e));
+        g_launches.fetch_add(1);
+        if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
+        {
+            ScopedTimer t(DCP_KERNEL_FWD, stream);
+            e = launch_small_attn(false, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
+                                  static_cast<const __nv_bfloat16*>(v), nullptr, lse, cu_seqlens, total_tokens, max_seqlen,
+                                  n_heads, head_dim, token_stride, causal != 0, scale, static_cast<__nv_bfloat16*>(o), nullptr,
+                                  nullptr, nullptr, sched.hdr, first_seq, dev.sm_count, stream);
+        }
+        if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: short-sequence kernel: %s", fn, cudaGetErrorString(e));
+        g_launches.fetch_add(1);
+        return DCP_OK;
+    }
     const bool input_order = g_input_order.load() != 0;
     {
         ScopedTimer t(DCP_KERNEL_PREP, stream);
@@ -263,7 +291,7 @@ static int attn_fwd_impl(const char* fn, bool merge, const void* q, const void* 
     p.head_dim = head_dim;
     p.total_tokens = total_tokens;
     p.row_stride = token_stride;
-    p.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
+    p.scale = scale;
     p.scale_log2 = p.scale * 1.4426950408889634f;
     {
         ScopedTimer t(DCP_KERNEL_FWD, stream);
@@ -324,6 +352,29 @@ static int attn_bwd_impl(const char* fn, const void* q, const void* k, const voi
     float* dq_acc = reinterpret_cast<float*>(base + align256(max_tiles(total_tokens, n_seqs) * n_heads * (size_t)(kTile * 16 * 2)));
 
     cudaError_t e;
+    if (short_sequence_path(n_seqs, total_tokens, max_seqlen)) {
+        int32_t* first_seq = const_cast<int32_t*>(sched.order);      // the work list's arrays are free on this path
+        {
+            ScopedTimer t(DCP_KERNEL_PREP, stream);
+            e = launch_small_check(true, cu_seqlens, n_seqs, total_tokens, max_seqlen, n_heads, sched.hdr, first_seq, dev.sm_count,
+                                   stream);
+        }
+        if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: boundary check kernel: %s", fn, cudaGetErrorString(e));
+        g_launches.fetch_add(1);
+        if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
+        {
+            ScopedTimer t(DCP_KERNEL_BWD_MAIN, stream);
+            e = launch_small_attn(true, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
+                                  static_cast<const __nv_bfloat16*>(v), static_cast<const __nv_bfloat16*>(d_o),
+                                  const_cast<float*>(lse), cu_seqlens, total_tokens, max_seqlen, n_heads, head_dim, token_stride,
+                                  causal != 0, softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim), nullptr,
+                                  static_cast<__nv_bfloat16*>(dq), static_cast<__nv_bfloat16*>(dk),
+                                  static_cast<__nv_bfloat16*>(dv), sched.hdr, first_seq, dev.sm_count, stream);
+        }
+        if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: short-sequence kernel: %s", fn, cudaGetErrorString(e));
+        g_launches.fetch_add(1);
+        return DCP_OK;
+    }
     const bool input_order = g_input_order.load() != 0;
     {
         ScopedTimer t(DCP_KERNEL_PREP, stream);
@@ -486,6 +537,11 @@ extern "C" int dcp_query_status(void* workspace, void* cuda_stream) {
 
 extern "C" int dcp_set_work_order(int input_order) {
     g_input_order.store(input_order ? 1 : 0);
+    return DCP_OK;
+}
+
+extern "C" int dcp_set_short_sequence_path(int enabled) {
+    g_short_path.store(enabled ? 1 : 0);
     return DCP_OK;
 }
 

@@ -83,4 +83,19 @@ cudaError_t launch_bwd_post(const float* dq_acc, __nv_bfloat16* dq, const int32_
                             int32_t n_heads, int32_t head_dim, int64_t row_stride, float scale, int n_sms,
                             cudaStream_t stream);
 
+// Batches in which no sequence exceeds kSmallSeqMaxLen tokens (the declared max_seqlen says so) skip the work list
+// and the 128-row tile kernels, see attn_small.cu.  The check kernel is the first of such a call (boundaries
+// consistent, no sequence longer than declared; it also fills first_seq, 2 n_seqs + 1 entries of scratch); the
+// attention kernel computes nothing if it found a fault.  The backward does not read `o`.
+constexpr int kSmallSeqMaxLen = 32;
+bool small_path_fits(int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen);
+cudaError_t launch_small_check(bool backward, const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen,
+                               int32_t n_heads, WorkspaceHeader* hdr, int32_t* first_seq, int n_sms, cudaStream_t stream);
+// forward: o and lse written (d_o, dq, dk, dv null); backward: lse read, dq, dk, dv written (o null)
+cudaError_t launch_small_attn(bool backward, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                              const __nv_bfloat16* d_o, float* lse, const int32_t* cu_seqlens, int32_t total_tokens,
+                              int32_t max_seqlen, int32_t n_heads, int32_t head_dim, int64_t row_stride, bool causal, float scale,
+                              __nv_bfloat16* o, __nv_bfloat16* dq, __nv_bfloat16* dk, __nv_bfloat16* dv, WorkspaceHeader* hdr,
+                              const int32_t* first_seq, int n_sms, cudaStream_t stream);
+
 }  // namespace dcp

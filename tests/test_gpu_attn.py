@@ -124,12 +124,88 @@ def test_many_short_sequences(causal):
     check_full([int(x) for x in rng.integers(1, 200, size=300)], 2, 64, causal, seed=5)
 
 
+@pytest.fixture(params=["short-sequence kernels", "tile kernels"])
+def both_paths(request):
+    """Batches whose longest sequence has at most 32 tokens take the per-sequence kernels by default; the tile
+    kernels (merged runs of short sequences) must keep handling them too."""
+    B.dcp_set_short_sequence_path(request.param == "short-sequence kernels")
+    yield request.param
+    B.dcp_set_short_sequence_path(True)
+
+
 @pytest.mark.parametrize("causal", [False, True])
 @pytest.mark.parametrize("d", [64, 128])
-def test_merged_tiny_sequences(causal, d):
+def test_merged_tiny_sequences(causal, d, both_paths):
     # a 2-D model's temporal axis: thousands of sequences of 1-13 tokens, several of which share one tile
     rng = np.random.default_rng(11)
     check_full([int(x) for x in rng.choice([1, 4, 8, 13], size=700)], 2, d, causal, seed=11)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("H,d", [(4, 128), (16, 128), (2, 64), (3, 72), (1, 8), (6, 40), (12, 104), (4, 120), (5, 16)])
+@pytest.mark.parametrize("max_len", [2, 13, 16, 17, 32])
+def test_short_sequence_kernels(causal, H, d, max_len):
+    """One CTA per (sequence, group of heads): every head-group width (4, 2, 1 heads), head dimensions with and
+    without a last half k-step, one and two 16-row blocks, empty sequences, the longest allowed sequence."""
+    rng = np.random.default_rng(1000 * max_len + H)
+    lengths = [int(x) for x in rng.integers(0, max_len + 1, size=150)] + [max_len, 0, max_len, 1]
+    check_full(lengths, H, d, causal, seed=50 + max_len, scale=0.0 if d != 40 else 0.2)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_short_sequence_kernels_on_single_tokens(causal):
+    # closed form for L = 1: O = V, lse = the one score, dV = dO, dQ = dK = 0
+    dev = "cuda"
+    T, H, d = 500, 4, 128
+    q, k, v, g = (x.to(dev) for x in inputs.make_qkvg(T, H, d, 3))
+    cu = torch.arange(T + 1, dtype=torch.int32, device=dev)
+    o, lse = B.dcp_varlen_attn_fwd(q, k, v, cu, 1, causal)
+    dq, dk, dv = B.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cu, 1, causal)
+    assert torch.equal(o, v) and torch.equal(dv, g)
+    score = (q.double() * k.double()).sum(-1) / d ** 0.5
+    assert float((lse.double() - score.t()).abs().max()) <= 1e-4
+    assert float(dq.float().abs().max()) <= 1e-4 and float(dk.float().abs().max()) <= 1e-4
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_short_sequence_kernels_agree_with_the_tile_kernels(causal):
+    dev = "cuda"
+    rng = np.random.default_rng(77)
+    lengths = [int(x) for x in rng.integers(1, 14, size=3000)]
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    T, H, d = int(cu[-1]), 8, 128
+    q, k, v, g = (x.to(dev) for x in inputs.make_qkvg(T, H, d, 78))
+    cud = torch.tensor(cu, device=dev)
+    out = []
+    for short in (True, False):
+        B.dcp_set_short_sequence_path(short)
+        try:
+            o, lse = B.dcp_varlen_attn_fwd(q, k, v, cud, 13, causal)
+            out.append((o, lse) + tuple(B.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cud, 13, causal)))
+        finally:
+            B.dcp_set_short_sequence_path(True)
+    for name, a, b in zip(("o", "lse", "dq", "dk", "dv"), *out):
+        # both are within tolerance of the oracle; against each other, a bf16 unit in the last place of the largest values
+        assert float((a.float() - b.float()).abs().max()) <= (MAX_ABS if name != "lse" else 1e-4), name
+
+
+def test_short_sequence_kernels_refuse_a_sequence_longer_than_declared():
+    dev = "cuda"
+    cu = torch.tensor([0, 5, 14, 20], dtype=torch.int32, device=dev)          # the middle sequence has 9 tokens
+    q, k, v, g = (x.to(dev) for x in inputs.make_qkvg(20, 4, 64, 5))
+    buf = Guarded(20, 4, 64, 3, dev)
+    before = [b.clone() for b in buf.bf16]
+    B.dcp_varlen_attn_fwd(q, k, v, cu, 8, False, out=buf.o, lse=buf.lse, workspace=buf.ws)
+    with pytest.raises(B.DcpError) as e:
+        B.dcp_query_status(buf.ws)
+    assert e.value.code == B.DCP_ERR_INVALID_ARG
+    B.dcp_varlen_attn_bwd(q, k, v, q, g, torch.zeros(4, 20, device=dev), cu, 8, False, dq=buf.dq, dk=buf.dk, dv=buf.dv,
+                          workspace=buf.ws)
+    with pytest.raises(B.DcpError):
+        B.dcp_query_status(buf.ws)
+    assert all(torch.equal(a, b) for a, b in zip(before, buf.bf16))           # nothing was computed
+    B.dcp_varlen_attn_fwd(q, k, v, cu, 9, False, out=buf.o, lse=buf.lse, workspace=buf.ws)      # declared correctly: fine
+    B.dcp_query_status(buf.ws)
 
 
 @pytest.mark.parametrize("causal", [False, True])
@@ -340,9 +416,17 @@ def test_inconsistent_boundaries_are_reported_not_used():
         assert bool(torch.isfinite(o.float()).all()) and not bool((o == 7.0).all())
 
 
-def test_understated_max_seqlen_cannot_overrun_the_workspace():
+@pytest.fixture
+def tile_kernels_only():
+    B.dcp_set_short_sequence_path(False)
+    yield
+    B.dcp_set_short_sequence_path(True)
+
+
+def test_understated_max_seqlen_cannot_overrun_the_workspace(tile_kernels_only):
     # 2000 sequences of 14 tokens declared as "at most 13": none is merged, so the batch has more tiles than
     # the workspace (sized on the promise) holds; the backward must refuse instead of indexing past its storage
+    # (on the tile kernels: the short-sequence kernels refuse the forward already, tested above)
     dev = "cuda"
     n, L, H, d = 2000, 14, 1, 64
     T = n * L
@@ -441,13 +525,14 @@ def test_cta_spans_are_recorded():
         assert int(end.max() - begin.min()) < 10 ** 9          # nanoseconds: well under a second
 
 
+@pytest.mark.parametrize("lengths", [[300, 5, 13, 129, 64, 700], [13, 1, 0, 7, 16, 9, 12, 3] * 40],
+                         ids=["tile kernels", "short-sequence kernels"])
 @pytest.mark.parametrize("causal", [False, True])
-def test_head_groups_inside_wider_tensors(causal):
+def test_head_groups_inside_wider_tensors(causal, lengths):
     """The strided entry points run a group of heads in place inside [T, H, d] tensors (the form the head-
     sharded sequence-parallel scheme needs): every group must give, bit for bit, what the plain calls give on
     a contiguous copy of that group, and must leave the other heads' outputs alone."""
     dev = "cuda"
-    lengths = [300, 5, 13, 129, 64, 700]
     cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
     T, H, d, p = int(cu[-1]), 6, 128, 3
     q, k, v, g = (x.to(dev) for x in inputs.make_qkvg(T, H, d, 97))
