@@ -651,7 +651,9 @@ struct StageLayout {
 };
 __host__ __device__ inline StageLayout stage_layout(int n_tiles, int rows, int head_dim, bool with_lse) {
     StageLayout l;
-    l.pitch = (uint32_t)head_dim * 2 + 16;          // 8 extra elements per row keep ldmatrix free of bank conflicts
+    // 16 or 32 extra bytes per row make the pitch an odd number of 16-byte units: ldmatrix and stmatrix touch eight
+    // rows at one column, which then fall into eight different bank groups
+    l.pitch = (uint32_t)head_dim * 2 + ((head_dim / 8) % 2 ? 32 : 16);
     l.tile_bytes = (uint32_t)rows * l.pitch;
     l.lse_off = (uint32_t)n_tiles * l.tile_bytes;
     l.stage_bytes = (l.lse_off + (with_lse ? (uint32_t)rows * 4 : 0) + 127) & ~127u;
