@@ -8,6 +8,7 @@
 namespace dcp {
 
 constexpr int kPrepThreads = 1024;
+constexpr int kRankInKernelMax = 256;     // above this many sequences the rank sort runs over several CTAs (rank_kernel)
 
 __device__ inline uint32_t block_exclusive_scan(uint32_t v, uint32_t* scratch, uint32_t* total);
 __device__ inline int block_exclusive_max_scan(int v, int* scratch);
@@ -92,24 +93,25 @@ __global__ void __launch_bounds__(kPrepThreads) merge_kernel(const int32_t* __re
     }
 }
 
-// One thread per input sequence of at most 128 tokens, over as many CTAs as needed: bounds[t] for
+// One warp per input sequence of at most 128 tokens, over as many CTAs as needed: bounds[t] for
 // each of its tokens t = (first, end) position of the sequence relative to the start of its virtual
-// sequence, one byte each.  merge_kernel has left that start in vstart[].
+// sequence, one byte each (the lanes write consecutive tokens).  merge_kernel has left that start in vstart[].
 __global__ void __launch_bounds__(256) bounds_kernel(const int32_t* __restrict__ cu, int32_t n_seqs,
                                                      const WorkspaceHeader* __restrict__ hdr,
                                                      const int32_t* __restrict__ vstart, uint16_t* __restrict__ bounds) {
-    const int i = blockIdx.x * 256 + threadIdx.x;
+    const int i = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (i >= n_seqs || hdr->call_bad) return;      // merge_kernel found the boundaries inconsistent
     const int32_t a = cu[i], b = cu[i + 1];
     if (b == a || b - a > kTile) return;
     const int32_t v0 = vstart[i];
     const uint16_t packed = (uint16_t)((a - v0) | ((b - v0) << 8));
-    for (int32_t t = a; t < b; ++t) bounds[t] = packed;
+    for (int32_t t = a + lane; t < b; t += 32) bounds[t] = packed;
 }
 
 // Rank sort, one thread per sequence over as many CTAs as needed: order[] = sequence ids sorted by
-// (length descending, id ascending).  Used on its own for batches of more than kPrepThreads
-// sequences; small batches do the same loop inside prep_kernel and save the launch.  Sequences
+// (length descending, id ascending).  Used on its own for batches of more than kRankInKernelMax
+// sequences (one CTA doing it for a thousand sequences takes 37 us, eight CTAs 4 us); small batches do the
+// same loop inside prep_kernel and save the launch.  Sequences
 // from *n_live on (if given) are empty padding: they keep their own index as rank and are not
 // compared against.
 __global__ void __launch_bounds__(256) rank_kernel(const int32_t* __restrict__ cu, int32_t n_seqs,
@@ -226,7 +228,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __res
     }
     if (ranked == 2) {
         for (int i = tid; i < n_seqs; i += kPrepThreads) order[i] = i;
-    } else if (!ranked) {                             // n_seqs <= kPrepThreads: one sequence per thread
+    } else if (!ranked) {                             // n_seqs <= kRankInKernelMax: one sequence per thread
         len_sh[tid] = tid < n_seqs ? cu[tid + 1] - cu[tid] : -1;
         __syncthreads();
         if (tid < n_seqs) {
@@ -283,7 +285,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const int32_t* __res
 }
 
 int prep_launches(int32_t n_seqs, bool merge, bool input_order) {
-    return (n_seqs > kPrepThreads && !input_order ? 2 : 1) + (merge ? (n_seqs > 0 ? 2 : 1) : 0);
+    return (n_seqs > kRankInKernelMax && !input_order ? 2 : 1) + (merge ? (n_seqs > 0 ? 2 : 1) : 0);
 }
 
 cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens, int32_t max_seqlen,
@@ -298,12 +300,12 @@ cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total
                                                      const_cast<int32_t*>(sched.vcu), const_cast<int32_t*>(sched.order));
         if (cudaError_t e = cudaGetLastError()) return e;
         if (n_seqs > 0)
-            bounds_kernel<<<(n_seqs + 255) / 256, 256, 0, stream>>>(cu_seqlens, n_seqs, sched.hdr, sched.order, bounds);
+            bounds_kernel<<<(n_seqs + 7) / 8, 256, 0, stream>>>(cu_seqlens, n_seqs, sched.hdr, sched.order, bounds);
         if (cudaError_t e = cudaGetLastError()) return e;
         cu = sched.vcu;
         n_live = &sched.hdr->n_vseq;
     }
-    const int ranked = input_order ? 2 : (n_seqs > kPrepThreads ? 1 : 0);
+    const int ranked = input_order ? 2 : (n_seqs > kRankInKernelMax ? 1 : 0);
     if (ranked == 1) {
         rank_kernel<<<(n_seqs + 255) / 256, 256, 0, stream>>>(cu, n_seqs, n_live, const_cast<int32_t*>(sched.order));
         if (cudaError_t e = cudaGetLastError()) return e;
@@ -312,6 +314,34 @@ cudaError_t launch_prep(const int32_t* cu_seqlens, int32_t n_seqs, int32_t total
                                                 const_cast<int32_t*>(sched.order), const_cast<uint32_t*>(sched.prefix),
                                                 const_cast<uint32_t*>(sched.tile_prefix), ranked, total_tokens, tile_capacity);
     return cudaGetLastError();
+}
+
+// The sequence that owns 128-row tile t: (sequence, first row of the tile inside it, its length, its first token).
+// A binary search of dependent loads, a few microseconds when they miss L1: the helper kernels below look up the
+// NEXT block's tile while the current block's loads are in flight.
+struct TileRef {
+    int seq, row0, len, tok0;
+};
+__device__ __forceinline__ TileRef find_tile(const int32_t* __restrict__ cu, const uint32_t* __restrict__ tile_prefix, int32_t n_seqs,
+                                             uint32_t t) {
+    int lo = 0, hi = n_seqs;
+    // when every sequence so far has exactly one tile (batches of merged short sequences), tile t belongs
+    // to sequence t: check that before paying for the search
+    if ((int)t < n_seqs && tile_prefix[t] <= t && tile_prefix[t + 1] > t) {
+        lo = (int)t;
+        hi = lo + 1;
+    }
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (tile_prefix[mid] <= t) lo = mid; else hi = mid;
+    }
+    while (lo + 1 < n_seqs && tile_prefix[lo + 1] <= t) ++lo;   // skip empty sequences
+    TileRef r;
+    r.seq = lo;
+    r.row0 = (int)(t - tile_prefix[lo]) * kTile;
+    r.tok0 = cu[lo];
+    r.len = cu[lo + 1] - r.tok0;
+    return r;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -335,20 +365,10 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
     const uint32_t n_blocks = tile_prefix[n_seqs] * (uint32_t)n_heads;
     for (uint32_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
         const uint32_t t = blk / n_heads, h = blk % n_heads;
-        int lo = 0, hi = n_seqs;                              // sequence owning tile t
-        // when every sequence so far has exactly one tile (batches of merged short sequences), tile t belongs
-        // to sequence t: check that before paying for a binary search of dependent loads
-        if ((int)t < n_seqs && tile_prefix[t] <= t && tile_prefix[t + 1] > t) {
-            lo = (int)t;
-            hi = lo + 1;
-        }
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (tile_prefix[mid] <= t) lo = mid; else hi = mid;
-        }
-        while (lo + 1 < n_seqs && tile_prefix[lo + 1] <= t) ++lo;   // skip empty sequences
-        const int row0 = (int)(t - tile_prefix[lo]) * kTile;
-        const int len = cu[lo + 1] - cu[lo];
+        // (looking the next block's tile up while this block's loads are in flight, as the post kernel does, made
+        // this kernel slower: 0.39 -> 0.44 ms on 131072 tokens x 16 heads)
+        const TileRef ref = find_tile(cu, tile_prefix, n_seqs, t);
+        const int row0 = ref.row0, len = ref.len, tok0 = ref.tok0;
         if (len > kTile) {
             // this (tile, head) block of the dQ accumulator; a sequence of a single tile needs none (its
             // one tile pair yields the whole dQ, which the main kernel writes directly)
@@ -358,66 +378,67 @@ __global__ void __launch_bounds__(256) bwd_pre_kernel(const __nv_bfloat16* __res
         }
         {
         uint8_t* out = reinterpret_cast<uint8_t*>(stats) + ((size_t)t * n_heads + h) * (kTile * 16 * 2);
-        // a warp takes rows warp, warp+8, ...; four rows per pass so that eight loads are in flight per lane
-        constexpr int kPer = D / 32;           // elements per lane: 2 or 4
-        const bool lane_live = lane * kPer < head_dim;
-        const int lane_col = lane_live ? lane * kPer : 0;
-        for (int r0 = warp; r0 < kTile; r0 += 32) {
-            float acc[4], nl[4];
-            uint2 a[4], b[4];
+        // Half a warp reads a row with 16-byte loads (D = 128; a quarter warp for D = 64), so that a warp
+        // instruction covers 2 (4) rows; a warp takes 16 rows per pass with eight loads of 16 bytes in flight per
+        // lane (the kernel waits on HBM latency: bytes in flight are what it runs on).
+        constexpr int kLanesPerRow = D / 8;                 // 16 or 8
+        constexpr int kRowsPerInst = 32 / kLanesPerRow;     // 2 or 4
+        constexpr int kU = 4;                               // row groups in flight per lane
+        const int sub = lane / kLanesPerRow, col = (lane % kLanesPerRow) * 8;
+        const bool lane_live = col < head_dim;
+        const int lane_col = lane_live ? col : 0;
+        for (int r0 = warp * kRowsPerInst * kU; r0 < kTile; r0 += 8 * kRowsPerInst * kU) {
+            uint4 a[kU], b[kU];
+            float nl[kU], acc[kU];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int r = r0 + 8 * u;
-                a[u] = make_uint2(0u, 0u);
-                b[u] = make_uint2(0u, 0u);
+            for (int u = 0; u < kU; ++u) {
+                const int r = r0 + u * kRowsPerInst + sub;
+                a[u] = make_uint4(0u, 0u, 0u, 0u);
+                b[u] = make_uint4(0u, 0u, 0u, 0u);
                 nl[u] = -1e30f;
                 if (row0 + r < len) {
-                    const size_t tok = (size_t)cu[lo] + row0 + r;
+                    const size_t tok = (size_t)tok0 + row0 + r;
                     // rows hold head_dim <= D columns; lanes past them re-read column 0 and drop it, so that the
-                    // loads stay unconditional and eight of them are in flight per lane
+                    // loads stay unconditional
                     const size_t row = tok * (size_t)row_stride + (size_t)h * head_dim + lane_col;
-                    if (kPer == 4) {
-                        a[u] = *reinterpret_cast<const uint2*>(o + row);
-                        b[u] = *reinterpret_cast<const uint2*>(d_o + row);
-                    } else {
-                        a[u].x = *reinterpret_cast<const uint32_t*>(o + row);
-                        b[u].x = *reinterpret_cast<const uint32_t*>(d_o + row);
-                    }
-                    if (!lane_live) a[u] = make_uint2(0u, 0u);
-                    if (lane == 0) nl[u] = -lse[(size_t)h * total_tokens + tok] * inv_scale;
+                    a[u] = *reinterpret_cast<const uint4*>(o + row);
+                    b[u] = *reinterpret_cast<const uint4*>(d_o + row);
+                    if (!lane_live) a[u] = make_uint4(0u, 0u, 0u, 0u);
+                    if (lane % kLanesPerRow == 0) nl[u] = -lse[(size_t)h * total_tokens + tok] * inv_scale;
                 }
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a[u].x));
-                const float2 a1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a[u].y));
-                const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b[u].x));
-                const float2 b1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b[u].y));
-                acc[u] = a0.x * b0.x + a0.y * b0.y + a1.x * b1.x + a1.y * b1.y;     // unused halves are zero
+            for (int u = 0; u < kU; ++u) {
+                const uint32_t aw[4] = {a[u].x, a[u].y, a[u].z, a[u].w}, bw[4] = {b[u].x, b[u].y, b[u].z, b[u].w};
+                float sum = 0.f;
 #pragma unroll
-                for (int sft = 16; sft > 0; sft >>= 1) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], sft);
+                for (int w = 0; w < 4; ++w) {
+                    const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&aw[w]));
+                    const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bw[w]));
+                    sum += x.x * y.x + x.y * y.y;
+                }
+#pragma unroll
+                for (int sft = kLanesPerRow / 2; sft > 0; sft >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, sft);
+                acc[u] = sum;
             }
-            // lane 0 holds the lse terms; lanes 0..3 write the lse chunk of row u, lanes 4..7 its D chunk
-            const int u = lane & 3;
-            float nl_b[4];
+            // the first lane of a row's group writes its lse chunk, the second its D chunk
+            const int role = lane % kLanesPerRow;
+            if (role < 2) {
 #pragma unroll
-            for (int t = 0; t < 4; ++t) nl_b[t] = __shfl_sync(0xffffffffu, nl[t], 0);
-            const float nl_u = u == 0 ? nl_b[0] : u == 1 ? nl_b[1] : u == 2 ? nl_b[2] : nl_b[3];
-            if (lane < 8) {
-                const int r = r0 + 8 * u;
-                const float acc_u = u == 0 ? acc[0] : u == 1 ? acc[1] : u == 2 ? acc[2] : acc[3];
-                const int which = lane >> 2;                      // 0: lse term -> column half 0, 1: D term -> half 1
-                const float x = which == 0 ? nl_u : -acc_u;
-                const __nv_bfloat16 b0 = __float2bfloat16(x);
-                const float r1 = x - __bfloat162float(b0);
-                const __nv_bfloat16 b1 = __float2bfloat16(r1);
-                const __nv_bfloat16 b2 = __float2bfloat16(r1 - __bfloat162float(b1));
-                uint4 v;
-                v.x = (uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16);
-                v.y = (uint32_t)__bfloat16_as_ushort(b2);
-                v.z = 0u;
-                v.w = 0u;
-                *reinterpret_cast<uint4*>(out + which * 2048 + (r / 8) * 128 + (r % 8) * 16) = v;
+                for (int u = 0; u < kU; ++u) {
+                    const int r = r0 + u * kRowsPerInst + sub;
+                    const float x = role == 0 ? nl[u] : -acc[u];      // every lane of the group holds the row's sum
+                    const __nv_bfloat16 b0 = __float2bfloat16(x);
+                    const float r1 = x - __bfloat162float(b0);
+                    const __nv_bfloat16 b1 = __float2bfloat16(r1);
+                    const __nv_bfloat16 b2 = __float2bfloat16(r1 - __bfloat162float(b1));
+                    uint4 v;
+                    v.x = (uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16);
+                    v.y = (uint32_t)__bfloat16_as_ushort(b2);
+                    v.z = 0u;
+                    v.w = 0u;
+                    *reinterpret_cast<uint4*>(out + role * 2048 + (r / 8) * 128 + (r % 8) * 16) = v;
+                }
             }
         }
         }
@@ -452,53 +473,53 @@ __global__ void __launch_bounds__(256) bwd_post_kernel(const float* __restrict__
     constexpr int kRowBytes = D * 2 + 16;                    // padded row of bf16
     __shared__ __align__(16) uint8_t tile[kTile * kRowBytes];
     const uint32_t n_blocks = tile_prefix[n_seqs] * (uint32_t)n_heads;
-    for (uint32_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
+    if (blockIdx.x >= n_blocks) return;
+    TileRef ref = find_tile(cu, tile_prefix, n_seqs, blockIdx.x / n_heads), ref_next = ref;
+    for (uint32_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x, ref = ref_next) {
         const uint32_t t = blk / n_heads, h = blk % n_heads;
-        int lo = 0, hi = n_seqs;                              // sequence owning tile t
-        // when every sequence so far has exactly one tile (batches of merged short sequences), tile t belongs
-        // to sequence t: check that before paying for a binary search of dependent loads
-        if ((int)t < n_seqs && tile_prefix[t] <= t && tile_prefix[t + 1] > t) {
-            lo = (int)t;
-            hi = lo + 1;
-        }
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (tile_prefix[mid] <= t) lo = mid; else hi = mid;
-        }
-        while (lo + 1 < n_seqs && tile_prefix[lo + 1] <= t) ++lo;   // skip empty sequences
-        const int row0 = (int)(t - tile_prefix[lo]) * kTile;
-        const int len = cu[lo + 1] - cu[lo];
+        const bool more = blk + gridDim.x < n_blocks;
+        const uint32_t t_next = (blk + gridDim.x) / n_heads;
+        const int row0 = ref.row0, len = ref.len;
         const int rows = min(kTile, len - row0);
-        if (len <= kTile) continue;       // a single tile pair: the main kernel has written dq itself
-        {
+        if (len <= kTile) {               // a single tile pair: the main kernel has written dq itself
+            if (more) ref_next = find_tile(cu, tile_prefix, n_seqs, t_next);
+            continue;
+        }
         const float4* src = reinterpret_cast<const float4*>(dq_acc + ((size_t)t * n_heads + h) * (kTile * D));
-        for (int e = threadIdx.x; e < kTile * D / 4; e += blockDim.x) {
-            const int c4 = e / kTile, r = e % kTile;
-            const float4 v = src[e];
-            __nv_bfloat162 lo2 = __floats2bfloat162_rn(v.x * scale, v.y * scale);
-            __nv_bfloat162 hi2 = __floats2bfloat162_rn(v.z * scale, v.w * scale);
-            uint2 pk;
-            pk.x = *reinterpret_cast<uint32_t*>(&lo2);
-            pk.y = *reinterpret_cast<uint32_t*>(&hi2);
-            *reinterpret_cast<uint2*>(tile + r * kRowBytes + c4 * 8) = pk;
+        // eight 16-byte loads in flight per thread before the first use (the kernel waits on HBM latency), and the
+        // next block's tile is looked up while the first eight are in flight
+        for (int e0 = threadIdx.x; e0 < kTile * D / 4; e0 += 8 * 256) {
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = src[e0 + u * 256];
+            if (e0 == (int)threadIdx.x && more) ref_next = find_tile(cu, tile_prefix, n_seqs, t_next);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int e = e0 + u * 256, c4 = e / kTile, r = e % kTile;
+                __nv_bfloat162 lo2 = __floats2bfloat162_rn(v[u].x * scale, v[u].y * scale);
+                __nv_bfloat162 hi2 = __floats2bfloat162_rn(v[u].z * scale, v[u].w * scale);
+                uint2 pk;
+                pk.x = *reinterpret_cast<uint32_t*>(&lo2);
+                pk.y = *reinterpret_cast<uint32_t*>(&hi2);
+                *reinterpret_cast<uint2*>(tile + r * kRowBytes + c4 * 8) = pk;
+            }
         }
         __syncthreads();
         const int kChunks = head_dim * 2 / 16;               // 16-byte chunks per stored row (head_dim <= D columns)
         for (int e = threadIdx.x; e < rows * kChunks; e += blockDim.x) {
             const int r = e / kChunks, c = e % kChunks;
             const uint4 v = *reinterpret_cast<const uint4*>(tile + r * kRowBytes + c * 16);
-            __nv_bfloat16* out = dq + ((size_t)cu[lo] + row0 + r) * (size_t)row_stride + (size_t)h * head_dim;
+            __nv_bfloat16* out = dq + ((size_t)ref.tok0 + row0 + r) * (size_t)row_stride + (size_t)h * head_dim;
             reinterpret_cast<uint4*>(out)[c] = v;
         }
         __syncthreads();
-        }
     }
 }
 
 cudaError_t launch_bwd_post(const float* dq_acc, __nv_bfloat16* dq, const int32_t* cu_seqlens, const SchedView& sched,
                             int32_t n_heads, int32_t head_dim, int64_t row_stride, float scale, int n_sms,
                             cudaStream_t stream) {
-    const int blocks = n_sms * 4;
+    const int blocks = n_sms * 6;
     if (head_dim > 64)
         bwd_post_kernel<128><<<blocks, 256, 0, stream>>>(dq_acc, dq, cu_seqlens, sched.tile_prefix, sched.n_seqs, n_heads,
                                                          head_dim, row_stride, scale);
