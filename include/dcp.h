@@ -234,7 +234,9 @@ int dcp_varlen_attn_fwd(const void* q, const void* k, const void* v, const int32
 /* Gradients of sum(o * d_o): q, k, v, o, d_o, lse (device, in) -> dq, dk, dv (device, out).
  * `causal` and `softmax_scale` must equal the forward call's.  workspace >= bwd_bytes; it holds
  * the fp32 dQ accumulator and the per-row D = sum_c dO*O.  dQ is summed with floating-point
- * atomics, so its low bits may differ from run to run. */
+ * atomics, so its low bits may differ from run to run.  When max_seqlen <= 32 (see
+ * dcp_set_short_sequence_path) D is formed as sum_j P_ij dP_ij instead, `o` is not read, and the
+ * result is the same from run to run. */
 int dcp_varlen_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
                         const float* lse, const int32_t* cu_seqlens, int32_t n_seqs, int32_t total_tokens,
                         int32_t max_seqlen, int32_t n_heads, int32_t head_dim, int32_t causal,
