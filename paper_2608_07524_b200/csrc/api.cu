@@ -276,10 +276,11 @@ static int attn_fwd_impl(const char* fn, bool merge, const void* q, const void* 
     g_launches.fetch_add(prep_launches(n_seqs, merge, input_order));
     if (total_tokens == 0 || n_seqs == 0) return DCP_OK;
 
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to;
     if (int rc = make_map(&tq, q, total_tokens, n_heads, head_dim, token_stride)) return rc;
     if (int rc = make_map(&tk, k, total_tokens, n_heads, head_dim, token_stride)) return rc;
     if (int rc = make_map(&tv, v, total_tokens, n_heads, head_dim, token_stride)) return rc;
+    if (int rc = make_map(&to, o, total_tokens, n_heads, head_dim, token_stride)) return rc;
 
     FwdParams p;
     p.cu_seqlens = merge ? sched.vcu : cu_seqlens;
@@ -295,7 +296,7 @@ static int attn_fwd_impl(const char* fn, bool merge, const void* q, const void* 
     p.scale_log2 = p.scale * 1.4426950408889634f;
     {
         ScopedTimer t(DCP_KERNEL_FWD, stream);
-        e = launch_attn_fwd(tq, tk, tv, p, head_dim, causal != 0, max_seqlen <= kShortItemMaxLen, dev.sm_count, stream);
+        e = launch_attn_fwd(tq, tk, tv, to, p, head_dim, causal != 0, max_seqlen <= kShortItemMaxLen, dev.sm_count, stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: attention kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(1);

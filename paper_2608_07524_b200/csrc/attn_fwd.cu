@@ -41,6 +41,7 @@ struct FwdShared {
     uint64_t kv_full[kKvStages], kv_empty[kKvStages];
     uint64_t s_full[2], p_part[2][4], o_full[2], o_free[2];
     uint64_t work_full[2], work_empty[2];
+    uint64_t stage_ready[2], stage_full[2];    // output staging buffer of a softmax group: free to write / written
     WorkItem work[2];
     uint32_t tmem_base;
     uint32_t abort_flag;
@@ -51,7 +52,9 @@ struct FwdCfg {
     static constexpr int kTileBytes = kTile * D * 2;   // one Q, K or V tile
     static constexpr int kBoxes = D / 64;               // TMA boxes per tile (64 columns = 128 bytes each)
     static constexpr int kBoxBytes = kTile * 128;
-    static constexpr int kSmemBytes = (2 + kKvStages) * kTileBytes + 1024;
+    static constexpr int kStageBytes = kTile * 128;     // 128 rows of 64 bf16 columns: what one TMA store box holds
+    static constexpr int kOffStage = (2 + kKvStages) * kTileBytes;   // one staging buffer per softmax group
+    static constexpr int kSmemBytes = kOffStage + 2 * kStageBytes + 1024;
     static constexpr uint32_t kS0 = 0, kS1 = 128, kO0 = 256, kO1 = 256 + D;   // tensor-memory columns
 };
 
@@ -204,6 +207,54 @@ __device__ __noinline__ void softmax_single_tile_item(FwdShared& sh, const FwdPa
     if (lane == 0) mbar_arrive(&sh.o_free[0]);
 }
 
+// Epilogue of a Q tile whose 128 rows all belong to the sequence: O = acc / l leaves tensor memory through a
+// staging buffer in shared memory and TMA stores, 64 columns (one box) at a time.  A thread owns a row, so storing
+// it directly costs 16 instructions of 32 scattered 16-byte pieces each, about a microsecond of the load/store
+// unit per tile: as much as a key tile's softmax, which is what short work items cannot afford (uniform batches
+// of 256-token sequences: forward 0.41 -> 0.36 ms).  Kept out of line so that the loop over key tiles is compiled
+// exactly as it would be without it (inlined it cost the long-sequence forward 6 %).  Called by the 128 threads
+// of a softmax group; n_staged = boxes this group has stored so far (the parity of its two barriers).
+template <int D>
+__device__ __noinline__ void store_whole_tile(FwdShared& sh, const CUtensorMap* tmap_o, uint8_t* stage, uint32_t o_tmem,
+                                              float inv_l, int t, int head, int tok_row0, uint32_t n_staged,
+                                              const WaitGuard guard) {
+    const int lane = threadIdx.x & 31, row_in_tile = threadIdx.x & 127;
+    const bool issuer = row_in_tile == 0;
+#pragma unroll
+    for (int half = 0; half < D / 64; ++half, ++n_staged) {
+        uint32_t acc[64];
+        tmem_ld_x32(o_tmem + half * 64, *reinterpret_cast<uint32_t(*)[32]>(&acc[0]));
+        tmem_ld_x32(o_tmem + half * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&acc[32]));
+        tmem_wait_ld();
+        if (half == D / 64 - 1) {       // O has left tensor memory: the next item's P V may start
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.o_free[t]);
+        }
+        if (issuer) {
+            bulk_store_wait_read();              // the previous store has read the staging buffer
+            mbar_arrive(&sh.stage_ready[t]);
+        }
+        mbar_wait(&sh.stage_ready[t], n_staged & 1u, guard);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            uint4 val;
+            val.x = pack_bf16x2(__uint_as_float(acc[c * 8 + 0]) * inv_l, __uint_as_float(acc[c * 8 + 1]) * inv_l);
+            val.y = pack_bf16x2(__uint_as_float(acc[c * 8 + 2]) * inv_l, __uint_as_float(acc[c * 8 + 3]) * inv_l);
+            val.z = pack_bf16x2(__uint_as_float(acc[c * 8 + 4]) * inv_l, __uint_as_float(acc[c * 8 + 5]) * inv_l);
+            val.w = pack_bf16x2(__uint_as_float(acc[c * 8 + 6]) * inv_l, __uint_as_float(acc[c * 8 + 7]) * inv_l);
+            *reinterpret_cast<uint4*>(stage + sw128_offset((uint32_t)row_in_tile, (uint32_t)c)) = val;
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.stage_full[t]);
+        if (issuer) {
+            if (mbar_wait(&sh.stage_full[t], n_staged & 1u, guard)) tma_store_3d(tmap_o, stage, half * 64, head, tok_row0);
+            bulk_store_commit();
+        }
+    }
+}
+
 // EARLY_Q: release a Q tile's slot as soon as its last S product has been issued (see the MMA warp).
 // TRIM: head_dim is at most D - 16, so the products skip the zero-padded columns: S sums over
 // ceil(head_dim / 16) steps instead of D / 16 and O is 16 * ceil(head_dim / 16) columns wide (head_dim 72,
@@ -211,7 +262,8 @@ __device__ __noinline__ void softmax_single_tile_item(FwdShared& sh, const FwdPa
 template <int D, bool CAUSAL, bool EARLY_Q, bool TRIM>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ FwdParams p) {
+                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
+                const __grid_constant__ FwdParams p) {
     using Cfg = FwdCfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -234,6 +286,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             mbar_init(&sh.o_free[i], 4);
             mbar_init(&sh.work_full[i], 1);
             mbar_init(&sh.work_empty[i], 9);   // 8 softmax warps + the MMA thread
+            mbar_init(&sh.stage_ready[i], 1);
+            mbar_init(&sh.stage_full[i], 4);   // one arrival per warp of the group
         }
         for (int i = 0; i < kKvStages; ++i) {
             mbar_init(&sh.kv_full[i], 1);
@@ -405,7 +459,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t s_tmem = tmem + lane_base + (t == 0 ? Cfg::kS0 : Cfg::kS1);
         const uint32_t o_tmem = tmem + lane_base + (t == 0 ? Cfg::kO0 : Cfg::kO1);
-        uint32_t n_work = 0, n_s = 0, use = 0;
+        uint32_t n_work = 0, n_s = 0, use = 0, n_staged = 0;
         while (true) {
             const uint32_t slot = n_work & 1u;
             const bool got = mbar_wait(&sh.work_full[slot], (n_work >> 1) & 1u, guard);
@@ -529,6 +583,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             const float inv_l = 1.0f / l;
             const bool valid = row < w.len;
             const size_t tok = (size_t)w.tok0 + (size_t)row;
+            if (r_tile + kTile <= w.len) {
+                // every row of the tile belongs to the sequence: it leaves through shared memory and TMA stores
+                store_whole_tile<D>(sh, &tmap_o, smem + Cfg::kOffStage + t * Cfg::kStageBytes, o_tmem, inv_l, t, w.head,
+                                    w.tok0 + r_tile, n_staged, guard);
+                n_staged += D / 64;
+                p.lse[(size_t)w.head * p.total_tokens + tok] = m * p.scale + __logf(l);
+                continue;
+            }
             __nv_bfloat16* out = p.o + tok * p.row_stride + w.head * p.head_dim;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
@@ -552,6 +614,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.o_free[t]);
         }
+        if ((tid & 127) == 0) bulk_store_wait_all();     // this group's stores are complete before the CTA ends
     }
 
     tc_fence_before();
@@ -561,28 +624,28 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 }
 
 template <int D, bool CAUSAL, bool EARLY_Q, bool TRIM>
-static cudaError_t launch_one(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
-                              int n_ctas, cudaStream_t stream) {
+static cudaError_t launch_one(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                              const FwdParams& p, int n_ctas, cudaStream_t stream) {
     auto kern = attn_fwd_kernel<D, CAUSAL, EARLY_Q, TRIM>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<D>::kSmemBytes);
     if (e != cudaSuccess) return e;
-    kern<<<n_ctas, kFwdThreads, FwdCfg<D>::kSmemBytes, stream>>>(tq, tk, tv, p);
+    kern<<<n_ctas, kFwdThreads, FwdCfg<D>::kSmemBytes, stream>>>(tq, tk, tv, to, p);
     return cudaGetLastError();
 }
 
 template <int D, bool TRIM>
-static cudaError_t launch_masked(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
-                                 bool causal, bool short_items, int n_ctas, cudaStream_t stream) {
-    if (causal) return launch_one<D, true, true, TRIM>(tq, tk, tv, p, n_ctas, stream);
-    return short_items ? launch_one<D, false, true, TRIM>(tq, tk, tv, p, n_ctas, stream)
-                       : launch_one<D, false, false, TRIM>(tq, tk, tv, p, n_ctas, stream);
+static cudaError_t launch_masked(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                                 const FwdParams& p, bool causal, bool short_items, int n_ctas, cudaStream_t stream) {
+    if (causal) return launch_one<D, true, true, TRIM>(tq, tk, tv, to, p, n_ctas, stream);
+    return short_items ? launch_one<D, false, true, TRIM>(tq, tk, tv, to, p, n_ctas, stream)
+                       : launch_one<D, false, false, TRIM>(tq, tk, tv, to, p, n_ctas, stream);
 }
 
-cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
-                            int head_dim, bool causal, bool short_items, int n_ctas, cudaStream_t stream) {
-    if (head_dim > 112) return launch_masked<128, false>(tq, tk, tv, p, causal, short_items, n_ctas, stream);
-    if (head_dim > 64) return launch_masked<128, true>(tq, tk, tv, p, causal, short_items, n_ctas, stream);
-    return launch_masked<64, false>(tq, tk, tv, p, causal, short_items, n_ctas, stream);
+cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                            const FwdParams& p, int head_dim, bool causal, bool short_items, int n_ctas, cudaStream_t stream) {
+    if (head_dim > 112) return launch_masked<128, false>(tq, tk, tv, to, p, causal, short_items, n_ctas, stream);
+    if (head_dim > 64) return launch_masked<128, true>(tq, tk, tv, to, p, causal, short_items, n_ctas, stream);
+    return launch_masked<64, false>(tq, tk, tv, to, p, causal, short_items, n_ctas, stream);
 }
 
 }  // namespace dcp

@@ -66,8 +66,9 @@ cudaError_t launch_copy_segments(const void* src, void* dst, const int32_t* seg,
 
 // short_items: no sequence of the batch is longer than a few dozen tiles, so work items are short and the
 // variant that releases Q slots early pays (under a causal mask it always does).
-cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
-                            int head_dim, bool causal, bool short_items, int n_ctas, cudaStream_t stream);
+// `to` = the same kind of map over o: whole tiles leave through shared memory and TMA stores.
+cudaError_t launch_attn_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                            const FwdParams& p, int head_dim, bool causal, bool short_items, int n_ctas, cudaStream_t stream);
 
 // Tile-aligned row statistics for the backward kernel (see BwdParams::stats) and dq_acc = 0.
 cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, const float* lse, const int32_t* cu_seqlens,
