@@ -444,24 +444,25 @@ def run_ours(args):
         others = {}
         del job, runner, step
         torch.cuda.empty_cache()
-        for name in WORKLOADS:
-            if name == args.workload:
+        # every other workload at head_dim 128, and the two axes of the 2-D model at the paper's own width (72)
+        for key, name, width in [(n, n, 128) for n in WORKLOADS] + [("spatial2d_d72", "spatial2d", 72), ("temporal2d_d72", "temporal2d", 72)]:
+            if name == args.workload and width == args.head_dim:
                 continue
             o_args = argparse.Namespace(**vars(args))
             o_args.drop_longer_than, o_args.longest_last = 0, False
-            o_args.layers, o_args.budget_gb, o_args.stream_batches, o_args.head_dim = 1, 180.0, 32, 128
+            o_args.layers, o_args.budget_gb, o_args.stream_batches, o_args.head_dim = 1, 180.0, 32, width
             try:
                 oj = Job(o_args, name, dev, rank)
                 n_steps = 2 if name in ("stream", "extreme") else 5
                 ms, tok, fl, _, pr = timed_steps(oj, n_steps, 3 if name != "stream" else 1, barrier)
                 v = fl / (ms * 1e-3) / 1e12
-                others[name] = {"workload": oj.desc, "steps": n_steps, "ms_per_step": ms / n_steps, "value": v, "unit": UNIT,
+                others[key] = {"workload": oj.desc, "steps": n_steps, "ms_per_step": ms / n_steps, "value": v, "unit": UNIT,
                                 "tokens_per_s": tok / (ms * 1e-3), "frac_of_bf16_peak_burst": v / peaks["burst"],
                                 "kernel_ms_per_step": {k: x[0] / n_steps for k, x in pr.items()},
                                 "sm_busy": oj.sm_busy()}
                 del oj
             except Exception as ex:
-                others[name] = {"error": str(ex)[:200]}
+                others[key] = {"error": str(ex)[:200]}
             torch.cuda.empty_cache()
 
     cpu_baseline = None
