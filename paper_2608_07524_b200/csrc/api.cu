@@ -392,6 +392,9 @@ static int attn_bwd_impl(const char* fn, const void* q, const void* k, const voi
     if (int rc = make_map(&tk, k, total_tokens, n_heads, head_dim, token_stride)) return rc;
     if (int rc = make_map(&tv, v, total_tokens, n_heads, head_dim, token_stride)) return rc;
     if (int rc = make_map(&tg, d_o, total_tokens, n_heads, head_dim, token_stride)) return rc;
+    CUtensorMap tdk, tdv;
+    if (int rc = make_map(&tdk, dk, total_tokens, n_heads, head_dim, token_stride)) return rc;
+    if (int rc = make_map(&tdv, dv, total_tokens, n_heads, head_dim, token_stride)) return rc;
 
     {
         ScopedTimer t(DCP_KERNEL_BWD_PRE, stream);
@@ -420,7 +423,7 @@ static int attn_bwd_impl(const char* fn, const void* q, const void* k, const voi
     p.scale_log2 = p.scale * 1.4426950408889634f;
     {
         ScopedTimer t(DCP_KERNEL_BWD_MAIN, stream);
-        e = launch_attn_bwd(tq, tk, tv, tg, p, head_dim, causal != 0, dev.sm_count, stream);
+        e = launch_attn_bwd(tq, tk, tv, tg, tdk, tdv, p, head_dim, causal != 0, dev.sm_count, stream);
     }
     if (e != cudaSuccess) return fail(DCP_ERR_CUDA, "%s: main kernel: %s", fn, cudaGetErrorString(e));
     g_launches.fetch_add(1);

@@ -76,8 +76,10 @@ cudaError_t launch_bwd_pre(const __nv_bfloat16* o, const __nv_bfloat16* d_o, con
                            int32_t total_tokens, int32_t n_heads, int32_t head_dim, int64_t row_stride, float scale,
                            int n_sms, cudaStream_t stream);
 
+// tdk, tdv = maps over dk and dv: whole key blocks leave through shared memory and TMA stores.
 cudaError_t launch_attn_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
-                            const BwdParams& p, int head_dim, bool causal, int n_ctas, cudaStream_t stream);
+                            const CUtensorMap& tdk, const CUtensorMap& tdv, const BwdParams& p, int head_dim, bool causal,
+                            int n_ctas, cudaStream_t stream);
 
 // dq[T, H, d] = bf16(scale * dq_acc), undoing the tile-blocked layout
 cudaError_t launch_bwd_post(const float* dq_acc, __nv_bfloat16* dq, const int32_t* cu_seqlens, const SchedView& sched,
