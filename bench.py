@@ -371,7 +371,8 @@ def run_ours(args):
         # timed region includes filling and draining the pipeline.
         runners = [runner, StreamRunner(max_tokens, max_seqs, H, d, causal, dev, value_seed=13 + 100 * rank)]
         pipe = HostPipeline(runners, T)
-        n_pipe = 4 * n_e2e       # long enough that filling and draining the pipeline is a small part
+        # long enough that filling and draining the pipeline (one step's copies in, one step's out) is a small part
+        n_pipe = min(max(4 * n_e2e, 2 * args.steps), 40)
 
         def pipeline(n):
             pipe.run(host_in, step, n)
