@@ -107,24 +107,64 @@ def dual_layer_profile(bucket_lengths: Sequence[int], n_heads: int, head_dim: in
     return ProfileTable(buckets, t_f, t_b, m)
 
 
+def _gpu_layer_head_group(n_heads: int, sp_size: int, head_dim: int, causal: bool, device) -> Callable[[List[int]], Tuple[float, float]]:
+    """One rank's share of a 'layer' under head-sharded sequence parallelism of size sp_size: forward + backward
+    on the first n_heads / sp_size heads, in place inside full-width [T, n_heads, head_dim] tensors (the strided
+    entry points, as a rank of a group runs them).  Returns (forward ms, backward ms)."""
+    import torch
+    from . import binding, inputs
+
+    def run(lengths: List[int]) -> Tuple[float, float]:
+        T, hg = sum(lengths), n_heads // sp_size
+        q, k, v, g = inputs.make_qkvg_device(T, n_heads, head_dim, 77, device)
+        o, dq, dk, dv = (torch.empty_like(q) for _ in range(4))
+        cu = torch.tensor([0] + list(torch.tensor(lengths).cumsum(0).tolist()), dtype=torch.int32, device=device)
+        hs = slice(0, hg)
+        binding.dcp_profile_enable(True)
+        binding.dcp_profile_read()
+        _, lse = binding.dcp_varlen_attn_fwd_strided(q[:, hs], k[:, hs], v[:, hs], cu, max(lengths), causal, o[:, hs])
+        torch.cuda.synchronize()
+        f = binding.dcp_profile_read()
+        binding.dcp_varlen_attn_bwd_strided(q[:, hs], k[:, hs], v[:, hs], o[:, hs], g[:, hs], lse, cu, max(lengths), causal,
+                                            dq[:, hs], dk[:, hs], dv[:, hs])
+        torch.cuda.synchronize()
+        b = binding.dcp_profile_read()
+        binding.dcp_profile_enable(False)
+        return sum(ms for ms, _ in f.values()), sum(ms for ms, _ in b.values())
+
+    return run
+
+
 def intra_candidates(seq_len: int, batch_sizes: Sequence[int], n_heads: int, head_dim: int, causal: bool, n_layers: int,
                      device="cuda", elt_bytes: int = 2, const_bytes: int = 0, fixed_cost_ns: int = 0,
-                     run_layer: Optional[Callable[[List[int]], Tuple[float, float]]] = None):
-    """The candidate table Algorithm 1 takes, for sequences of one length on one GPU: one row (b, 1) per
-    batch size b, measured the dual-layer way (the batch of b sequences runs twice, the second run is
-    kept).  Row = (b, p = 1, t_f, m, T_(b,1), M_(b,1)) with t_f the measured forward time of one layer for
-    the whole batch in ns, m = 4 b L H d e the bytes a layer keeps when it is not recomputed,
-    T = Lambda (2 t_f + t_b) + T_C the modelled time with every layer recomputed (Section 3.5) and
-    M = Lambda b L H d e + M_C (Eq. 6 at r = Lambda)."""
+                     run_layer: Optional[Callable[[List[int]], Tuple[float, float]]] = None,
+                     sp_sizes: Sequence[int] = (1,)):
+    """The candidate table Algorithm 1 takes, for sequences of one length: one row (b, p) per batch size b and
+    sequence-parallel size p, measured the dual-layer way (the batch of b sequences runs twice, the second run
+    is kept).  Row = (b, p, t_f, m, T_(b,p), M_(b,p)) with t_f the measured forward time of one layer for the
+    whole batch in ns, m the bytes a layer keeps when it is not recomputed, T = Lambda (2 t_f + t_b) + T_C the
+    modelled time with every layer recomputed (Section 3.5) and M = Lambda m_inp + M_C (Eq. 6 at r = Lambda).
+    For p > 1 a row describes ONE RANK of a head-sharded group (Section 4.1): its time is that of its
+    n_heads / p heads over all tokens, measured on this GPU through the strided entry points, and its memory
+    that of its 1 / p of the tokens.  What a row for p > 1 leaves out is the time the tiles take to cross
+    NVLink, which one GPU cannot show: the ranks of a group fetch remote tiles inside the same kernels."""
     from . import binding
-    run = run_layer if run_layer is not None else _gpu_layer(n_heads, head_dim, causal, device)
     rows = []
-    for b in batch_sizes:
-        run([seq_len] * b)                                  # first layer: warm-up, discarded
-        f_ms, b_ms = run([seq_len] * b)                     # second layer: recorded
-        act, inp = binding.dcp_activation_bytes(b * seq_len, n_heads, head_dim, elt_bytes)
-        rows.append(binding.dcp_intra_candidate_from_profile(b, 1, int(round(f_ms * 1e6)), int(round(b_ms * 1e6)), act, inp,
-                                                             n_layers, const_bytes, fixed_cost_ns))
+    for p in sp_sizes:
+        if p < 1 or n_heads % p != 0:
+            raise ValueError(f"sequence-parallel size {p} does not divide {n_heads} heads")
+        if run_layer is not None:
+            run = run_layer
+        elif p == 1:
+            run = _gpu_layer(n_heads, head_dim, causal, device)
+        else:
+            run = _gpu_layer_head_group(n_heads, p, head_dim, causal, device)
+        for b in batch_sizes:
+            run([seq_len] * b)                                  # first layer: warm-up, discarded
+            f_ms, b_ms = run([seq_len] * b)                     # second layer: recorded
+            act, inp = binding.dcp_activation_bytes(-(-b * seq_len // p), n_heads, head_dim, elt_bytes)
+            rows.append(binding.dcp_intra_candidate_from_profile(b, p, int(round(f_ms * 1e6)), int(round(b_ms * 1e6)), act, inp,
+                                                                 n_layers, const_bytes, fixed_cost_ns))
     return rows
 
 

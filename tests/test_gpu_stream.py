@@ -158,3 +158,26 @@ def test_algorithm_1_setting_measured_on_the_device_and_applied():
     close("dk", runner.dk[:T], rdk)
     close("dv", runner.dv[:T], rdv)
     assert float(np.max(np.abs(runner.lse[: H * T].view(H, T).double().cpu().numpy() - Lse))) <= LSE_ABS
+
+
+def test_algorithm_1_candidates_over_batch_size_and_sequence_parallel_size():
+    """Algorithm 1's table with both of its dimensions: rows (b, p) for p = 1, 2, 4, each measured on this device
+    as one rank's share (its heads of all tokens, in place inside full-width tensors; what crosses NVLink is
+    not in a one-GPU measurement).  The selection is compared with the exhaustive oracle on the SAME table, with
+    room for everything and with so little memory that only a sharded setting fits."""
+    L, heads, lam = 8192, 16, 4                       # enough work that a quarter of the heads takes visibly less time
+    cands = intra_candidates(L, [1, 2], heads, 128, False, lam, fixed_cost_ns=20000, sp_sizes=(1, 2, 4))
+    assert [(c[0], c[1]) for c in cands] == [(1, 1), (2, 1), (1, 2), (2, 2), (1, 4), (2, 4)]
+    assert all(c[2] > 0 and c[4] > 0 for c in cands)
+    by = {(c[0], c[1]): c for c in cands}
+    for b in (1, 2):                                   # a rank of a larger group holds less and works less
+        assert by[(b, 1)][5] > by[(b, 2)][5] > by[(b, 4)][5]
+        assert by[(b, 1)][2] > by[(b, 4)][2]
+    roomy = 1 << 40
+    idx, r, t = B.dcp_intra_select(cands, roomy, lam)
+    assert (idx, r, t) == oracle.intra_select(cands, roomy, lam) and r == 0
+    # less than any p = 1 row needs even with every layer recomputed; (1, 2), (1, 4) and (2, 4) still fit
+    tight = min(by[(1, 1)][5], by[(2, 1)][5]) - 1
+    assert tight >= by[(1, 2)][5] and tight >= by[(2, 4)][5]
+    idx, r, t = B.dcp_intra_select(cands, tight, lam)
+    assert (idx, r, t) == oracle.intra_select(cands, tight, lam) and cands[idx][1] >= 2
