@@ -261,6 +261,32 @@ class Job:
         return out
 
 
+def virtual_rank_balance(dev, world: int = 8, n_global: int = 2):
+    """Section 2.3 / 4.2 of the paper on one GPU: the imbalance ratio (slowest rank's time over the mean) of `world`
+    data-parallel ranks, with every rank's forward + backward MEASURED on this GPU one after the other.  A global
+    step is `world` batches of the stream; `as_drawn` gives rank r batch r, `sharded` deals all their sequences out
+    with the library's dcp_shard_sequences (longest first to the least loaded rank, load = L^2)."""
+    from paper_2608_07524_b200 import inputs
+    from paper_2608_07524_b200.profiler import _gpu_layer
+    from paper_2608_07524_b200.shard import shard_sequences, imbalance
+    run = _gpu_layer(16, 128, False, dev)
+    batches = inputs.stream_batches()[: world * n_global]
+    out = {"as_drawn": [], "sharded": [], "sharded_model": []}
+    run(batches[0])                                              # warm-up
+    for gstep in range(n_global):
+        group = batches[gstep * world:(gstep + 1) * world]
+        everything = [L for b in group for L in b]
+        owned = shard_sequences(everything, world)
+        for key, parts in (("as_drawn", group), ("sharded", [[everything[i] for i in idx] for idx in owned])):
+            times = [sum(run(list(part))) if part else 0.0 for part in parts]
+            out[key].append(max(times) / (sum(times) / len(times)))
+        out["sharded_model"].append(imbalance(everything, world))
+    return {"workload": f"{n_global} global steps of {world} stream batches (24 sequences each), every rank's fwd + bwd timed on this GPU",
+            "ranks": world, "max_over_mean_as_drawn": sum(out["as_drawn"]) / n_global,
+            "max_over_mean_sharded": sum(out["sharded"]) / n_global,
+            "max_over_mean_sharded_by_the_L2_model": sum(out["sharded_model"]) / n_global}
+
+
 def timed_steps(job, steps, warmup, barrier):
     """(ms over `steps` steps, tokens, flops, launches, per-kernel profile) after `warmup` untimed steps."""
     import torch
@@ -465,6 +491,11 @@ def run_ours(args):
             except Exception as ex:
                 others[key] = {"error": str(ex)[:200]}
             torch.cuda.empty_cache()
+        try:
+            others["balance_w8"] = virtual_rank_balance(dev)
+        except Exception as ex:
+            others["balance_w8"] = {"error": str(ex)[:200]}
+        torch.cuda.empty_cache()
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:

@@ -60,5 +60,8 @@ def test_cuda_arm_prints_the_contract_line():
     assert base["kind"] == "oracle" and base["value"] > 0 and base["cores"] >= 1
     busy = line["sm_busy"]
     assert busy["fwd"]["ctas"] > 0 and busy["bwd_main"]["max_over_mean"] >= 1.0
-    assert set(line["others"]) == {"video", "extreme", "stream", "spatial2d", "temporal2d", "spatial2d_d72", "temporal2d_d72"}
+    assert set(line["others"]) == {"video", "extreme", "stream", "spatial2d", "temporal2d", "spatial2d_d72", "temporal2d_d72",
+                                   "balance_w8"}
+    balance = line["others"].pop("balance_w8")
+    assert 1.0 <= balance["max_over_mean_sharded"] <= balance["max_over_mean_as_drawn"]
     assert all("error" not in o and o["value"] > 0 for o in line["others"].values())
