@@ -524,6 +524,50 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_uniform(args):
+    """Not the contract line: one JSON line per sequence length for batches of equal sequences (131072 tokens, 16
+    heads of --head-dim, bidirectional), forward + backward, with the per-kernel times.  It shows where the paths
+    change (short-sequence kernels up to 32 tokens, one tile per sequence up to 128, work items of growing
+    length after that) and what each costs against the HBM and tensor rooflines."""
+    import torch
+    from paper_2608_07524_b200 import binding as B
+    dev, H, d, total = "cuda:0", 16, args.head_dim, 131072
+    torch.cuda.set_device(0)
+    for L in [int(x) for x in args.uniform.split(",")]:
+        n = max(1, total // L)
+        T = n * L
+        cu = torch.arange(0, T + 1, L, dtype=torch.int32, device=dev)
+        q, k, v, g = (torch.randn(T, H, d, device=dev, dtype=torch.bfloat16) for _ in range(4))
+        ws = B.alloc_workspace(T, n, H, d, True, dev)
+        o, dq, dk, dv = (torch.empty_like(q) for _ in range(4))
+        lse = torch.empty(H, T, device=dev)
+
+        def step():
+            B.dcp_varlen_attn_fwd(q, k, v, cu, L, False, 0.0, out=o, lse=lse, workspace=ws)
+            B.dcp_varlen_attn_bwd(q, k, v, o, g, lse, cu, L, False, 0.0, dq=dq, dk=dk, dv=dv, workspace=ws)
+
+        for _ in range(max(args.warmup, 3)):
+            step()
+        B.dcp_query_status(ws)
+        B.dcp_profile_enable(True)
+        B.dcp_profile_read()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        prof = B.dcp_profile_read()
+        B.dcp_profile_enable(False)
+        ms = e0.elapsed_time(e1) / args.steps
+        print(json.dumps({"uniform_tokens_per_sequence": L, "sequences": n, "tokens": T, "heads": H, "head_dim": d,
+                          "ms_per_step": ms, "tflops": 14.0 * n * L * L * d * H / (ms * 1e-3) / 1e12,
+                          "algorithmic_gb_per_s": T * H * (12 * d * 2 + 12) / (ms * 1e-3) / 1e9,
+                          "kernel_ms_per_step": {k_: x[0] / args.steps for k_, x in prof.items()}}), flush=True)
+        del q, k, v, g, o, dq, dk, dv, lse, ws
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -547,8 +591,12 @@ def main():
     ap.add_argument("--no-others", action="store_true", help="skip the short runs of the other workloads")
     ap.add_argument("--drop-longer-than", type=int, default=0,
                     help="profiling aid: drop sequences longer than this from the workload (0 = keep all)")
+    ap.add_argument("--uniform", default="", metavar="L[,L...]",
+                    help="instead of the contract line: batches of equal sequences of these lengths, one JSON line each")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.uniform:
+        run_uniform(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
